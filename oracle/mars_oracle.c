@@ -1,0 +1,301 @@
+/*
+ * mars_oracle.c -- TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, single-pass-per-row CPU statement of margin-aware speculative
+ * verification (MARS), written from the paper's text:
+ *   - top-2 tokens of a logits row and the logit ratio r = z(2)/z(1)   (Sec. 3.3, Eq. 4)
+ *   - three-way rule: exact match / adaptive relaxation / rejection     (Sec. 3.4)
+ *   - chain verification loop with stop at the first failure            (Algorithm 1)
+ *   - bonus token when every draft is accepted                          (Table 1 caption)
+ *   - token-tree form of the same rule                                  (Sec. 2.3)
+ *   - logits from the output projection z = W_o h + b_o                 (Eq. 2; logits
+ *     are produced by the Python wrapper with an fp64 matmul, the rule below then
+ *     runs on double rows)
+ *
+ * Only tests, the smoke check and the benchmark's CPU-baseline leg may call this file.
+ * It shares no code, header, table or helper with the CUDA library.
+ *
+ * Precision: the paper never states one.  Decisions on stored logits are taken in
+ * fp32: bf16 widens exactly to fp32, every comparison is an IEEE fp32 comparison and
+ * the ratio is one round-to-nearest fp32 division.  Build with
+ *   gcc -O2 -fno-fast-math -ffp-contract=off -fopenmp -shared -fPIC
+ * The "_f64" entry points take the same decisions in fp64 on double logits.
+ *
+ * Readings where the paper is silent (each is a convention of this repository):
+ *   - threshold is strict: r == theta rejects (the paper writes r > theta throughout);
+ *   - sign guard: relaxation needs z(1) > 0 unless MARS_ORACLE_SIGN_LITERAL is set;
+ *     with the guard, r > theta agrees with the paper's equivalent margin form
+ *     Delta < (1-theta) z(1) (Eq. 6) for every sign when theta < 1;
+ *   - total order on a row: larger value first, lower token id first among equal
+ *     values (IEEE ==, so -0 == +0); NaN counts as -inf;
+ *   - tree: node i>0 is accepted iff its parent is accepted and tok[i] passes the
+ *     three-way rule on the parent's row; the result is the deepest accepted node,
+ *     lowest node index among equally deep ones; the emitted next token is the top-1
+ *     of that node's row.
+ *   Pinned by tests against: a sort-based top-2, the paper's Fig. 2 worked example,
+ *   planted ratios one ulp around theta, strict-greedy equivalence for theta >= 1,
+ *   brute-force path enumeration on all small trees, closed-form acceptance rates.
+ *   Parity unpinned by the paper (conventions only): the sign guard, NaN handling,
+ *   the tie rules (equal logits; equally deep accepted paths).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define MARS_ORACLE_SIGN_LITERAL 1u
+#define MARS_ORACLE_SHARED_PARENT 2u
+
+enum { ORACLE_BF16 = 0, ORACLE_FP32 = 1, ORACLE_FP64 = 2 };
+
+int mars_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* bf16 is the upper half of an fp32 word: widening is exact. */
+static float bf16_to_f32(uint16_t h)
+{
+    uint32_t w = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return f;
+}
+
+/* ---- total order on (value, token id): Sec. 3.3 names z(1) >= z(2); ties by id ---- */
+static int beats_f32(float ax, int64_t aj, float bx, int64_t bj)
+{
+    return (ax > bx) || (ax == bx && aj < bj);
+}
+static int beats_f64(double ax, int64_t aj, double bx, int64_t bj)
+{
+    return (ax > bx) || (ax == bx && aj < bj);
+}
+
+/*
+ * Top-2 of one row (Algorithm 1, "identify top-2 tokens"; Sec. 3.3).
+ * get(j) is the j-th logit widened to the decision type, NaN mapped to -inf.
+ */
+#define DEFINE_TOP2(NAME, T, BEATS, NEG_INF)                                            \
+    static void NAME(const void *row, int dtype, int64_t V, T *val2, int32_t *id2)      \
+    {                                                                                   \
+        T bx = 0, sx = 0;                                                               \
+        int64_t bj = -1, sj = -1;                                                       \
+        for (int64_t j = 0; j < V; ++j) {                                               \
+            T x;                                                                        \
+            if (dtype == ORACLE_BF16) x = (T)bf16_to_f32(((const uint16_t *)row)[j]);   \
+            else if (dtype == ORACLE_FP32) x = (T)((const float *)row)[j];              \
+            else x = (T)((const double *)row)[j];                                       \
+            if (x != x) x = NEG_INF;                                                    \
+            if (bj < 0 || BEATS(x, j, bx, bj)) {                                        \
+                sx = bx; sj = bj;                                                       \
+                bx = x;  bj = j;                                                        \
+            } else if (sj < 0 || BEATS(x, j, sx, sj)) {                                 \
+                sx = x;  sj = j;                                                        \
+            }                                                                           \
+        }                                                                               \
+        val2[0] = bx + (T)0; val2[1] = sx + (T)0; /* -0 -> +0 */                        \
+        id2[0] = (int32_t)bj; id2[1] = (int32_t)sj;                                     \
+    }
+
+DEFINE_TOP2(top2_row_f32, float, beats_f32, -INFINITY)
+DEFINE_TOP2(top2_row_f64, double, beats_f64, -INFINITY)
+
+/* Eq. 4 and the "Adaptive Relaxation" condition r > theta, one IEEE division. */
+int mars_oracle_relax_f32(float z1, float z2, float theta, uint32_t flags)
+{
+    int guard = (flags & MARS_ORACLE_SIGN_LITERAL) ? 1 : (z1 > 0.0f);
+    volatile float r = z2 / z1;
+    return guard && (r > theta);
+}
+int mars_oracle_relax_f64(double z1, double z2, double theta, uint32_t flags)
+{
+    int guard = (flags & MARS_ORACLE_SIGN_LITERAL) ? 1 : (z1 > 0.0);
+    volatile double r = z2 / z1;
+    return guard && (r > theta);
+}
+
+/* The three-way rule for one draft token against one row's top-2 (Sec. 3.4).
+ * Returns 1 exact match, 2 relaxed accept, 0 reject. */
+static int rule(int32_t t, const int32_t *id2, int relax)
+{
+    if (t < 0) return 0;
+    if (t == id2[0]) return 1;
+    if (t == id2[1] && relax) return 2;
+    return 0;
+}
+
+/*
+ * Top-2 of R rows.  Rows are independent; the loop over rows may run on several
+ * host threads, the scan of a row is always the sequential one above.
+ *   logits : [R, ld] of dtype (0 bf16, 1 fp32, 2 fp64); only the first V of a row are read
+ *   val    : [R,2] float (dtype 0/1) or double (dtype 2);  id : [R,2]
+ */
+void mars_oracle_top2(const void *logits, int dtype, int64_t ld, int64_t R, int64_t V,
+                      void *val, int32_t *id)
+{
+    size_t e = dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < R; ++r) {
+        const char *row = (const char *)logits + (size_t)r * (size_t)ld * e;
+        if (dtype == ORACLE_FP64) top2_row_f64(row, dtype, V, (double *)val + 2 * r, id + 2 * r);
+        else top2_row_f32(row, dtype, V, (float *)val + 2 * r, id + 2 * r);
+    }
+}
+
+static void fill(int32_t *p, int n, int32_t v)
+{
+    if (!p) return;
+    for (int i = 0; i < n; ++i) p[i] = v;
+}
+
+/*
+ * Tree resolve for ONE sequence from per-row top-2 records (Sec. 2.3 names the tree,
+ * Sec. 3.4 / Algorithm 1 give the per-token decision and the stop at the first failure).
+ *   relax[i]   : adaptive-relaxation bit of row i
+ *   tok[i]     : draft token at node i (tok[0] ignored); parent[i] < i, parent[0] = -1
+ *   outputs    : accept_len, out_tokens[Dcap+1], path_nodes[Dcap+1] (may be NULL),
+ *                out_len, status, node_flags[N] (may be NULL)
+ */
+static void resolve_tree(const int32_t *id /*[N,2]*/, const uint8_t *relax, const int32_t *tok,
+                         const int32_t *parent, int N, int Dcap, int32_t *accept_len,
+                         int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
+                         int32_t *status, uint8_t *node_flags, int32_t *depth /*scratch[N]*/,
+                         uint8_t *acc /*scratch[N]*/)
+{
+    int st = 0;
+    if (parent[0] != -1) st = 1;
+    for (int i = 1; i < N && !st; ++i)
+        if (parent[i] >= i || parent[i] < -1) st = 1;
+
+    int best = 0;
+    if (!st) {
+        acc[0] = 1; depth[0] = 0;
+        if (node_flags) node_flags[0] = 4;
+        for (int i = 1; i < N; ++i) {
+            int p = parent[i];
+            int how = 0;
+            if (p >= 0) how = rule(tok[i], id + 2 * p, relax[p]);
+            acc[i] = (uint8_t)(p >= 0 && acc[p] && how != 0);
+            depth[i] = p >= 0 ? depth[p] + 1 : 0;
+            if (node_flags) node_flags[i] = (uint8_t)((how == 1 ? 1 : 0) | (how == 2 ? 2 : 0) | (acc[i] ? 4 : 0));
+            /* deepest accepted node; strict > keeps the lowest index among equals */
+            if (acc[i] && depth[i] > depth[best]) best = i;
+        }
+        if (depth[best] > Dcap) st = 2;
+    }
+    fill(out_tokens, Dcap + 1, -1);
+    fill(path_nodes, Dcap + 1, -1);
+    if (st) {
+        if (node_flags) { memset(node_flags, 0, (size_t)N); node_flags[0] = 4 | 8; }
+        *accept_len = 0; *out_len = 1;
+        out_tokens[0] = id[0];
+        if (path_nodes) path_nodes[0] = 0;
+        if (status) *status = st;
+        return;
+    }
+    int a = depth[best];
+    for (int n = best, d = a; d >= 0; --d, n = parent[n]) {
+        if (d > 0) out_tokens[d - 1] = tok[n];
+        if (path_nodes) path_nodes[d] = n;
+        if (node_flags) node_flags[n] |= 8;
+    }
+    out_tokens[a] = id[2 * best]; /* correction token, or the bonus token at a leaf */
+    *accept_len = a; *out_len = a + 1;
+    if (status) *status = 0;
+}
+
+/*
+ * Whole path, tree form.  logits [B*N, ld]; tok [B,N]; parent [B,N] (or [N] with
+ * MARS_ORACLE_SHARED_PARENT); outputs as resolve_tree, per sequence.
+ * dbg_val [B*N,2] / dbg_id [B*N,2] / node_flags [B,N] may be NULL.
+ * dtype 2 (double logits) takes every decision in fp64.
+ * scratch: caller-provided, B*N*(8+8+8) bytes is ample.
+ */
+void mars_oracle_verify_tree(const void *logits, int dtype, int64_t ld, const int32_t *tok,
+                             const int32_t *parent, int B, int N, int64_t V, double theta,
+                             uint32_t flags, int Dcap, int32_t *accept_len, int32_t *out_tokens,
+                             int32_t *path_nodes, int32_t *out_len, int32_t *status,
+                             void *dbg_val, int32_t *dbg_id, uint8_t *node_flags, void *val_buf,
+                             int32_t *id_buf, uint8_t *relax_buf, int32_t *depth_buf,
+                             uint8_t *acc_buf)
+{
+    int64_t R = (int64_t)B * N;
+    mars_oracle_top2(logits, dtype, ld, R, V, val_buf, id_buf);
+    for (int64_t r = 0; r < R; ++r) {
+        if (dtype == ORACLE_FP64) {
+            const double *v = (const double *)val_buf + 2 * r;
+            relax_buf[r] = (uint8_t)mars_oracle_relax_f64(v[0], v[1], theta, flags);
+            if (dbg_val) { ((double *)dbg_val)[2 * r] = v[0]; ((double *)dbg_val)[2 * r + 1] = v[1]; }
+        } else {
+            const float *v = (const float *)val_buf + 2 * r;
+            relax_buf[r] = (uint8_t)mars_oracle_relax_f32(v[0], v[1], (float)theta, flags);
+            if (dbg_val) { ((float *)dbg_val)[2 * r] = v[0]; ((float *)dbg_val)[2 * r + 1] = v[1]; }
+        }
+        if (dbg_id) { dbg_id[2 * r] = id_buf[2 * r]; dbg_id[2 * r + 1] = id_buf[2 * r + 1]; }
+    }
+    for (int b = 0; b < B; ++b) {
+        const int32_t *par = (flags & MARS_ORACLE_SHARED_PARENT) ? parent : parent + (size_t)b * N;
+        resolve_tree(id_buf + 2 * (size_t)b * N, relax_buf + (size_t)b * N, tok + (size_t)b * N, par,
+                     N, Dcap, accept_len + b, out_tokens + (size_t)b * (Dcap + 1),
+                     path_nodes ? path_nodes + (size_t)b * (Dcap + 1) : NULL, out_len + b,
+                     status ? status + b : NULL, node_flags ? node_flags + (size_t)b * N : NULL,
+                     depth_buf, acc_buf);
+    }
+}
+
+/*
+ * Whole path, chain form: a literal walk of Algorithm 1 over K rows and K-1 drafts.
+ * Row i is the target's distribution for draft i; if every draft is accepted the last
+ * row supplies the bonus token (Table 1 caption), so out_len <= K.
+ *   draft [B,K-1]; out_tokens [B,K] padded with -1.
+ */
+void mars_oracle_verify_chain(const void *logits, int dtype, int64_t ld, const int32_t *draft,
+                              int B, int K, int64_t V, double theta, uint32_t flags,
+                              int32_t *accept_len, int32_t *out_tokens, int32_t *out_len,
+                              void *dbg_val, int32_t *dbg_id, void *val_buf, int32_t *id_buf)
+{
+    int64_t R = (int64_t)B * K;
+    mars_oracle_top2(logits, dtype, ld, R, V, val_buf, id_buf);
+    if (dbg_id) memcpy(dbg_id, id_buf, (size_t)R * 2 * sizeof(int32_t));
+    if (dbg_val) memcpy(dbg_val, val_buf, (size_t)R * 2 * (dtype == ORACLE_FP64 ? 8 : 4));
+    for (int b = 0; b < B; ++b) {
+        int32_t *out = out_tokens + (size_t)b * K;
+        fill(out, K, -1);
+        int n = 0, stopped = 0;
+        for (int i = 0; i < K - 1 && !stopped; ++i) {
+            int64_t r = (int64_t)b * K + i;
+            int relax;
+            if (dtype == ORACLE_FP64) {
+                const double *v = (const double *)val_buf + 2 * r;
+                relax = mars_oracle_relax_f64(v[0], v[1], theta, flags);
+            } else {
+                const float *v = (const float *)val_buf + 2 * r;
+                relax = mars_oracle_relax_f32(v[0], v[1], (float)theta, flags);
+            }
+            int32_t t = draft[(size_t)b * (K - 1) + i];
+            if (t >= 0 && t == id_buf[2 * r]) {
+                out[n++] = t;                       /* exact match: keep draft */
+            } else if (t >= 0 && t == id_buf[2 * r + 1] && relax) {
+                out[n++] = t;                       /* adaptive relaxation: keep draft */
+            } else {
+                out[n++] = id_buf[2 * r];           /* correction: target top-1, stop */
+                stopped = 1;
+            }
+        }
+        if (stopped) {
+            accept_len[b] = n - 1;
+        } else {
+            accept_len[b] = n;
+            out[n++] = id_buf[2 * ((int64_t)b * K + (K - 1))]; /* bonus token */
+        }
+        out_len[b] = n;
+    }
+}

@@ -1,0 +1,185 @@
+"""ctypes front end of the CPU oracle (TEST INFRASTRUCTURE, not a product path).
+
+Builds ``mars_oracle.c`` with gcc on first use and exposes numpy-level calls for the
+tests, the smoke check and the benchmark's CPU-baseline leg.  Nothing here imports, or
+is imported by, the CUDA library or its Python binding.
+
+Arrays: logits are numpy arrays of shape [R, ld] holding bf16 bit patterns
+(``uint16``), ``float32`` or ``float64``; token / parent arrays are ``int32``.
+
+The one piece of arithmetic done here rather than in C is the output projection
+z = W_o h + b_o (Eq. 2 of the paper), evaluated as an fp64 numpy matmul.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mars_oracle.c")
+_LIB = os.path.join(_HERE, "libmars_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+SIGN_LITERAL = 1
+SHARED_PARENT = 2
+
+_DT = {np.dtype(np.uint16): 0, np.dtype(np.float32): 1, np.dtype(np.float64): 2}
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (no fast-math, no FMA contraction, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-std=c11", "-O2", "-fno-fast-math", "-ffp-contract=off", "-fopenmp",
+               "-shared", "-fPIC", "-Wall", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            L = ctypes.CDLL(_LIB)
+            vp, i32, i64, u32, f64 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
+                                      ctypes.c_uint32, ctypes.c_double)
+            L.mars_oracle_threads.restype = ctypes.c_int
+            L.mars_oracle_top2.argtypes = [vp, i32, i64, i64, i64, vp, vp]
+            L.mars_oracle_top2.restype = None
+            L.mars_oracle_relax_f32.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float, u32]
+            L.mars_oracle_relax_f32.restype = ctypes.c_int
+            L.mars_oracle_relax_f64.argtypes = [f64, f64, f64, u32]
+            L.mars_oracle_relax_f64.restype = ctypes.c_int
+            L.mars_oracle_verify_tree.argtypes = [vp, i32, i64, vp, vp, i32, i32, i64, f64, u32,
+                                                  i32] + [vp] * 13
+            L.mars_oracle_verify_tree.restype = None
+            L.mars_oracle_verify_chain.argtypes = [vp, i32, i64, vp, i32, i32, i64, f64, u32] + [vp] * 7
+            L.mars_oracle_verify_chain.restype = None
+            _lib = L
+    return _lib
+
+
+def threads() -> int:
+    """Host threads the row loop will use (OpenMP default)."""
+    return int(lib().mars_oracle_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check_logits(logits, V):
+    if logits.ndim != 2 or not logits.flags.c_contiguous or logits.dtype not in _DT:
+        raise ValueError("logits must be a C-contiguous [R, ld] array of uint16/float32/float64")
+    V = logits.shape[1] if V is None else int(V)
+    if V < 2 or V > logits.shape[1]:
+        raise ValueError("need 2 <= V <= ld")
+    return _DT[logits.dtype], V
+
+
+def top2(logits: np.ndarray, V: int | None = None):
+    """Per-row top-2 (values [R,2], ids [R,2]) under (value desc, id asc), NaN = -inf."""
+    dt, V = _check_logits(logits, V)
+    R, ld = logits.shape
+    val = np.empty((R, 2), np.float64 if dt == 2 else np.float32)
+    idx = np.empty((R, 2), np.int32)
+    lib().mars_oracle_top2(_p(logits), dt, ld, R, V, _p(val), _p(idx))
+    return val, idx
+
+
+def relax(z1, z2, theta, flags: int = 0, fp64: bool = False) -> bool:
+    """Adaptive-relaxation bit for one row: sign guard and r = z2/z1 > theta."""
+    if fp64:
+        return bool(lib().mars_oracle_relax_f64(float(z1), float(z2), float(theta), flags))
+    return bool(lib().mars_oracle_relax_f32(float(z1), float(z2), float(theta), flags))
+
+
+def verify_tree(logits, tok, parent, theta, flags: int = 0, Dcap: int | None = None,
+                V: int | None = None) -> dict:
+    """Tree verification of B sequences of N nodes; see mars_oracle.c for the rule."""
+    dt, V = _check_logits(logits, V)
+    tok = np.ascontiguousarray(tok, np.int32)
+    parent = np.ascontiguousarray(parent, np.int32)
+    B, N = tok.shape
+    if parent.ndim == 1:
+        flags |= SHARED_PARENT
+    elif flags & SHARED_PARENT:
+        raise ValueError("SHARED_PARENT needs a 1-D parent array")
+    if logits.shape[0] != B * N or parent.shape[-1] != N:
+        raise ValueError("shape mismatch")
+    if Dcap is None:
+        Dcap = N - 1
+    out = {
+        "accept_len": np.empty(B, np.int32),
+        "out_tokens": np.empty((B, Dcap + 1), np.int32),
+        "path_nodes": np.empty((B, Dcap + 1), np.int32),
+        "out_len": np.empty(B, np.int32),
+        "seq_status": np.empty(B, np.int32),
+        "top2_val": np.empty((B * N, 2), np.float64 if dt == 2 else np.float32),
+        "top2_id": np.empty((B * N, 2), np.int32),
+        "node_flags": np.empty((B, N), np.uint8),
+    }
+    val = np.empty((B * N, 2), np.float64)
+    idb = np.empty((B * N, 2), np.int32)
+    rl = np.empty(B * N, np.uint8)
+    dp = np.empty(N, np.int32)
+    ac = np.empty(N, np.uint8)
+    lib().mars_oracle_verify_tree(_p(logits), dt, logits.shape[1], _p(tok), _p(parent), B, N, V,
+                                  float(theta), flags, Dcap, _p(out["accept_len"]),
+                                  _p(out["out_tokens"]), _p(out["path_nodes"]), _p(out["out_len"]),
+                                  _p(out["seq_status"]), _p(out["top2_val"]), _p(out["top2_id"]),
+                                  _p(out["node_flags"]), _p(val), _p(idb), _p(rl), _p(dp), _p(ac))
+    return out
+
+
+def verify_chain(logits, draft, theta, flags: int = 0, V: int | None = None) -> dict:
+    """Chain verification (Algorithm 1 plus the bonus token): K rows, K-1 drafts."""
+    dt, V = _check_logits(logits, V)
+    draft = np.ascontiguousarray(draft, np.int32)
+    B, Km1 = draft.shape
+    K = Km1 + 1
+    if logits.shape[0] != B * K:
+        raise ValueError("shape mismatch")
+    out = {
+        "accept_len": np.empty(B, np.int32),
+        "out_tokens": np.empty((B, K), np.int32),
+        "out_len": np.empty(B, np.int32),
+        "top2_val": np.empty((B * K, 2), np.float64 if dt == 2 else np.float32),
+        "top2_id": np.empty((B * K, 2), np.int32),
+    }
+    val = np.empty((B * K, 2), np.float64)
+    idb = np.empty((B * K, 2), np.int32)
+    lib().mars_oracle_verify_chain(_p(logits), dt, logits.shape[1], _p(draft), B, K, V,
+                                   float(theta), flags, _p(out["accept_len"]),
+                                   _p(out["out_tokens"]), _p(out["out_len"]), _p(out["top2_val"]),
+                                   _p(out["top2_id"]), _p(val), _p(idb))
+    return out
+
+
+def bf16_bits_to_f64(a: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns (uint16) to float64."""
+    return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def lmhead_logits(hidden_bits: np.ndarray, w_bits: np.ndarray, bias=None) -> np.ndarray:
+    """z = W_o h + b_o (Eq. 2) in fp64 from bf16 operands: hidden [M,d], w [V,d] -> [M,V]."""
+    z = bf16_bits_to_f64(hidden_bits) @ bf16_bits_to_f64(w_bits).T
+    if bias is not None:
+        z = z + np.asarray(bias, np.float64)[None, :]
+    return np.ascontiguousarray(z)
+
+
+def lmhead_verify_tree(hidden_bits, w_bits, bias, tok, parent, theta, flags: int = 0,
+                       Dcap: int | None = None) -> dict:
+    """Output projection in fp64 followed by the tree rule taken in fp64."""
+    z = lmhead_logits(hidden_bits, w_bits, bias)
+    out = verify_tree(z, tok, parent, float(np.float32(theta)), flags, Dcap)
+    out["logits"] = z
+    return out
