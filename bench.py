@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the MARS verification hot path (libmars) on B200.
+
+One "step" is one full verification call over one batch: stream every logits row, top-2,
+margin rule, longest accepted path, emit.  The default workload is the serving-scale
+batched tree verification (256 sequences x 60-node depth-6 trees = 15 360 rows, |V| =
+151 936, bf16 logits, 4.67 GB per step), the configuration on which the HBM-roofline target
+is stated.  Prints ONE JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With N > 1 (torchrun) every rank verifies its own batch of the same shape (sequences are
+independent: no data-path collective); the time is the maximum over ranks.
+`--impl reference` times the CPU oracle on the host cores instead of the CUDA library.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_15498_b200 import synth  # noqa: E402
+
+METRIC = "verified_positions_per_sec"
+UNIT = "positions/s"
+L2_BYTES = 126 * 1024 * 1024
+HBM_NOMINAL_GBS = 8000.0
+HBM_FALLBACK_GBS = 6650.0
+
+WORKLOADS = {
+    "cfg3_bf16": lambda dev, seed: synth.cfg3(dev, seed=seed, dtype=torch.bfloat16),
+    "cfg3_fp32": lambda dev, seed: synth.cfg3(dev, seed=seed, dtype=torch.float32),
+    "cfg2": lambda dev, seed: synth.cfg2(dev, seed=seed),
+    "cfg1": lambda dev, seed: synth.cfg1(dev, seed=seed),
+    "cfg0": lambda dev, seed: synth.cfg0(dev, seed=seed),
+}
+BASE_SEED = {"cfg3_bf16": 3, "cfg3_fp32": 3, "cfg2": 2, "cfg1": 1, "cfg0": 0}
+
+
+# ------------------------------------------------------------------------------ helpers
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback (earlier pool measurement)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
+
+    BAD = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20}
+    NOTED = {"sw_power_cap": 0x4}
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.period = period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = int(vis.split(",")[device_index]) if vis and vis.split(",")[0].isdigit() else device_index
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+
+    def _poll(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for name, bit in {**self.BAD, **self.NOTED}.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self) -> dict:
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def reduce_max_time_sum_units(elapsed_ms: float, units: float, world: int):
+    """Whole-job figures from per-rank ones: slowest rank's time, all ranks' units."""
+    if world == 1:
+        return elapsed_ms, units
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------ arms
+
+def run_oracle_sample(w, host_logits, seqs: int):
+    from oracle import mars_oracle as orc
+    n = seqs * w.N
+    t0 = time.perf_counter()
+    orc.verify_tree(host_logits[:n], w.tok[:seqs], w.parent[:seqs], w.theta)
+    return time.perf_counter() - t0, n, orc.threads()
+
+
+def reference_arm(args, rank: int):
+    """The CPU oracle, as it stands, on the host cores; rank 0 only."""
+    if rank != 0:
+        return
+    seed = BASE_SEED[args.workload]
+    if args.workload in ("cfg0", "cfg1"):
+        w = WORKLOADS[args.workload]("cpu", seed)
+    else:   # bounded sample: 16 whole sequences of the same recipe per step
+        maker, kw = {"cfg3_bf16": (synth.cfg3, dict(dtype=torch.bfloat16)),
+                     "cfg3_fp32": (synth.cfg3, dict(dtype=torch.float32)),
+                     "cfg2": (synth.cfg2, {})}[args.workload]
+        w = maker("cpu", seed=seed, B=16, **kw)
+    seqs = w.B
+    host = synth.to_numpy_bits(w.logits)
+    for _ in range(args.warmup):
+        run_oracle_sample(w, host, seqs)
+    t = 0.0
+    cores = 1
+    for _ in range(args.steps):
+        dt, n, cores = run_oracle_sample(w, host, seqs)
+        t += dt
+    value = seqs * w.N * args.steps / t
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.logits.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "B": w.B, "N": w.N, "V": w.V, "theta": w.theta,
+                   "note": "CPU oracle; each step is a bounded sample of the workload"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{seqs} sequences x {w.N} rows per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        reference_arm(args, rank)
+        return
+
+    args.steps = 2000 if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else max(args.warmup, 3)
+
+    from paper_2601_15498_b200 import build, mars
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    barrier(world)
+    mars.lib()
+
+    # ---- inputs, resident in HBM; every rank gets its own batch of the same shape ----
+    w = WORKLOADS[args.workload](dev, BASE_SEED[args.workload] + 1000 * rank)
+    dt_code = mars.BF16 if w.logits.dtype == torch.bfloat16 else mars.FP32
+    copies = 1
+    if w.logits_bytes < 3 * L2_BYTES:   # small workloads: rotate over copies so that no step finds
+        copies = -(-3 * L2_BYTES // w.logits_bytes)   # its rows in L2
+    logits = [w.logits] + [w.logits.clone() for _ in range(copies - 1)]
+    tok = torch.as_tensor(w.tok, device=dev)
+    parent = torch.as_tensor(w.parent, device=dev)
+    draft = torch.as_tensor(w.draft, device=dev)
+    ws = torch.empty(mars.workspace_bytes(w.B, w.N, w.V, dt_code), dtype=torch.uint8, device=dev)
+    out = mars.alloc_outputs(w.B, w.N, w.N - 1, dev)
+
+    def step(i, lg=None):
+        lg = logits[i % copies] if lg is None else lg
+        if w.kind == "chain":
+            mars.verify_chain(lg, draft, w.theta, workspace=ws, out=out)
+        else:
+            mars.verify_tree(lg, tok, parent, w.theta, workspace=ws, out=out)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps between two events on the launching stream ----
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for i in range(args.steps):
+            step(i)
+        e1.record()
+        torch.cuda.synchronize()
+    barrier(world)
+    elapsed_ms = e0.elapsed_time(e1)
+    total_ms, total_units = reduce_max_time_sum_units(elapsed_ms, float(w.R * args.steps), world)
+    value = total_units / (total_ms * 1e-3)
+    ms_per_step = total_ms / args.steps
+
+    # ---- end to end: host buffers in, results out, copies inside the timed region ----
+    h_logits = torch.empty(w.logits.shape, dtype=w.logits.dtype, pin_memory=True)
+    h_logits.copy_(w.logits)
+    h_tok = torch.as_tensor(w.tok).pin_memory()
+    h_par = torch.as_tensor(w.parent).pin_memory()
+    h_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype, pin_memory=True)
+             for k in ("accept_len", "out_tokens", "out_len")}
+    d_logits = torch.empty_like(w.logits)
+
+    def e2e_step():
+        d_logits.copy_(h_logits, non_blocking=True)
+        tok.copy_(h_tok, non_blocking=True)
+        parent.copy_(h_par, non_blocking=True)
+        if w.kind == "chain":
+            draft.copy_(tok[:, 1:])
+        step(0, d_logits)
+        for k, h in h_out.items():
+            h.copy_(out[k], non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier(world)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    f1.record()
+    torch.cuda.synchronize()
+    e2e_ms, e2e_units = reduce_max_time_sum_units(f0.elapsed_time(f1), float(w.R * args.e2e_steps), world)
+    h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4
+    d2h = sum(h.numel() * h.element_size() for h in h_out.values())
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the one kernel on the path (algorithmic bytes: every logit once) ----
+    peak, peak_src = measured_hbm_peak()
+    achieved = w.logits_bytes / (elapsed_ms / args.steps * 1e-3) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get(args.workload)
+        except Exception:
+            traffic = None
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        host = synth.to_numpy_bits(h_logits)
+        seqs = min(w.B, max(1, 7680 // w.N))
+        run_oracle_sample(w, host, min(seqs, 2))
+        dt, n, cores = run_oracle_sample(w, host, seqs)
+        cpu = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"first {seqs} sequences ({n} rows) of the same workload, one pass, {dt:.2f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.logits.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "kind": w.kind, "B": w.B, "N": w.N, "V": w.V,
+                   "theta": w.theta, "rows_per_step": w.R, "logits_bytes_per_step": w.logits_bytes,
+                   "l2": ("inputs larger than L2" if copies == 1 else
+                          f"rotating over {copies} input copies, {copies * w.logits_bytes} B > L2"),
+                   "parallelism": f"dp{world} (independent sequences, no collective)"},
+        "us_per_step": 1e3 * ms_per_step,
+        "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "kernel": "mars::verify_kernel", "algorithmic_bytes_per_launch": w.logits_bytes},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

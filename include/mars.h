@@ -1,0 +1,140 @@
+/*
+ * mars.h -- C ABI of libmars: margin-aware speculative verification (MARS) on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * For every draft position of a batch of speculative-decoding chains or token trees
+ * the library streams the target model's logits row over the vocabulary, reduces it
+ * to its top-2 (z1, id1, z2, id2), applies the paper's three-way rule, resolves each
+ * sequence's longest accepted root-to-node path and emits the accepted length, the
+ * accepted tokens and the correction / bonus token.
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless a comment says
+ *     "host".  The library never allocates, frees or synchronises; it enqueues work on
+ *     `cuda_stream` (a cudaStream_t passed as void*, NULL = the default stream) and
+ *     returns.  Outputs are valid once the stream has passed that point.
+ *   - The return value reports host-detectable errors only; on error nothing is
+ *     launched and no output is touched.  Data-dependent problems are reported per
+ *     sequence in `seq_status`.
+ *   - Layout: B sequences, N rows ("nodes") per sequence, row r = b*N + node; the
+ *     logits matrix is [B*N, ld] with row stride `ld` >= V elements; only the first V
+ *     elements of a row are read.  Rows may start at any element-aligned address;
+ *     16-byte-aligned rows (ld*sizeof(elem) % 16 == 0 and an aligned base) take the
+ *     vector path end to end.
+ *   - Decisions are taken in fp32: bf16 logits widen exactly, the ratio is one IEEE
+ *     round-to-nearest fp32 division, the comparison with theta is strict.
+ *   - Total order on a row: larger value first, lower token id first among equal
+ *     values (-0 == +0); NaN counts as -inf.  Reported values have -0 replaced by +0.
+ */
+#ifndef MARS_H_
+#define MARS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MARS_OK = 0,
+    MARS_ERR_INVALID_ARG = 1, /* NULL required pointer, B<1, N<1, V<2, ld<V, NaN theta, ... */
+    MARS_ERR_WORKSPACE = 2,   /* workspace NULL, misaligned (256 B) or too small           */
+    MARS_ERR_UNSUPPORTED = 3, /* N or V above the supported caps, unknown dtype / flag      */
+    MARS_ERR_CUDA = 4         /* a CUDA runtime call (memset / launch) reported an error    */
+} mars_status_t;
+
+typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
+
+/* flags */
+#define MARS_SIGN_LITERAL 1u  /* drop the z1 > 0 guard: relax whenever z2/z1 > theta          */
+#define MARS_SHARED_PARENT 2u /* `parent` is one [N] array shared by all sequences            */
+
+#define MARS_MAX_NODES 1024   /* cap on N (rows per sequence)                                 */
+
+/* per-sequence status values written to seq_status */
+#define MARS_SEQ_OK 0
+#define MARS_SEQ_BAD_TREE 1   /* parent[0] != -1, or for i>0 parent[i] >= i or parent[i] < -1 */
+#define MARS_SEQ_DEPTH_CAP 2  /* the accepted path is deeper than Dcap                          */
+#define MARS_SEQ_TIMEOUT 3    /* a bounded device-side wait gave up (mars_lmhead_verify only)  */
+
+/* Optional extra outputs; the struct lives in HOST memory, its members are device
+ * pointers, any of which may be NULL. */
+typedef struct {
+    float *top2_val;     /* [B*N, 2]  z1, z2 of every row                                   */
+    int32_t *top2_id;    /* [B*N, 2]  id1, id2 of every row                                 */
+    uint8_t *node_flags; /* [B, N]    bit0 token == parent's top-1; bit1 token == parent's
+                                      top-2 and the parent row relaxes; bit2 accepted (every
+                                      ancestor accepted too); bit3 on the emitted path        */
+} mars_debug_out_t;
+
+/*
+ * Bytes of workspace (device memory, 256-byte aligned) that one call with these sizes
+ * needs.  Host function, no CUDA call.  Returns 0 for unsupported sizes.  The workspace
+ * holds per-slice top-2 records for rows that are split over several thread blocks and
+ * one arrival counter per sequence; its contents need not be initialised or preserved.
+ * Two calls that may overlap on the GPU need separate workspaces.
+ */
+size_t mars_workspace_bytes(int B, int N, int V, mars_dtype_t dt);
+
+/*
+ * Chain verification: Algorithm 1 of the paper ("Margin-Aware Speculative Verification
+ * Algorithm") with the three-way rule of Sec. 3.4 (exact match / adaptive relaxation
+ * r = z(2)/z(1) > theta, Eq. 4 / rejection and correction), plus the bonus token of the
+ * Table 1 caption when every draft is accepted.
+ *
+ *   logits     [B*K, ld] of `dt`; row b*K + i is the target's distribution that judges
+ *              draft[b, i]; row K-1 only supplies the bonus token.
+ *   draft      int32 [B, K-1]; a negative id or an id >= V never matches.
+ *   K          rows per sequence (K-1 drafts), 1 <= K <= MARS_MAX_NODES.
+ *   theta      threshold; any non-NaN float; theta >= 1 is strict greedy verification
+ *              (Sec. 2.3) unless MARS_SIGN_LITERAL is set.
+ *   accept_len int32 [B]    number of accepted drafts a, 0 <= a <= K-1.
+ *   out_tokens int32 [B, K] the a accepted drafts followed by the top-1 of row a
+ *              (correction if a < K-1, bonus if a == K-1); unused slots are -1.
+ *   out_len    int32 [B]    a + 1.
+ *   seq_status int32 [B] or NULL; always MARS_SEQ_OK for chains.
+ *   dbg        host pointer or NULL.
+ */
+mars_status_t mars_verify_chain(const void *logits, int64_t ld, mars_dtype_t dt,
+                                const int32_t *draft, int B, int K, int V, float theta,
+                                uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
+                                int32_t *out_len, int32_t *seq_status,
+                                const mars_debug_out_t *dbg, void *workspace,
+                                size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Tree verification: the same per-token rule (Sec. 3.4) on a token tree (Sec. 2.3,
+ * "tree-based methods ... verify many competing prefixes in a single forward pass").
+ * Node 0 is the root (the last committed token) and is always accepted.  Node i > 0 is
+ * accepted iff its parent is accepted and tok[i] passes the rule against the PARENT's
+ * row.  The result is the deepest accepted node, lowest node index among equally deep
+ * ones; the emitted next token is the top-1 of that node's row.
+ *
+ *   logits     [B*N, ld]; row b*N + i is the target's distribution after consuming the
+ *              path root -> node i.
+ *   tok        int32 [B, N]; tok[., 0] is ignored; negative = padding node.
+ *   parent     int32 [B, N] ([N] with MARS_SHARED_PARENT); parent[0] = -1,
+ *              parent[i] < i; parent[i] == -1 for i > 0 marks an absent node.
+ *   Dcap       capacity of the path outputs; must be >= 0.  If the accepted path is
+ *              deeper, the sequence gets MARS_SEQ_DEPTH_CAP and the safe output.
+ *   out_tokens int32 [B, Dcap+1]; path_nodes int32 [B, Dcap+1] or NULL (node ids of the
+ *              emitted path, root first); unused slots are -1.
+ *   seq_status int32 [B] or NULL.  A sequence whose status is not MARS_SEQ_OK gets the
+ *              safe output: accept_len 0, out_len 1, out_tokens[0] = top-1 of the root
+ *              row, path_nodes[0] = 0, node_flags = {root: accepted|on path, rest 0}.
+ */
+mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt,
+                               const int32_t *tok, const int32_t *parent, int B, int N, int V,
+                               float theta, uint32_t flags, int32_t *accept_len,
+                               int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
+                               int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Static, human-readable name of a status code (host memory, never NULL). */
+const char *mars_status_string(mars_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MARS_H_ */

@@ -1,0 +1,405 @@
+// libmars: streaming top-2 over logits rows fused with the MARS verification tail.
+//
+// One kernel per call.  A thread block owns one slice of one logits row (a whole row when
+// the batch has enough rows to fill the GPU, 1/S of a row otherwise) and streams it once
+// from HBM with 16-byte loads.  Each thread keeps an exact top-2 (values and token ids) in
+// registers, but touches it only for the few batches that can still change the answer:
+//
+//   - a batch of kU 16-byte vectors per thread is first reduced to its maximum with packed
+//     bf16x2 (or fp32) max instructions -- about one instruction per two bf16 elements;
+//   - the batch is skipped unless its maximum beats the thread's own runner-up AND is not
+//     below T2, a lower bound on the slice's runner-up value that the whole block shares
+//     through shared memory (order-preserving integer encoding, atomicMax);
+//   - the bound is bootstrapped from the first batch with a warp-level top-2 of the batch
+//     maxima, so that no thread pays the exact path for its first batch.
+//
+// Why skipping is exact: threads visit their elements in increasing token id, so an element
+// equal to the thread's runner-up loses the id tie-break; and an element below a value that
+// two other elements of the slice reach cannot be in the slice's top-2.
+//
+// Finished slices meet in global memory: the block writes its 16-byte record, bumps the
+// sequence's arrival counter, and the block that arrives last (nobody waits, nobody spins)
+// merges the records of the sequence and runs the verification tail of mars_common.cuh.
+#include "mars_common.cuh"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+
+#include "mars.h"
+
+namespace mars {
+
+constexpr int kThreads = 256;  // threads per block
+constexpr int kU = 4;          // 16-byte vectors per thread per batch (64 B in flight each)
+constexpr int kTargetBlocks = 148 * 8;     // split rows until the grid has about this many blocks
+constexpr int kMinSliceBytes = 8 * 1024;   // ... but never below this many bytes per slice
+
+struct Params {
+    const void *logits;
+    long long ld;
+    int V;
+    int N;
+    int S;   // slices per row
+    int L;   // elements per slice (multiple of 16)
+    Rec *partial;        // [R*S]
+    unsigned *counters;  // [B]
+    TailArgs tail;
+};
+
+// ---- order-preserving float <-> uint encoding for the shared bound ----------------------
+__device__ __forceinline__ unsigned enc(float x)
+{
+    unsigned b = __float_as_uint(x + 0.0f);
+    return b ^ ((unsigned)((int)b >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ float dec(unsigned e)
+{
+    return __uint_as_float(e ^ ((e & 0x80000000u) ? 0x80000000u : 0xffffffffu));
+}
+
+// Insert one element's value into the block-wide multiset top-2 {T1 >= T2}.  Every element
+// is published at most once, so T2 never exceeds the slice's true runner-up value.
+__device__ __forceinline__ void publish(unsigned *sT, float x)
+{
+    unsigned e = enc(x);
+    if (e > *(volatile unsigned *)&sT[1]) {
+        unsigned old = atomicMax(&sT[0], e);
+        unsigned y = min(old, e);
+        if (y > *(volatile unsigned *)&sT[1]) atomicMax(&sT[1], y);
+    }
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));  // NaN operand -> the other one
+    return d;
+}
+
+template <int DT> struct Elem;
+
+template <> struct Elem<MARS_BF16> {
+    static constexpr int kBytes = 2;
+    static constexpr int kVec = 8;
+    typedef uint32_t packed_t;  // two bf16 lanes
+    static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u); }
+    static __device__ __forceinline__ packed_t vred(const uint4 &v) { return bmax2(bmax2(v.x, v.y), bmax2(v.z, v.w)); }
+    static __device__ __forceinline__ packed_t pmax(packed_t a, packed_t b) { return bmax2(a, b); }
+    static __device__ __forceinline__ float to_float(packed_t m)
+    {
+        return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+    }
+    static __device__ __forceinline__ float elem(const uint4 &v, int k)
+    {
+        uint32_t w = (k >> 1) == 0 ? v.x : (k >> 1) == 1 ? v.y : (k >> 1) == 2 ? v.z : v.w;
+        return (k & 1) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16);
+    }
+    static __device__ __forceinline__ float scalar(const void *row, int j)
+    {
+        return __uint_as_float((uint32_t)((const unsigned short *)row)[j] << 16);
+    }
+};
+
+template <> struct Elem<MARS_FP32> {
+    static constexpr int kBytes = 4;
+    static constexpr int kVec = 4;
+    typedef float packed_t;
+    static __device__ __forceinline__ uint4 neg_inf() { return make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u); }
+    static __device__ __forceinline__ packed_t vred(const uint4 &v)
+    {
+        return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
+                     fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+    }
+    static __device__ __forceinline__ packed_t pmax(packed_t a, packed_t b) { return fmaxf(a, b); }
+    static __device__ __forceinline__ float to_float(packed_t m) { return m; }
+    static __device__ __forceinline__ float elem(const uint4 &v, int k)
+    {
+        return __uint_as_float(k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w);
+    }
+    static __device__ __forceinline__ float scalar(const void *row, int j) { return ((const float *)row)[j]; }
+};
+
+// Exact insert of one element into the thread's top-2.  Valid because a thread sees its
+// elements in increasing token id: equality never displaces.
+template <bool PUBLISH>
+__device__ __forceinline__ void insert(Rec &s, float x, int idx, unsigned *sT)
+{
+    if (x > s.z2) {
+        if (x > s.z1) { s.z2 = s.z1; s.id2 = s.id1; s.z1 = x; s.id1 = idx; }
+        else { s.z2 = x; s.id2 = idx; }
+        if (PUBLISH) publish(sT, x);
+    }
+}
+
+template <int DT, bool PUBLISH>
+__device__ __forceinline__ void process_batch(const uint4 (&v)[kU], const typename Elem<DT>::packed_t (&q)[kU],
+                                              float bm, float T2, int idx0, Rec &s, unsigned *sT)
+{
+    typedef Elem<DT> E;
+    if (bm > s.z2 && bm >= T2) {
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            float qf = E::to_float(q[u]);
+            if (qf > s.z2 && qf >= T2) {
+                int base = idx0 + u * kThreads * E::kVec;
+#pragma unroll
+                for (int k = 0; k < E::kVec; ++k) insert<PUBLISH>(s, E::elem(v[u], k), base + k, sT);
+            }
+        }
+    }
+}
+
+template <int DT, bool GUARD>
+__device__ __forceinline__ float load_batch(const uint4 *vbase, int v0, int nvec, uint4 (&v)[kU],
+                                            typename Elem<DT>::packed_t (&q)[kU])
+{
+    typedef Elem<DT> E;
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+        int vi = v0 + u * kThreads;
+        if (!GUARD || vi < nvec) v[u] = ld_stream(vbase + vi);
+        else v[u] = E::neg_inf();
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) q[u] = E::vred(v[u]);
+    return E::to_float(E::pmax(E::pmax(q[0], q[1]), E::pmax(q[2], q[3])));
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
+{
+    typedef Elem<DT> E;
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    __shared__ unsigned sT[2];
+    __shared__ Rec s_warp[kThreads / 32];
+    __shared__ int s_last;
+
+    const int tid = threadIdx.x;
+    const long long blk = blockIdx.x;
+    const long long row = blk / p.S;
+    const int slice = (int)(blk - row * p.S);
+    const int b = (int)(row / p.N);
+
+    const int lo = slice * p.L;
+    const int hi = min(p.V, lo + p.L);
+    const char *rowp = (const char *)p.logits + (size_t)row * (size_t)p.ld * E::kBytes;
+
+    // [lo, hi) = head scalars | 16-byte vectors | tail scalars
+    const uintptr_t a0 = (uintptr_t)(rowp + (size_t)lo * E::kBytes);
+    int nhead = (int)(((16 - (a0 & 15)) & 15) / E::kBytes);
+    nhead = min(nhead, max(hi - lo, 0));
+    const int vlo = lo + nhead;
+    const int nvec = max(hi - vlo, 0) / E::kVec;
+    const int tlo = vlo + nvec * E::kVec;
+    const int ntail = max(hi - tlo, 0);
+    const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
+
+    if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
+    __syncthreads();
+
+    Rec s = empty_rec();
+    if (tid < nhead) insert<false>(s, E::scalar(rowp, lo + tid), lo + tid, sT);
+
+    constexpr int kBatchVecs = kThreads * kU;
+    const int nfull = nvec / kBatchVecs;
+    uint4 v[kU];
+    typename E::packed_t q[kU];
+
+    // ---- batch 0: bootstrap the shared bound from the batch maxima, then process ----
+    float bm = (nfull > 0) ? load_batch<DT, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, true>(vbase, tid, nvec, v, q);
+    {
+        float a1 = (bm == bm) ? bm : -INFINITY, a2 = -INFINITY;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            float b1 = __shfl_xor_sync(0xffffffffu, a1, m), b2 = __shfl_xor_sync(0xffffffffu, a2, m);
+            a2 = fmaxf(fminf(a1, b1), fmaxf(a2, b2));
+            a1 = fmaxf(a1, b1);
+        }
+        if ((tid & 31) == 0) { publish(sT, a1); publish(sT, a2); }
+    }
+    __syncthreads();
+    float T2 = dec(*(volatile unsigned *)&sT[1]);
+    process_batch<DT, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
+
+    // ---- steady state ----
+    for (int bi = 1; bi < nfull; ++bi) {
+        bm = load_batch<DT, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
+        T2 = dec(*(volatile unsigned *)&sT[1]);
+        process_batch<DT, true>(v, q, bm, T2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
+    }
+    if (nfull > 0 && nfull * kBatchVecs < nvec) {
+        bm = load_batch<DT, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        T2 = dec(*(volatile unsigned *)&sT[1]);
+        process_batch<DT, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
+    }
+    if (tid < ntail) insert<false>(s, E::scalar(rowp, tlo + tid), tlo + tid, sT);
+
+    // ---- block merge under the full total order ----
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) s = merge(s, shfl_xor_rec(s, m));
+    if ((tid & 31) == 0) s_warp[tid >> 5] = s;
+    __syncthreads();
+    if (tid == 0) {
+        Rec r = s_warp[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) r = merge(r, s_warp[w]);
+        p.partial[blk] = r;
+        __threadfence();
+        unsigned ticket = atomicAdd(&p.counters[b], 1u);
+        s_last = (ticket == (unsigned)(p.N * p.S - 1)) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+
+    // ---- last block of the sequence: merge slices, verify, emit ----
+    __threadfence();
+    const int S = p.S;
+    const Rec *seq_partial = p.partial + (size_t)b * p.N * S;
+    verify_tail(p.tail, b, smem_dyn, [&](int i) {
+        Rec acc = empty_rec();
+        for (int k = 0; k < S; ++k) {
+            int4 w = __ldcg(reinterpret_cast<const int4 *>(seq_partial + (size_t)i * S + k));
+            Rec r;
+            r.z1 = __int_as_float(w.x); r.id1 = w.y; r.z2 = __int_as_float(w.z); r.id2 = w.w;
+            acc = merge(acc, r);
+        }
+        return finish_record(acc);
+    });
+    if (tid == 0) p.counters[b] = 0;
+}
+
+// ------------------------------------------------------------------------- host side
+
+struct Split { int S; int L; };
+
+static Split choose_split(long long R, int V, int dt)
+{
+    const int es = dt == MARS_BF16 ? 2 : 4;
+    long long S = 1;
+    const char *force = getenv("MARS_FORCE_SPLIT");  // test hook: force slices per row
+    int min_elems = kMinSliceBytes / es;
+    if (force && atoi(force) >= 1) { S = atoi(force); min_elems = 64; }
+    else if (R < kTargetBlocks) S = (kTargetBlocks + R - 1) / R;
+    long long smax = V / min_elems;
+    if (smax < 1) smax = 1;
+    if (S > smax) S = smax;
+    long long L = (V + S - 1) / S;
+    L = (L + 15) / 16 * 16;
+    Split sp;
+    sp.L = (int)L;
+    sp.S = (int)((V + L - 1) / L);
+    return sp;
+}
+
+static size_t counters_bytes(int B) { return ((size_t)B * sizeof(unsigned) + 255) / 256 * 256; }
+
+static bool sizes_supported(int B, int N, int V, int dt)
+{
+    if (B < 1 || N < 1 || V < 2) return false;
+    if (dt != MARS_BF16 && dt != MARS_FP32) return false;
+    if (N > MARS_MAX_NODES) return false;
+    if (V > (1 << 30)) return false;
+    if ((long long)B * N > (1ll << 40)) return false;
+    return true;
+}
+
+static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
+                         const int32_t *parent, int chain, int B, int N, int V, float theta,
+                         uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
+                         int32_t *path_nodes, int32_t *out_len, int Dcap, int32_t *seq_status,
+                         const mars_debug_out_t *dbg, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream)
+{
+    if (B < 1 || N < 1 || V < 2 || !logits || !accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
+    if (ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
+    if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
+    if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT)) return MARS_ERR_UNSUPPORTED;
+    if (!sizes_supported(B, N, V, (int)dt)) return MARS_ERR_UNSUPPORTED;
+    const int es = dt == MARS_BF16 ? 2 : 4;
+    if ((uintptr_t)logits % es) return MARS_ERR_INVALID_ARG;
+    const long long R = (long long)B * N;
+    const Split sp = choose_split(R, V, (int)dt);
+    if (R * sp.S > 0x7fffffffll) return MARS_ERR_UNSUPPORTED;
+    const size_t need = counters_bytes(B) + (size_t)R * sp.S * sizeof(Rec);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;
+
+    Params p;
+    p.logits = logits; p.ld = ld; p.V = V; p.N = N; p.S = sp.S; p.L = sp.L;
+    p.counters = (unsigned *)workspace;
+    p.partial = (Rec *)((char *)workspace + counters_bytes(B));
+    p.tail.tok = tok; p.tail.parent = parent;
+    p.tail.accept_len = accept_len; p.tail.out_tokens = out_tokens; p.tail.path_nodes = path_nodes;
+    p.tail.out_len = out_len; p.tail.seq_status = seq_status;
+    p.tail.dbg_val = dbg ? dbg->top2_val : nullptr;
+    p.tail.dbg_id = dbg ? dbg->top2_id : nullptr;
+    p.tail.dbg_flags = dbg ? dbg->node_flags : nullptr;
+    p.tail.N = N; p.tail.Dcap = Dcap; p.tail.theta = theta; p.tail.flags = flags; p.tail.chain = chain;
+
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(p.counters, 0, (size_t)B * sizeof(unsigned), st) != cudaSuccess) return MARS_ERR_CUDA;
+    const unsigned grid = (unsigned)(R * sp.S);
+    const size_t smem = tail_smem_bytes(N);
+    if (dt == MARS_BF16) verify_kernel<MARS_BF16><<<grid, kThreads, smem, st>>>(p);
+    else verify_kernel<MARS_FP32><<<grid, kThreads, smem, st>>>(p);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+}
+
+}  // namespace mars
+
+extern "C" {
+
+size_t mars_workspace_bytes(int B, int N, int V, mars_dtype_t dt)
+{
+    if (!mars::sizes_supported(B, N, V, (int)dt)) return 0;
+    const long long R = (long long)B * N;
+    const mars::Split sp = mars::choose_split(R, V, (int)dt);
+    return mars::counters_bytes(B) + (size_t)R * sp.S * sizeof(mars::Rec);
+}
+
+mars_status_t mars_verify_chain(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *draft,
+                                int B, int K, int V, float theta, uint32_t flags, int32_t *accept_len,
+                                int32_t *out_tokens, int32_t *out_len, int32_t *seq_status,
+                                const mars_debug_out_t *dbg, void *workspace, size_t workspace_bytes,
+                                void *cuda_stream)
+{
+    if (flags & MARS_SHARED_PARENT) return MARS_ERR_INVALID_ARG;
+    return mars::run(logits, ld, dt, draft, nullptr, 1, B, K, V, theta, flags, accept_len, out_tokens,
+                     nullptr, out_len, K - 1, seq_status, dbg, workspace, workspace_bytes, cuda_stream);
+}
+
+mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
+                               const int32_t *parent, int B, int N, int V, float theta, uint32_t flags,
+                               int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
+                               int32_t *out_len, int Dcap, int32_t *seq_status,
+                               const mars_debug_out_t *dbg, void *workspace, size_t workspace_bytes,
+                               void *cuda_stream)
+{
+    return mars::run(logits, ld, dt, tok, parent, 0, B, N, V, theta, flags, accept_len, out_tokens,
+                     path_nodes, out_len, Dcap, seq_status, dbg, workspace, workspace_bytes, cuda_stream);
+}
+
+const char *mars_status_string(mars_status_t s)
+{
+    switch (s) {
+    case MARS_OK: return "ok";
+    case MARS_ERR_INVALID_ARG: return "invalid argument";
+    case MARS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MARS_ERR_UNSUPPORTED: return "unsupported size, dtype or flag";
+    case MARS_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,186 @@
+"""ctypes binding of libmars (argument marshalling only).
+
+Every step of verification runs inside the CUDA library; this module turns torch CUDA
+tensors into device pointers, provides the workspace and the current stream, and checks
+the returned status.  There is no CPU path: a missing library or a failed call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+import torch
+
+from . import build as _build
+
+BF16, FP32 = 0, 1
+SIGN_LITERAL, SHARED_PARENT = 1, 2
+MAX_NODES = 1024
+
+_lock = threading.Lock()
+_lib = None
+
+
+class MarsError(RuntimeError):
+    pass
+
+
+class _DebugOut(ctypes.Structure):
+    _fields_ = [("top2_val", ctypes.c_void_p), ("top2_id", ctypes.c_void_p),
+                ("node_flags", ctypes.c_void_p)]
+
+
+def lib() -> ctypes.CDLL:
+    """Open libmars.so (built in-tree by ``build.build()``); raises if it is missing."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            path = _build.LIB
+            if not os.path.exists(path):
+                raise MarsError(f"{path} not found: run paper_2601_15498_b200.build.build() "
+                                "(nvcc, sm_100a); there is no fallback path")
+            L = ctypes.CDLL(path)
+            vp, i32, i64, u32, f32, sz = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
+                                          ctypes.c_uint32, ctypes.c_float, ctypes.c_size_t)
+            L.mars_workspace_bytes.argtypes = [i32, i32, i32, i32]
+            L.mars_workspace_bytes.restype = sz
+            L.mars_verify_chain.argtypes = [vp, i64, i32, vp, i32, i32, i32, f32, u32, vp, vp, vp,
+                                            vp, ctypes.POINTER(_DebugOut), vp, sz, vp]
+            L.mars_verify_chain.restype = i32
+            L.mars_verify_tree.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, u32, vp, vp,
+                                           vp, vp, i32, vp, ctypes.POINTER(_DebugOut), vp, sz, vp]
+            L.mars_verify_tree.restype = i32
+            L.mars_status_string.argtypes = [i32]
+            L.mars_status_string.restype = ctypes.c_char_p
+            _lib = L
+    return _lib
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise MarsError(f"{what}: {lib().mars_status_string(code).decode()} (status {code})")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return FP32
+    raise MarsError(f"logits must be bfloat16 or float32, got {t.dtype}")
+
+
+def _dev_i32(x, device) -> torch.Tensor:
+    t = torch.as_tensor(x)
+    if t.dtype != torch.int32 or t.device != device or not t.is_contiguous():
+        t = t.to(device=device, dtype=torch.int32).contiguous()
+    return t
+
+
+def workspace_bytes(B: int, N: int, V: int, dtype_code: int) -> int:
+    return int(lib().mars_workspace_bytes(B, N, V, dtype_code))
+
+
+def _workspace(B, N, V, dt, device, workspace):
+    need = workspace_bytes(B, N, V, dt)
+    if need == 0:
+        raise MarsError("unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, workspace.numel() * workspace.element_size()
+
+
+def _logits_args(logits: torch.Tensor, rows: int, V):
+    if not logits.is_cuda:
+        raise MarsError("logits must live in device memory")
+    if logits.dim() != 2 or logits.stride(1) != 1 or logits.shape[0] != rows:
+        raise MarsError("logits must be [rows, >=V] with unit inner stride")
+    V = logits.shape[1] if V is None else int(V)
+    return _dtype_code(logits), int(logits.stride(0)), V
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def verify_tree(logits: torch.Tensor, tok, parent, theta: float, flags: int = 0,
+                Dcap: int | None = None, V: int | None = None, debug: bool = False,
+                workspace: torch.Tensor | None = None, out: dict | None = None) -> dict:
+    """mars_verify_tree on the current stream.  Returns device tensors; asynchronous."""
+    dev = logits.device
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    dt, ld, V = _logits_args(logits, B * N, V)
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    workspace, wbytes = _workspace(B, N, V, dt, dev, workspace)
+    if out is None:
+        out = alloc_outputs(B, N, Dcap, dev, debug)
+    dbg = None
+    if "top2_val" in out:
+        dbg = _DebugOut(out["top2_val"].data_ptr(), out["top2_id"].data_ptr(),
+                        out["node_flags"].data_ptr())
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_tree(
+            logits.data_ptr(), ld, dt, tok.data_ptr(), parent.data_ptr(), B, N, V, float(theta),
+            flags, out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(),
+            out["path_nodes"].data_ptr(), out["out_len"].data_ptr(), Dcap,
+            out["seq_status"].data_ptr(), ctypes.byref(dbg) if dbg is not None else None,
+            workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_verify_tree")
+    out["_keepalive"] = (tok, parent, workspace)
+    return out
+
+
+def verify_chain(logits: torch.Tensor, draft, theta: float, flags: int = 0, V: int | None = None,
+                 debug: bool = False, workspace: torch.Tensor | None = None,
+                 out: dict | None = None) -> dict:
+    """mars_verify_chain on the current stream: K rows and K-1 drafts per sequence."""
+    dev = logits.device
+    draft = _dev_i32(draft, dev)
+    B, Km1 = draft.shape
+    K = Km1 + 1
+    dt, ld, V = _logits_args(logits, B * K, V)
+    workspace, wbytes = _workspace(B, K, V, dt, dev, workspace)
+    if out is None:
+        out = alloc_outputs(B, K, K - 1, dev, debug)
+    dbg = None
+    if "top2_val" in out:
+        dbg = _DebugOut(out["top2_val"].data_ptr(), out["top2_id"].data_ptr(),
+                        out["node_flags"].data_ptr())
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_chain(
+            logits.data_ptr(), ld, dt, draft.data_ptr() if Km1 > 0 else None, B, K, V,
+            float(theta), flags, out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(),
+            out["out_len"].data_ptr(), out["seq_status"].data_ptr(),
+            ctypes.byref(dbg) if dbg is not None else None, workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_verify_chain")
+    out["_keepalive"] = (draft, workspace)
+    return out
+
+
+def alloc_outputs(B: int, N: int, Dcap: int, device, debug: bool = False) -> dict:
+    """Output buffers in device memory (filled with a poison value so that unwritten
+    slots are noticed)."""
+    def full(shape, dtype, v):
+        return torch.full(shape, v, dtype=dtype, device=device)
+    out = {
+        "accept_len": full((B,), torch.int32, -777),
+        "out_tokens": full((B, Dcap + 1), torch.int32, -777),
+        "path_nodes": full((B, Dcap + 1), torch.int32, -777),
+        "out_len": full((B,), torch.int32, -777),
+        "seq_status": full((B,), torch.int32, -777),
+    }
+    if debug:
+        out["top2_val"] = full((B * N, 2), torch.float32, float("nan"))
+        out["top2_id"] = full((B * N, 2), torch.int32, -777)
+        out["node_flags"] = full((B, N), torch.uint8, 255)
+    return out
+
+
+def to_host(out: dict) -> dict:
+    """Synchronise and copy every output tensor to numpy."""
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy() for k, v in out.items() if isinstance(v, torch.Tensor)}

@@ -1,0 +1,97 @@
+"""The C-ABI library builds for sm_100a, loads, and exports every symbol that include/*.h
+declares.  Only host-side calls are made here (size queries, status strings, argument checks
+that return before any CUDA call)."""
+import ctypes
+import glob
+import os
+import re
+
+import pytest
+
+from paper_2601_15498_b200 import build, mars
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    names = []
+    for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        src = open(h).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names += re.findall(r"\b(mars_[a-z0-9_]+)\s*\(", src)
+    return sorted(set(names))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return mars.lib()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_functions()
+    assert {"mars_verify_chain", "mars_verify_tree", "mars_workspace_bytes",
+            "mars_status_string"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+        getattr(lib, n)
+
+
+def test_status_strings(lib):
+    seen = {lib.mars_status_string(c) for c in range(5)}
+    assert len(seen) == 5 and all(s for s in seen)
+    assert lib.mars_status_string(99) == b"unknown status"
+
+
+def test_workspace_bytes_host_only(lib, monkeypatch):
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    wb = lib.mars_workspace_bytes
+    assert wb(0, 1, 100, 0) == 0 and wb(1, 0, 100, 0) == 0 and wb(1, 1, 1, 0) == 0
+    assert wb(1, 1025, 100, 0) == 0 and wb(1, 1, 100, 7) == 0
+    # whole rows per block once the batch fills the GPU: one 16-byte record per row + counters
+    assert wb(256, 60, 151936, 0) == 1024 + 256 * 60 * 16
+    # few rows: rows are split, the workspace grows with the number of slices
+    small = wb(1, 6, 32000, 1)
+    assert small % 16 == 0 and 256 + 6 * 16 < small <= 256 + 6 * 16 * 64
+    assert wb(1, 60, 151936, 0) > 256 + 60 * 16
+    monkeypatch.setenv("MARS_FORCE_SPLIT", "3")
+    assert wb(2, 5, 4000, 1) == 256 + 10 * 3 * 16
+
+
+def test_argument_checks_return_before_any_cuda_call(lib):
+    """NULL pointers and bad sizes are rejected on the host (no GPU is needed to see that)."""
+    n = None
+    dummy = ctypes.c_void_p(256)
+    assert lib.mars_verify_tree(n, 10, 0, n, n, 1, 1, 10, 0.9, 0, n, n, n, n, 0, n, None, n, 0, n) == 1
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 0, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 dummy, 1 << 20, n) == 1
+    # ld < V
+    assert lib.mars_verify_chain(dummy, 5, 0, dummy, 1, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 dummy, 1 << 20, n) == 1
+    # NaN theta
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, float("nan"), 0, dummy, dummy, dummy,
+                                 n, None, dummy, 1 << 20, n) == 1
+    # unknown flag / too many nodes / unknown dtype
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 128, dummy, dummy, dummy, n, None,
+                                 dummy, 1 << 20, n) == 3
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2000, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 dummy, 1 << 20, n) == 3
+    assert lib.mars_verify_chain(dummy, 10, 5, dummy, 1, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 dummy, 1 << 20, n) == 3
+    # workspace: missing, too small, misaligned
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 n, 0, n) == 2
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 dummy, 16, n) == 2
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 0, dummy, dummy, dummy, n, None,
+                                 ctypes.c_void_p(260), 1 << 20, n) == 2
+    # misaligned logits pointer for the element size
+    assert lib.mars_verify_chain(ctypes.c_void_p(257), 10, 1, dummy, 1, 2, 10, 0.9, 0, dummy, dummy,
+                                 dummy, n, None, dummy, 1 << 20, n) == 1
+
+
+def test_missing_library_is_an_error(monkeypatch, tmp_path):
+    monkeypatch.setattr(mars, "_lib", None)
+    monkeypatch.setattr(build, "LIB", str(tmp_path / "nope.so"))
+    with pytest.raises(mars.MarsError, match="no fallback"):
+        mars.lib()

@@ -1,0 +1,289 @@
+"""Parity of the CUDA library with the CPU oracle, element by element, through the C ABI.
+
+Bar: bit-exact for token ids, lengths, paths, flags and statuses; the fp32 top-2 values are
+compared as bit patterns too (both sides take every decision in fp32).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mars_oracle as orc
+from paper_2601_15498_b200 import mars, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+KEYS_TREE = ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "top2_id",
+             "node_flags")
+
+
+def assert_same(got: dict, want: dict, keys, what=""):
+    for k in keys:
+        g, w = got[k], want[k]
+        assert g.shape == w.shape, (what, k, g.shape, w.shape)
+        if not np.array_equal(g, w):
+            bad = np.argwhere(g != w)[:5]
+            raise AssertionError(f"{what}: {k} differs at {bad.tolist()}: got {g[tuple(bad[0])]}, "
+                                 f"want {w[tuple(bad[0])]}")
+    g, w = got["top2_val"], want["top2_val"]
+    assert np.array_equal(g.view(np.uint32), w.view(np.uint32)), (what, "top2_val")
+
+
+def run_tree(logits, tok, parent, theta, flags=0, Dcap=None, V=None):
+    out = mars.to_host(mars.verify_tree(logits, tok, parent, theta, flags, Dcap, V, debug=True))
+    ref = orc.verify_tree(synth.to_numpy_bits(logits), tok, parent, theta, flags, Dcap, V)
+    return out, ref
+
+
+def run_chain(logits, draft, theta, flags=0, V=None):
+    out = mars.to_host(mars.verify_chain(logits, draft, theta, flags, V, debug=True))
+    ref = orc.verify_chain(synth.to_numpy_bits(logits), draft, theta, flags, V)
+    return out, ref
+
+
+@pytest.fixture(autouse=True)
+def _no_forced_split(monkeypatch):
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+
+
+# ------------------------------------------------------------------ the named workloads
+
+def test_cfg0_chain_b1_fp32():
+    w = synth.cfg0(DEV)
+    out, ref = run_chain(w.logits, w.draft, w.theta)
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), w.name)
+    assert (out["seq_status"] == 0).all()
+
+
+def test_cfg0_many_seeds_statistics():
+    """Same recipe, 512 sequences: parity, and the mean accepted length near its closed form."""
+    w = synth.cfg0(DEV, seed=100, B=512)
+    out, ref = run_chain(w.logits, w.draft, w.theta)
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), w.name)
+    p = 0.6 + 0.25 * 0.4 * (0.1 / 0.15)
+    mean = sum(p ** k for k in range(1, 6))
+    assert abs(out["accept_len"].mean() - mean) < 0.25
+
+
+def test_cfg1_tree_b1_bf16():
+    w = synth.cfg1(DEV)
+    out, ref = run_tree(w.logits, w.tok, w.parent, w.theta)
+    assert_same(out, ref, KEYS_TREE, w.name)
+
+
+@pytest.mark.parametrize("theta", [0.8, 0.9, 0.95, 1.5])
+def test_cfg2_batched_chain_theta_sweep(theta):
+    w = synth.cfg2(DEV, theta=theta)
+    out, ref = run_chain(w.logits, w.draft, theta)
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), f"{w.name} theta={theta}")
+    if theta > 1:   # strict greedy: accepted drafts equal the argmax of their rows
+        top1 = ref["top2_id"][:, 0].reshape(w.B, w.N)
+        for b in range(w.B):
+            a = out["accept_len"][b]
+            assert (w.draft[b, :a] == top1[b, :a]).all()
+            assert a == w.N - 1 or w.draft[b, a] != top1[b, a]
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_cfg3_reduced_batch_full_parity(dtype):
+    w = synth.cfg3(DEV, B=24, dtype=dtype)      # 1440 rows: whole rows per block (no split)
+    out, ref = run_tree(w.logits, w.tok, w.parent, w.theta)
+    assert_same(out, ref, KEYS_TREE, w.name)
+    assert out["accept_len"].max() >= 3
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_cfg3_full_size_sampled(dtype):
+    """The serving-scale workload in the launch configuration the benchmark times; the oracle
+    checks a sample of whole sequences, every sequence is checked for validity."""
+    w = synth.cfg3(DEV, dtype=dtype)
+    assert w.R == 15360
+    out = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, debug=True))
+    rng = np.random.default_rng(0)
+    sample = sorted(set(rng.choice(w.B, 10, replace=False).tolist()) | {0, w.B - 1})
+    rows = np.concatenate([np.arange(b * w.N, (b + 1) * w.N) for b in sample])
+    sub = w.logits[torch.as_tensor(rows, device=DEV)]
+    ref = orc.verify_tree(synth.to_numpy_bits(sub), w.tok[sample], w.parent[sample], w.theta)
+    got = {k: (v[rows] if k in ("top2_val", "top2_id") else v[sample]) for k, v in out.items()}
+    assert_same(got, ref, KEYS_TREE, w.name)
+    # properties that hold for every sequence
+    assert (out["seq_status"] == 0).all()
+    assert ((out["accept_len"] >= 0) & (out["accept_len"] <= w.max_depth)).all()
+    assert (out["out_len"] == out["accept_len"] + 1).all()
+    ids = out["top2_id"].reshape(w.B, w.N, 2)
+    for b in range(w.B):
+        a = out["accept_len"][b]
+        path = out["path_nodes"][b, :a + 1]
+        assert path[0] == 0
+        for k in range(1, a + 1):
+            n, p = path[k], path[k - 1]
+            assert w.parent[b, n] == p and w.tok[b, n] in ids[b, p]
+            assert out["out_tokens"][b, k - 1] == w.tok[b, n]
+        assert out["out_tokens"][b, a] == ids[b, path[a], 0]
+    # top-2 values of every row against torch's own top-k on the device (values only)
+    for r0 in range(0, w.R, 1024):
+        tv = torch.topk(w.logits[r0:r0 + 1024].float(), 2, dim=1).values.cpu().numpy()
+        assert np.array_equal(tv, out["top2_val"][r0:r0 + 1024])
+
+
+# ------------------------------------------------------------------ shapes and layouts
+
+@pytest.mark.parametrize("V", [2, 3, 7, 8, 9, 257, 4099, 32000, 151936])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_odd_vocab_sizes(V, dtype):
+    w = synth.tree_workload("odd", 3, 9, 3, 3, V, dtype, DEV, 40 + V % 13, 0.9, 3.0, 15.0, 30.0, 0.5)
+    out, ref = run_tree(w.logits, w.tok, w.parent, 0.9)
+    assert_same(out, ref, KEYS_TREE, f"V={V} {dtype}")
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("ld_extra,offset", [(1, 0), (3, 1), (5, 3), (8, 0), (13, 7)])
+def test_unaligned_rows_with_canaries(dtype, ld_extra, offset):
+    """Rows that start off a 16-byte boundary, ld > V, and a huge value in every element the
+    library must not read: padding columns and guard rows before and after."""
+    B, N, V = 4, 7, 5003
+    ld = V + ld_extra
+    w = synth.tree_workload("canary", B, N, 3, 3, V, dtype, DEV, 77, 0.9, 3.0, 15.0, 30.0, 0.5)
+    big = torch.full((B * N + 2, ld + offset), 3.0e38, dtype=dtype, device=DEV)
+    view = big[1:-1, offset:offset + ld]
+    view[:, :V] = w.logits
+    assert view.stride(0) == ld + offset
+    out = mars.to_host(mars.verify_tree(view, w.tok, w.parent, 0.9, V=V, debug=True))
+    ref = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, 0.9)
+    assert_same(out, ref, KEYS_TREE, f"ld+{ld_extra} off {offset}")
+
+
+@pytest.mark.parametrize("S", [1, 2, 3, 7, 16, 61])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_forced_row_split(monkeypatch, S, dtype):
+    """The merge is associative and commutative: any number of slices gives the same bits."""
+    monkeypatch.setenv("MARS_FORCE_SPLIT", str(S))
+    w = synth.tree_workload("split", 5, 12, 4, 3, 40000 + 7, dtype, DEV, 5, 0.9, 3.0, 15.0, 30.0, 0.5)
+    out, ref = run_tree(w.logits, w.tok, w.parent, 0.9)
+    assert_same(out, ref, KEYS_TREE, f"S={S}")
+
+
+def test_large_tree_more_than_64_nodes():
+    for N, depth in ((65, 10), (200, 12), (1024, 40)):
+        w = synth.tree_workload("big", 3, N, depth, 4, 3000, torch.bfloat16, DEV, N, 0.9, 3.0, 15.0,
+                                30.0, 0.5)
+        # aim most tokens at the leading ids so that deep paths are accepted
+        out, ref = run_tree(w.logits, w.tok, w.parent, 0.85)
+        assert_same(out, ref, KEYS_TREE, f"N={N}")
+    # a long chain through the tree path (N > 64) and through the chain entry point
+    w = synth.chain_workload("long", 2, 100, 2000, torch.float32, DEV, 3, 0.9, 2.0, 20.0, 20.0, 0.4)
+    lead = torch.topk(w.logits, 2, dim=1).indices.cpu().numpy().reshape(2, 100, 2)
+    draft = lead[:, :-1, 0].astype(np.int32).copy()
+    draft[1, 70] = 5                                # sequence 1 stops at depth 70
+    out, ref = run_chain(w.logits, draft, 0.9)
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "long chain")
+    assert out["accept_len"].tolist() == [99, 70]
+
+
+# ------------------------------------------------------------------ degenerate rows
+
+def special_rows(V, dtype):
+    z = torch.randn((12, V), dtype=torch.float32) * 3
+    z[0] = 1.5                                   # constant row
+    z[1] = torch.round(z[1])                     # heavy ties
+    z[2] = float("-inf")                         # all -inf
+    z[3] = float("nan")                          # all NaN
+    z[4] = float("-inf"); z[4, V - 1] = 0.5      # one finite entry, last position
+    z[5] = float("-inf"); z[5, 0] = -2.0
+    z[6, 5] = float("inf"); z[6, V // 2] = float("inf")
+    z[7] = -torch.abs(z[7]) - 1                  # all negative: z1 < 0
+    z[8] = 0.0; z[8, 3] = -0.0                   # zeros of both signs
+    z[9, 1::2] = float("nan")
+    z[10, :] = -5.0; z[10, V - 2] = 4.0; z[10, V - 1] = 4.0    # tie at the very end
+    z[11, :] = 7.0; z[11, 0] = float("nan")
+    return z.to(dtype).to(DEV)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("V", [9, 2048, 2048 * 9 + 5])
+@pytest.mark.parametrize("flags", [0, mars.SIGN_LITERAL])
+def test_degenerate_rows(dtype, V, flags):
+    z = special_rows(V, dtype)
+    N = z.shape[0]
+    parent = np.arange(-1, N - 1, dtype=np.int32)[None, :]
+    ids = orc.top2(synth.to_numpy_bits(z))[1]
+    for which in (0, 1):                          # drafts = top-1 of every row, then top-2
+        tok = np.full((1, N), -1, np.int32)
+        tok[0, 1:] = ids[:-1, which]
+        for theta in (0.9, 0.0, -1.0):
+            out, ref = run_tree(z, tok, parent, theta, flags)
+            assert_same(out, ref, KEYS_TREE, f"V={V} which={which} theta={theta} flags={flags}")
+
+
+def test_one_ulp_around_theta_on_device():
+    th = np.float32(0.9)
+    rows = []
+    for k in (-3, 0, 4):
+        z1 = np.float32(2.0 ** k)
+        on = np.float32(th * z1)
+        for z2 in (np.nextafter(on, np.float32(np.inf), dtype=np.float32), on,
+                   np.nextafter(on, np.float32(-np.inf), dtype=np.float32)):
+            r = np.full(64, -1.0, np.float32)
+            r[10], r[20] = z1, z2
+            rows.append(r)
+            rows.append(r)                       # second row of the 2-row chain (bonus)
+    z = torch.from_numpy(np.stack(rows)).to(DEV)
+    draft = np.full((len(rows) // 2, 1), 20, np.int32)
+    out, ref = run_chain(z, draft, float(th))
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "ulp")
+    assert out["accept_len"].tolist() == [1, 0, 0] * 3
+
+
+# ------------------------------------------------------------------ trees: flags and statuses
+
+def test_shared_parent_padding_malformed_and_depth_cap():
+    w = synth.tree_workload("t", 6, 20, 5, 3, 1000, torch.bfloat16, DEV, 9, 0.9, 3.0, 15.0, 30.0, 0.5)
+    par = w.parent.copy()
+    tok = w.tok.copy()
+    par[1, 7] = -1                     # absent node
+    tok[2, 3] = -4                     # padding token
+    par[3, 0] = 0                      # malformed: root has a parent
+    par[4, 5] = 5                      # malformed: parent[i] >= i
+    par[5, 9] = -2                     # malformed: below -1
+    tok[0, 4] = 5000                   # id beyond the vocabulary
+    out, ref = run_tree(w.logits, tok, par, 0.9)
+    assert_same(out, ref, KEYS_TREE, "statuses")
+    assert out["seq_status"].tolist() == [0, 0, 0, 1, 1, 1]
+    out, ref = run_tree(w.logits, tok, par, 0.9, Dcap=1)
+    assert_same(out, ref, KEYS_TREE, "depth cap")
+    assert 2 in out["seq_status"]
+    # one parent array shared by all sequences
+    out, ref = run_tree(w.logits, w.tok, w.parent[0], 0.9)
+    assert_same(out, ref, KEYS_TREE, "shared parent")
+
+
+def test_host_errors_launch_nothing():
+    w = synth.tree_workload("t", 2, 5, 3, 3, 100, torch.float32, DEV, 1, 0.9, 3.0, 15.0, 30.0, 0.5)
+    out = mars.alloc_outputs(2, 5, 4, DEV)
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.verify_tree(w.logits, w.tok, w.parent, float("nan"), out=out)
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.verify_tree(w.logits, w.tok, w.parent, 0.9, V=1, out=out)
+    with pytest.raises(mars.MarsError, match="workspace"):
+        mars.verify_tree(w.logits, w.tok, w.parent, 0.9, out=out,
+                         workspace=torch.empty(256, dtype=torch.uint8, device=DEV))
+    with pytest.raises(mars.MarsError, match="unsupported"):
+        mars.verify_tree(w.logits, w.tok, w.parent, 0.9, flags=64, out=out)
+    torch.cuda.synchronize()
+    assert (out["accept_len"].cpu().numpy() == -777).all()      # nothing was written
+
+
+def test_workspace_reuse_and_non_default_stream():
+    """Back-to-back calls on one workspace (stale contents) and on a side stream."""
+    w = synth.cfg2(DEV, seed=12, B=8)
+    need = mars.workspace_bytes(w.B, w.N, w.V, mars.BF16)
+    ws = torch.randint(0, 255, (need,), dtype=torch.uint8, device=DEV)      # garbage
+    ref = orc.verify_chain(synth.to_numpy_bits(w.logits), w.draft, 0.9)
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        outs = [mars.verify_chain(w.logits, w.draft, 0.9, debug=True, workspace=ws) for _ in range(3)]
+    st.synchronize()
+    for o in outs:
+        assert_same(mars.to_host(o), ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "reuse")
