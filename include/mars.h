@@ -131,6 +131,39 @@ mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt,
                                int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * Bytes of workspace (device memory, 256-byte aligned) for mars_lmhead_verify with these
+ * sizes.  Host function, no CUDA call.  Returns 0 for unsupported sizes (d must be a
+ * multiple of 64).  Contents need not be initialised or preserved.
+ */
+size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d);
+
+/*
+ * Output projection fused with tree verification: the logits z = W_o h + b_o (Eq. 2 of the
+ * paper) are accumulated in fp32 from bf16 operands on the tensor cores and reduced to each
+ * row's top-2 inside the GEMM epilogue, so they never reach HBM; the rows' records then go
+ * through the same rule and tree resolution as mars_verify_tree.
+ *
+ *   hidden   bf16 [B*N, d], row-major, 16-byte aligned; row b*N + i is the hidden state
+ *            after consuming the path root -> node i.
+ *   w_vocab  bf16 [V, d], row-major, 16-byte aligned (W_o).
+ *   bias     fp32 [V] or NULL (b_o).
+ *   d        hidden size, a multiple of 64.
+ *   dbg->top2_val receives the fp32-accumulated logits z1, z2 of every row.
+ *   Remaining arguments, outputs and per-sequence statuses are those of mars_verify_tree.
+ *   Accumulation order differs from a sequential sum, so near-ties may resolve differently
+ *   from an fp64 evaluation; decisions are still taken in fp32 on the accumulated values.
+ *   If a bounded device-side wait gives up (which indicates a fault in the pipeline, not a
+ *   property of the data), every sequence gets MARS_SEQ_TIMEOUT, accept_len 0, out_len 0 and
+ *   out_tokens / path_nodes filled with -1.
+ */
+mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const float *bias, int d,
+                                 const int32_t *tok, const int32_t *parent, int B, int N, int V,
+                                 float theta, uint32_t flags, int32_t *accept_len,
+                                 int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
+                                 int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Static, human-readable name of a status code (host memory, never NULL). */
 const char *mars_status_string(mars_status_t s);
 

@@ -60,6 +60,16 @@ int mars_oracle_threads(void)
 #endif
 }
 
+/* Host threads for the loop over rows (the container may see more cores than it may use). */
+void mars_oracle_set_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 /* bf16 is the upper half of an fp32 word: widening is exact. */
 static float bf16_to_f32(uint16_t h)
 {

@@ -51,6 +51,9 @@ def lib() -> ctypes.CDLL:
             vp, i32, i64, u32, f64 = (ctypes.c_void_p, ctypes.c_int, ctypes.c_int64,
                                       ctypes.c_uint32, ctypes.c_double)
             L.mars_oracle_threads.restype = ctypes.c_int
+            L.mars_oracle_set_threads.argtypes = [ctypes.c_int]
+            L.mars_oracle_set_threads.restype = None
+            L.mars_oracle_set_threads(usable_cores())
             L.mars_oracle_top2.argtypes = [vp, i32, i64, i64, i64, vp, vp]
             L.mars_oracle_top2.restype = None
             L.mars_oracle_relax_f32.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float, u32]
@@ -64,6 +67,31 @@ def lib() -> ctypes.CDLL:
             L.mars_oracle_verify_chain.restype = None
             _lib = L
     return _lib
+
+
+def usable_cores() -> int:
+    """Cores this process may really use: scheduler affinity, capped by the cgroup CPU quota.
+    OpenMP's default (every core of the machine) oversubscribes a quota-limited container."""
+    n = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    for path in ("/sys/fs/cgroup/cpu.max", "/sys/fs/cgroup/cpu/cpu.cfs_quota_us"):
+        try:
+            with open(path) as f:
+                parts = f.read().split()
+            if path.endswith("cpu.max"):
+                if parts[0] != "max":
+                    n = min(n, max(1, int(int(parts[0]) / int(parts[1]))))
+            else:
+                quota = int(parts[0])
+                if quota > 0:
+                    with open("/sys/fs/cgroup/cpu/cpu.cfs_period_us") as g:
+                        n = min(n, max(1, int(quota / int(g.read()))))
+            break
+        except Exception:
+            continue
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env and env.isdigit() and int(env) >= 1:
+        n = min(n, int(env))
+    return max(1, min(n, 32))
 
 
 def threads() -> int:

@@ -1,0 +1,478 @@
+// libmars: LM-head projection fused with the top-2 epilogue and the verification tail.
+//
+// z = H W^T (+ b)  (Eq. 2 of the paper: z_t = W_o h_t + b_o), H bf16 [M, d], W bf16 [V, d],
+// fp32 accumulation in tensor memory.  The logits are never written to HBM: each epilogue
+// thread owns one logits row (one TMEM lane) and keeps that row's running top-2 across the
+// vocabulary tiles it sees; 16-byte records go to the workspace and a small second kernel
+// merges them per row and runs the verification tail.
+//
+// Kernel 1 (persistent, one block per SM, 192 threads, warp-specialised):
+//   warp 0      TMA producer: H tile [128 x 64] and W tile [256 x 64] (128-byte swizzle) per
+//               k-block into a 4-stage shared-memory ring, completion on mbarriers.
+//   warp 1      allocates the 512 TMEM columns and issues tcgen05.mma (M=128, N=256, K=16,
+//               kind::f16 with bf16 operands, fp32 accumulate); tcgen05.commit releases the
+//               ring stage / publishes the accumulator.
+//   warps 2..5  epilogue: tcgen05.ld of the finished accumulator (double-buffered, so the next
+//               tile's MMAs overlap), bias, per-row running top-2.
+// Work item = (vocabulary chunk of kChunkTiles N-tiles, M-tile); items are dealt round-robin
+// with the M-tile index fastest, so the blocks that run together share W tiles through L2 and
+// W crosses HBM about once.
+//
+// Every wait on an mbarrier is bounded (clock64 budget).  A wait that gives up raises a
+// block-wide abort flag and a status word in the workspace; all roles then fall through to
+// the common exit, which drains outstanding copies (bounded), frees TMEM and returns.
+#include "mars_common.cuh"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdlib>
+#include <mutex>
+
+#include "mars.h"
+
+namespace mars {
+
+constexpr int kBM = 128;          // rows of H per tile = TMEM lanes
+constexpr int kBN = 256;          // vocabulary entries per tile = TMEM columns per accumulator
+constexpr int kBK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kStages = 4;
+constexpr int kChunkTiles = 6;    // N-tiles per work item
+constexpr int kLmThreads = 192;
+constexpr uint32_t kABytes = kBM * kBK * 2;   // 16 KB
+constexpr uint32_t kBBytes = kBN * kBK * 2;   // 32 KB
+constexpr uint32_t kStageBytes = kABytes + kBBytes;
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kWaitCycles = 2000000000ll;   // about a second at B200 clocks
+constexpr size_t kLmSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+
+struct LmParams {
+    int M, V, d;
+    int n_mtiles, n_ntiles, n_chunks, n_items;
+    const float *bias;   // [V] or null
+    Rec *partial;        // [M, n_chunks]
+    unsigned *status;    // workspace word: 0 ok, else MARS_SEQ_TIMEOUT
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the budget ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(status, (unsigned)MARS_SEQ_TIMEOUT);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// 32 lanes x 32 columns of 32-bit: thread t of the warp gets row (lane base + t), 32 columns.
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);   // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                         // leading byte offset (unused with swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                         // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                         // layout: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
+                            ((uint32_t)(kBM >> 4) << 24);
+
+// ----------------------------------------------------------------------------- GEMM + top-2
+
+__global__ void __launch_bounds__(kLmThreads, 1)
+lmhead_top2_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+                   const LmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned ring
+    const uint32_t bars = tiles + kStages * kStageBytes;           // barriers after the ring
+    const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
+    const uint32_t tfull0 = bars + 16 * kStages, tempty0 = tfull0 + 16, drain = tempty0 + 16;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kblocks = p.d / kBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+        mbar_init(drain, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int *abort_flag = &s_abort;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t armed = 0, armed_parity = 0;     // per-stage bit: a load is outstanding
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                const int mt = item % p.n_mtiles, chunk = item / p.n_mtiles;
+                const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
+                for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                        const uint32_t fb = full0 + 8 * stage;
+                        mbar_expect_tx(fb, kStageBytes);
+                        const uint32_t a_dst = tiles + stage * kStageBytes;
+                        tma_load_2d(a_dst, &map_h, kb * kBK, mt * kBM, fb);
+                        tma_load_2d(a_dst + kABytes, &map_w, kb * kBK, nt * kBN, fb);
+                        armed |= 1u << stage;
+                        armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (*abort_flag) {
+                // give this block's own outstanding copies a bounded time to land
+                for (int s = 0; s < kStages; ++s) {
+                    if (!(armed >> s & 1u)) continue;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full0 + 8 * s, (armed_parity >> s) & 1u) && clock64() - t0 < 20000000ll) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+                const int chunk = item / p.n_mtiles;
+                const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
+                for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+                    if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * kBN;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles + stage * kStageBytes;
+                        const uint64_t adesc = umma_desc_k_sw128(a_addr);
+                        const uint64_t bdesc = umma_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBK / kUmmaK; ++k)   // 32 bytes along K per step
+                            tc_mma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_commit(empty0 + 8 * stage);           // stage reusable once these MMAs retire
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit(tfull0 + 8 * acc);                 // accumulator complete
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                }
+            }
+            // all MMAs issued by this thread must retire before TMEM is freed
+            tc_commit(drain);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(drain, 0) && clock64() - t0 < kWaitCycles) {}
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                 // TMEM lanes this warp may read
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
+            const int mt = item % p.n_mtiles, chunk = item / p.n_mtiles;
+            const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
+            const int row = mt * kBM + row_in_tile;
+            Rec rec = empty_rec();
+            for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+                // warp-uniform outcome: the TMEM loads below are warp-collective
+                ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
+#pragma unroll 1
+                for (int c = 0; c < kBN / 32; ++c) {
+                    float v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    const int col0 = nt * kBN + c * 32;
+                    if (p.bias) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += (col0 + j < p.V) ? __ldg(p.bias + col0 + j) : 0.0f;
+                    }
+                    float m = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) m = fmaxf(m, v[j]);
+                    if (m > rec.z2) {   // columns come in increasing token id: equality never displaces
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float x = v[j];
+                            if (x > rec.z2 && col0 + j < p.V) {
+                                if (x > rec.z1) { rec.z2 = rec.z1; rec.id2 = rec.id1; rec.z1 = x; rec.id1 = col0 + j; }
+                                else { rec.z2 = x; rec.id2 = col0 + j; }
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty0 + 8 * acc);   // accumulator free for the next tile
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (ok && row < p.M) p.partial[(size_t)row * p.n_chunks + chunk] = rec;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ----------------------------------------------------------------------------- tail kernel
+
+__global__ void __launch_bounds__(128) lmhead_tail_kernel(const LmParams p, const TailArgs t)
+{
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    const int b = blockIdx.x;
+    if (*(volatile unsigned *)p.status != 0) {
+        // a device-side wait gave up: no valid result for any sequence
+        if (threadIdx.x == 0) {
+            t.accept_len[b] = 0;
+            t.out_len[b] = 0;
+            if (t.seq_status) t.seq_status[b] = MARS_SEQ_TIMEOUT;
+        }
+        for (int k = threadIdx.x; k <= t.Dcap; k += blockDim.x) {
+            t.out_tokens[(size_t)b * (t.Dcap + 1) + k] = -1;
+            if (t.path_nodes) t.path_nodes[(size_t)b * (t.Dcap + 1) + k] = -1;
+        }
+        return;
+    }
+    const int nch = p.n_chunks;
+    const Rec *base = p.partial + (size_t)b * t.N * nch;
+    verify_tail(t, b, smem_dyn, [&](int i) {
+        Rec acc = empty_rec();
+        for (int k = 0; k < nch; ++k) acc = merge(acc, base[(size_t)i * nch + k]);
+        return finish_record(acc);
+    });
+}
+
+// ----------------------------------------------------------------------------- host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    });
+    return fn;
+}
+
+// bf16 [rows, d] row-major -> boxes of [box_rows x 64] elements, 128-byte swizzle, zero fill.
+static bool make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t d, uint32_t box_rows)
+{
+    EncodeTiledFn enc = encode_tiled();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {d, rows};
+    cuuint64_t strides[1] = {d * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct LmShape { int n_mtiles, n_ntiles, n_chunks, n_items; };
+
+static LmShape lm_shape(long long M, int V)
+{
+    LmShape s;
+    s.n_mtiles = (int)((M + kBM - 1) / kBM);
+    s.n_ntiles = (V + kBN - 1) / kBN;
+    s.n_chunks = (s.n_ntiles + kChunkTiles - 1) / kChunkTiles;
+    s.n_items = s.n_mtiles * s.n_chunks;
+    return s;
+}
+
+static bool lm_supported(int B, int N, int V, int d)
+{
+    if (B < 1 || N < 1 || N > MARS_MAX_NODES || V < 2 || V > (1 << 30)) return false;
+    if (d < kBK || d % kBK != 0 || d > (1 << 20)) return false;
+    if ((long long)B * N > (1ll << 24)) return false;
+    return true;
+}
+
+}  // namespace mars
+
+extern "C" {
+
+size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d)
+{
+    if (!mars::lm_supported(B, N, V, d)) return 0;
+    const mars::LmShape s = mars::lm_shape((long long)B * N, V);
+    return 256 + (size_t)B * N * s.n_chunks * sizeof(mars::Rec);
+}
+
+mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const float *bias, int d,
+                                 const int32_t *tok, const int32_t *parent, int B, int N, int V, float theta,
+                                 uint32_t flags, int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
+                                 int32_t *out_len, int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
+                                 void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    using namespace mars;
+    if (!hidden || !w_vocab || !tok || !parent || !accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
+    if (B < 1 || N < 1 || V < 2 || d < 1 || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
+    if (((uintptr_t)hidden & 15) || ((uintptr_t)w_vocab & 15)) return MARS_ERR_INVALID_ARG;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT)) return MARS_ERR_UNSUPPORTED;
+    if (!lm_supported(B, N, V, d)) return MARS_ERR_UNSUPPORTED;
+    const size_t need = mars_lmhead_workspace_bytes(B, N, V, d);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;
+
+    const long long M = (long long)B * N;
+    const LmShape s = lm_shape(M, V);
+    LmParams p;
+    p.M = (int)M; p.V = V; p.d = d;
+    p.n_mtiles = s.n_mtiles; p.n_ntiles = s.n_ntiles; p.n_chunks = s.n_chunks; p.n_items = s.n_items;
+    p.bias = bias;
+    p.status = (unsigned *)workspace;
+    p.partial = (Rec *)((char *)workspace + 256);
+
+    CUtensorMap map_h, map_w;
+    if (!make_map(&map_h, hidden, (uint64_t)M, (uint64_t)d, kBM)) return MARS_ERR_CUDA;
+    if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, kBN)) return MARS_ERR_CUDA;
+
+    TailArgs t;
+    t.tok = tok; t.parent = parent; t.accept_len = accept_len; t.out_tokens = out_tokens;
+    t.path_nodes = path_nodes; t.out_len = out_len; t.seq_status = seq_status;
+    t.dbg_val = dbg ? dbg->top2_val : nullptr;
+    t.dbg_id = dbg ? dbg->top2_id : nullptr;
+    t.dbg_flags = dbg ? dbg->node_flags : nullptr;
+    t.N = N; t.Dcap = Dcap; t.theta = theta; t.flags = flags; t.chain = 0;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MARS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MARS_ERR_CUDA;
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kLmSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return MARS_ERR_CUDA;
+
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(p.status, 0, 256, st) != cudaSuccess) return MARS_ERR_CUDA;
+    const int grid = s.n_items < sms ? s.n_items : sms;
+    lmhead_top2_kernel<<<grid, kLmThreads, kLmSmemBytes, st>>>(map_h, map_w, p);
+    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    lmhead_tail_kernel<<<B, 128, tail_smem_bytes(N), st>>>(p, t);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+}
+
+}  // extern "C"

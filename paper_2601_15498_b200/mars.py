@@ -51,6 +51,11 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_tree.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, u32, vp, vp,
                                            vp, vp, i32, vp, ctypes.POINTER(_DebugOut), vp, sz, vp]
             L.mars_verify_tree.restype = i32
+            L.mars_lmhead_workspace_bytes.argtypes = [i32, i32, i32, i32]
+            L.mars_lmhead_workspace_bytes.restype = sz
+            L.mars_lmhead_verify.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, f32, u32, vp, vp,
+                                             vp, vp, i32, vp, ctypes.POINTER(_DebugOut), vp, sz, vp]
+            L.mars_lmhead_verify.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -158,6 +163,50 @@ def verify_chain(logits: torch.Tensor, draft, theta: float, flags: int = 0, V: i
             ctypes.byref(dbg) if dbg is not None else None, workspace.data_ptr(), wbytes, _stream())
     _check(code, "mars_verify_chain")
     out["_keepalive"] = (draft, workspace)
+    return out
+
+
+def lmhead_verify(hidden: torch.Tensor, w_vocab: torch.Tensor, bias, tok, parent, theta: float,
+                  flags: int = 0, Dcap: int | None = None, debug: bool = False,
+                  workspace: torch.Tensor | None = None, out: dict | None = None) -> dict:
+    """mars_lmhead_verify on the current stream: hidden bf16 [B*N, d], w_vocab bf16 [V, d]."""
+    dev = hidden.device
+    if not (hidden.is_cuda and w_vocab.is_cuda and hidden.dtype == torch.bfloat16
+            and w_vocab.dtype == torch.bfloat16 and hidden.is_contiguous() and w_vocab.is_contiguous()):
+        raise MarsError("hidden and w_vocab must be contiguous bfloat16 device tensors")
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    M, d = hidden.shape
+    V = w_vocab.shape[0]
+    if M != B * N or w_vocab.shape[1] != d:
+        raise MarsError("shape mismatch")
+    if bias is not None:
+        bias = bias.to(device=dev, dtype=torch.float32).contiguous()
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    need = int(lib().mars_lmhead_workspace_bytes(B, N, V, d))
+    if need == 0:
+        raise MarsError("unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if out is None:
+        out = alloc_outputs(B, N, Dcap, dev, debug)
+    dbg = None
+    if "top2_val" in out:
+        dbg = _DebugOut(out["top2_val"].data_ptr(), out["top2_id"].data_ptr(),
+                        out["node_flags"].data_ptr())
+    with torch.cuda.device(dev):
+        code = lib().mars_lmhead_verify(
+            hidden.data_ptr(), w_vocab.data_ptr(), bias.data_ptr() if bias is not None else None, d,
+            tok.data_ptr(), parent.data_ptr(), B, N, V, float(theta), flags,
+            out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(), out["path_nodes"].data_ptr(),
+            out["out_len"].data_ptr(), Dcap, out["seq_status"].data_ptr(),
+            ctypes.byref(dbg) if dbg is not None else None, workspace.data_ptr(),
+            workspace.numel(), _stream())
+    _check(code, "mars_lmhead_verify")
+    out["_keepalive"] = (tok, parent, workspace, bias)
     return out
 
 
