@@ -140,8 +140,10 @@ def make_tokens(parent: np.ndarray, lead: np.ndarray, V: int, seed: int, p_top1:
             t = _draft_mix(rng, lead[b, p], V, p_top1, p_top2)
             if dedupe_siblings:
                 s = seen.setdefault(p, set())
-                while t in s:
+                tries = 0
+                while t in s and len(s) < V and tries < 64:   # tiny vocabularies may not allow it
                     t = int(rng.integers(V))
+                    tries += 1
                 s.add(t)
             tok[b, i] = t
     return tok
