@@ -39,12 +39,15 @@ HBM_NOMINAL_GBS = 8000.0
 HBM_FALLBACK_GBS = 6650.0
 
 WORKLOADS = {
-    "cfg3_bf16": lambda dev, seed: synth.cfg3(dev, seed=seed, dtype=torch.bfloat16),
-    "cfg3_fp32": lambda dev, seed: synth.cfg3(dev, seed=seed, dtype=torch.float32),
-    "cfg2": lambda dev, seed: synth.cfg2(dev, seed=seed),
-    "cfg1": lambda dev, seed: synth.cfg1(dev, seed=seed),
-    "cfg0": lambda dev, seed: synth.cfg0(dev, seed=seed),
+    "cfg3_bf16": lambda dev, seed, B=256: synth.cfg3(dev, seed=seed, B=B, dtype=torch.bfloat16),
+    "cfg3_fp32": lambda dev, seed, B=256: synth.cfg3(dev, seed=seed, B=B, dtype=torch.float32),
+    "cfg2": lambda dev, seed, B=64: synth.cfg2(dev, seed=seed, B=B),
+    "cfg1": lambda dev, seed, B=1: synth.cfg1(dev, seed=seed, B=B),
+    "cfg0": lambda dev, seed, B=1: synth.cfg0(dev, seed=seed, B=B),
 }
+FULL_NAME = {"cfg3_bf16": "cfg3_tree_b256_n60_v151936_bf16", "cfg3_fp32": "cfg3_tree_b256_n60_v151936_fp32",
+             "cfg2": "cfg2_chain_b64_k8_v151936_bf16", "cfg1": "cfg1_tree_b1_n60_v151936_bf16",
+             "cfg0": "cfg0_chain_b1_k6_v32000_fp32"}
 BASE_SEED = {"cfg3_bf16": 3, "cfg3_fp32": 3, "cfg2": 2, "cfg1": 1, "cfg0": 0}
 
 
@@ -175,8 +178,8 @@ def reference_arm(args, rank: int):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.logits.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "B": w.B, "N": w.N, "V": w.V, "theta": w.theta,
-                   "note": "CPU oracle; each step is a bounded sample of the workload"},
+        "config": {"workload": FULL_NAME[args.workload], "B": w.B, "N": w.N, "V": w.V, "theta": w.theta,
+                   "note": "CPU oracle; each step is a bounded sample (B sequences) of the workload"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{seqs} sequences x {w.N} rows per step"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -194,6 +197,8 @@ def main():
     ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the number of sequences (smaller cases for profiler captures)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -221,7 +226,10 @@ def main():
     mars.lib()
 
     # ---- inputs, resident in HBM; every rank gets its own batch of the same shape ----
-    w = WORKLOADS[args.workload](dev, BASE_SEED[args.workload] + 1000 * rank)
+    if args.batch:
+        w = WORKLOADS[args.workload](dev, BASE_SEED[args.workload] + 1000 * rank, args.batch)
+    else:
+        w = WORKLOADS[args.workload](dev, BASE_SEED[args.workload] + 1000 * rank)
     dt_code = mars.BF16 if w.logits.dtype == torch.bfloat16 else mars.FP32
     copies = 1
     if w.logits_bytes < 3 * L2_BYTES:   # small workloads: rotate over copies so that no step finds
@@ -261,36 +269,41 @@ def main():
     ms_per_step = total_ms / args.steps
 
     # ---- end to end: host buffers in, results out, copies inside the timed region ----
-    h_logits = torch.empty(w.logits.shape, dtype=w.logits.dtype, pin_memory=True)
-    h_logits.copy_(w.logits)
-    h_tok = torch.as_tensor(w.tok).pin_memory()
-    h_par = torch.as_tensor(w.parent).pin_memory()
-    h_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype, pin_memory=True)
-             for k in ("accept_len", "out_tokens", "out_len")}
-    d_logits = torch.empty_like(w.logits)
+    e2e = None
+    h_logits = None
+    if args.e2e_steps > 0:
+        h_logits = torch.empty(w.logits.shape, dtype=w.logits.dtype, pin_memory=True)
+        h_logits.copy_(w.logits)
+        h_tok = torch.as_tensor(w.tok).pin_memory()
+        h_par = torch.as_tensor(w.parent).pin_memory()
+        h_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype, pin_memory=True)
+                 for k in ("accept_len", "out_tokens", "out_len")}
+        d_logits = torch.empty_like(w.logits)
 
-    def e2e_step():
-        d_logits.copy_(h_logits, non_blocking=True)
-        tok.copy_(h_tok, non_blocking=True)
-        parent.copy_(h_par, non_blocking=True)
-        if w.kind == "chain":
-            draft.copy_(tok[:, 1:])
-        step(0, d_logits)
-        for k, h in h_out.items():
-            h.copy_(out[k], non_blocking=True)
+        def e2e_step():
+            d_logits.copy_(h_logits, non_blocking=True)
+            tok.copy_(h_tok, non_blocking=True)
+            parent.copy_(h_par, non_blocking=True)
+            if w.kind == "chain":
+                draft.copy_(tok[:, 1:])
+            step(0, d_logits)
+            for k, h in h_out.items():
+                h.copy_(out[k], non_blocking=True)
 
-    e2e_step()
-    torch.cuda.synchronize()
-    barrier(world)
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for _ in range(args.e2e_steps):
         e2e_step()
-    f1.record()
-    torch.cuda.synchronize()
-    e2e_ms, e2e_units = reduce_max_time_sum_units(f0.elapsed_time(f1), float(w.R * args.e2e_steps), world)
-    h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4
-    d2h = sum(h.numel() * h.element_size() for h in h_out.values())
+        torch.cuda.synchronize()
+        barrier(world)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        f1.record()
+        torch.cuda.synchronize()
+        e2e_ms, e2e_units = reduce_max_time_sum_units(f0.elapsed_time(f1), float(w.R * args.e2e_steps), world)
+        h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4
+        d2h = sum(h.numel() * h.element_size() for h in h_out.values())
+        e2e = {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
 
     if rank != 0:
         if world > 1:
@@ -311,7 +324,7 @@ def main():
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        host = synth.to_numpy_bits(h_logits)
+        host = synth.to_numpy_bits(h_logits if h_logits is not None else w.logits)
         seqs = min(w.B, max(1, 7680 // w.N))
         run_oracle_sample(w, host, min(seqs, 2))
         dt, n, cores = run_oracle_sample(w, host, seqs)
@@ -331,8 +344,7 @@ def main():
         "us_per_step": 1e3 * ms_per_step,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,
         "clocks": clocks.summary(),
-        "e2e": {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps},
+        "e2e": e2e,
         "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,

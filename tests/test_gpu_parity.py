@@ -263,7 +263,7 @@ def test_host_errors_launch_nothing():
     out = mars.alloc_outputs(2, 5, 4, DEV)
     with pytest.raises(mars.MarsError, match="invalid argument"):
         mars.verify_tree(w.logits, w.tok, w.parent, float("nan"), out=out)
-    with pytest.raises(mars.MarsError, match="invalid argument"):
+    with pytest.raises(mars.MarsError, match="unsupported sizes"):      # V < 2: no workspace size
         mars.verify_tree(w.logits, w.tok, w.parent, 0.9, V=1, out=out)
     with pytest.raises(mars.MarsError, match="workspace"):
         mars.verify_tree(w.logits, w.tok, w.parent, 0.9, out=out,
