@@ -41,7 +41,8 @@ typedef enum {
     MARS_ERR_INVALID_ARG = 1, /* NULL required pointer, B<1, N<1, V<2, ld<V, NaN theta, ... */
     MARS_ERR_WORKSPACE = 2,   /* workspace NULL, misaligned (256 B) or too small           */
     MARS_ERR_UNSUPPORTED = 3, /* N or V above the supported caps, unknown dtype / flag      */
-    MARS_ERR_CUDA = 4         /* a CUDA runtime call (memset / launch) reported an error    */
+    MARS_ERR_CUDA = 4,        /* a CUDA runtime call (memset / launch) reported an error    */
+    MARS_ERR_STATIC_CAPACITY = 5 /* mars_verify_tree_static: batch too large for the built-in scratch */
 } mars_status_t;
 
 typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
@@ -163,6 +164,46 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
                                  int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
                                  int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * mars_verify_tree for callers that must not allocate device memory.  (The paper has no
+ * counterpart; this is a deployment convenience of the library.)
+ *
+ * Who needs it: code that runs inside somebody else's memory regime -- an inference server
+ * that has handed all free HBM to its KV-cache pool at start-up, a plug-in op inside another
+ * runtime, a latency-critical loop where cudaMalloc's implicit device synchronisation is not
+ * acceptable.  Such callers cannot create the workspace that mars_verify_tree asks for, so
+ * this variant brings its own: a fixed array of mars_static_scratch_bytes() bytes (1 MiB)
+ * that is part of the library image.  Every GPU on which the library is loaded holds that
+ * array until the process exits, whether or not this function is ever called.
+ *
+ * The function itself calls no cudaMalloc / cudaFree and no allocating library routine; it
+ * issues one cudaMemsetAsync (a few bytes) and one kernel launch on `cuda_stream`, exactly
+ * like mars_verify_tree.  Inputs and outputs are still the caller's buffers.
+ *
+ *   - Capacity: the batch must satisfy mars_workspace_bytes(B, N, V, dt) <=
+ *     mars_static_scratch_bytes(); otherwise MARS_ERR_STATIC_CAPACITY is returned and
+ *     nothing is launched.  (The serving-scale batch of 256 x 60 rows needs 241 KiB.)
+ *   - First call on a device: looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and caches it per device.  Make this first call outside any stream
+ *     capture.  A failure of the look-up is reported as MARS_ERR_CUDA.
+ *   - All calls on one device share the one array.  It keeps whatever the previous call left
+ *     in it; the function clears the part that must start at zero (the per-sequence arrival
+ *     counters) on the stream before its kernel.  Two calls whose GPU work may overlap --
+ *     different streams without an ordering between them, or several host threads -- race on
+ *     the array and give undefined results: serialise them, or use mars_verify_tree with
+ *     separate workspaces.
+ *   - Arguments, outputs and statuses otherwise as mars_verify_tree.
+ */
+mars_status_t mars_verify_tree_static(const void *logits, int64_t ld, mars_dtype_t dt,
+                                      const int32_t *tok, const int32_t *parent, int B, int N,
+                                      int V, float theta, uint32_t flags, int32_t *accept_len,
+                                      int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
+                                      int Dcap, int32_t *seq_status, const mars_debug_out_t *dbg,
+                                      void *cuda_stream);
+
+/* Size in bytes of the built-in scratch array used by mars_verify_tree_static (host, pure). */
+size_t mars_static_scratch_bytes(void);
 
 /* Static, human-readable name of a status code (host memory, never NULL). */
 const char *mars_status_string(mars_status_t s);

@@ -25,6 +25,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 #include "mars.h"
 
@@ -390,9 +391,63 @@ mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt, 
                      path_nodes, out_len, Dcap, seq_status, dbg, workspace, workspace_bytes, cuda_stream);
 }
 
+// ---- verification without any caller-provided or allocated scratch -------------------------
+//
+// Scratch for mars_verify_tree_static lives in this fixed device array.  Every GPU that loads
+// the library keeps these bytes until the process exits.  In host code the name
+// `g_static_scratch` is only a handle for the runtime, not a device address: the address
+// that kernels can use is obtained once per device with cudaGetSymbolAddress.
+#define MARS_STATIC_SCRATCH_BYTES (1u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[MARS_STATIC_SCRATCH_BYTES];
+
+namespace mars {
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mu;
+static void *g_static_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (looked up on first use).
+static mars_status_t static_scratch(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MARS_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return MARS_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return MARS_OK;
+}
+}  // namespace mars
+
+size_t mars_static_scratch_bytes(void) { return MARS_STATIC_SCRATCH_BYTES; }
+
+mars_status_t mars_verify_tree_static(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
+                                      const int32_t *parent, int B, int N, int V, float theta,
+                                      uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
+                                      int32_t *path_nodes, int32_t *out_len, int Dcap,
+                                      int32_t *seq_status, const mars_debug_out_t *dbg, void *cuda_stream)
+{
+    // sizes first: nothing is looked up or launched for a batch that cannot fit
+    const size_t need = mars_workspace_bytes(B, N, V, dt);
+    if (need == 0) return (B < 1 || N < 1 || V < 2) ? MARS_ERR_INVALID_ARG : MARS_ERR_UNSUPPORTED;
+    if (need > MARS_STATIC_SCRATCH_BYTES) return MARS_ERR_STATIC_CAPACITY;
+    void *scratch = nullptr;
+    const mars_status_t st = mars::static_scratch(&scratch);
+    if (st != MARS_OK) return st;
+    // The arrival counters at the front of the scratch must start at zero; run() clears them
+    // on the stream before the kernel.  Everything else in the array is overwritten before
+    // it is read, so the previous call's leftovers are harmless.
+    return mars::run(logits, ld, dt, tok, parent, 0, B, N, V, theta, flags, accept_len, out_tokens,
+                     path_nodes, out_len, Dcap, seq_status, dbg, scratch, MARS_STATIC_SCRATCH_BYTES,
+                     cuda_stream);
+}
+
 const char *mars_status_string(mars_status_t s)
 {
     switch (s) {
+    case MARS_ERR_STATIC_CAPACITY: return "batch needs more scratch than the built-in static array holds";
     case MARS_OK: return "ok";
     case MARS_ERR_INVALID_ARG: return "invalid argument";
     case MARS_ERR_WORKSPACE: return "workspace missing, misaligned or too small";

@@ -56,6 +56,11 @@ def lib() -> ctypes.CDLL:
             L.mars_lmhead_verify.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, f32, u32, vp, vp,
                                              vp, vp, i32, vp, ctypes.POINTER(_DebugOut), vp, sz, vp]
             L.mars_lmhead_verify.restype = i32
+            L.mars_verify_tree_static.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, u32, vp,
+                                                  vp, vp, vp, i32, vp, ctypes.POINTER(_DebugOut), vp]
+            L.mars_verify_tree_static.restype = i32
+            L.mars_static_scratch_bytes.argtypes = []
+            L.mars_static_scratch_bytes.restype = sz
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -136,6 +141,39 @@ def verify_tree(logits: torch.Tensor, tok, parent, theta: float, flags: int = 0,
             workspace.data_ptr(), wbytes, _stream())
     _check(code, "mars_verify_tree")
     out["_keepalive"] = (tok, parent, workspace)
+    return out
+
+
+def verify_tree_static(logits: torch.Tensor, tok: torch.Tensor, parent: torch.Tensor, theta: float,
+                       out: dict, flags: int = 0, Dcap: int | None = None,
+                       V: int | None = None) -> dict:
+    """mars_verify_tree_static on the current stream.
+
+    For callers that may not allocate device memory: the library's built-in scratch array
+    replaces the workspace, and this wrapper allocates nothing either -- `tok`, `parent`
+    (int32 device tensors) and every buffer in `out` (see ``alloc_outputs``) must already
+    exist.  Calls that may overlap on the GPU must not share a device (they share the array).
+    """
+    dev = logits.device
+    for t in (tok, parent):
+        if not (t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()):
+            raise MarsError("tok and parent must be contiguous int32 device tensors")
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    dt, ld, V = _logits_args(logits, B * N, V)
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    dbg = None
+    if "top2_val" in out:
+        dbg = _DebugOut(out["top2_val"].data_ptr(), out["top2_id"].data_ptr(),
+                        out["node_flags"].data_ptr())
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_tree_static(
+            logits.data_ptr(), ld, dt, tok.data_ptr(), parent.data_ptr(), B, N, V, float(theta),
+            flags, out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(),
+            out["path_nodes"].data_ptr(), out["out_len"].data_ptr(), Dcap,
+            out["seq_status"].data_ptr(), ctypes.byref(dbg) if dbg is not None else None, _stream())
+    _check(code, "mars_verify_tree_static")
     return out
 
 
