@@ -122,6 +122,19 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def ncu_traffic(workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic_per_launch.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 2 and parts[0] == workload:
+                    return int(parts[1])
+    except Exception:
+        pass
+    return None
+
+
 def reduce_max_time_sum_units(elapsed_ms: float, units: float, world: int):
     """Whole-job figures from per-rank ones: slowest rank's time, all ranks' units."""
     if world == 1:
@@ -188,15 +201,173 @@ def reference_arm(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
+def measured_bf16_peak(sustained: bool):
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    key = "bf16_tflops_sustained" if sustained else "bf16_tflops"
+    try:
+        with open(path) as f:
+            return float(json.load(f)[key]), f"measured (MEASURED_PEAKS.json, {key})"
+    except Exception:
+        return (1400.0 if sustained else 1590.0), "fallback (earlier pool measurement)"
+
+
+def lmhead_arm(args, rank: int, world: int, local: int):
+    """Fused LM-head + tree verification: hidden [64 x 60, 4096] bf16, W_vocab [151 936, 4096]
+    bf16 (a model weight: resident in HBM in both the device-timed and the end-to-end figure),
+    logits never stored.  Bound: tensor pipe (2 M d V flop per step)."""
+    from paper_2601_15498_b200 import build, mars
+    steps = 30 if args.steps is None else args.steps
+    warm = 3 if args.warmup is None else max(args.warmup, 3)
+    B = args.batch or 64
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        from oracle import mars_oracle as orc
+        w = synth.cfg4_operands("cpu", seed=4, B=1)
+        hb, wb = synth.to_numpy_bits(w.hidden), synth.to_numpy_bits(w.w_vocab)
+        tok = np.full((1, w.N), -1, np.int32)
+        t = 0.0
+        n = max(1, min(steps, 2))
+        for _ in range(n):
+            t0 = time.perf_counter()
+            orc.lmhead_verify_tree(hb, wb, None, tok, w.parent, w.theta)
+            t += time.perf_counter() - t0
+        value = w.N * n / t
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": n, "warmup": 0, "ms_per_step": 1e3 * t / n, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "cfg4_lmhead_b64_n60_v151936_d4096", "B": 1, "N": w.N, "V": w.V,
+                       "d": w.d, "note": "fp64 oracle; each step is one sequence (60 rows)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.usable_cores(), "kind": "oracle",
+                             "sample": "1 sequence x 60 rows per step (numpy fp64 matmul + C rule)"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}), flush=True)
+        return
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build()
+    barrier(world)
+    w = synth.cfg4_operands(dev, seed=4 + 1000 * rank, B=B)
+    M = w.B * w.N
+    # draft tokens aim at the leading ids of a device fp32 matmul (inputs only)
+    lead = np.empty((M, 2), np.int64)
+    for r0 in range(0, M, 480):
+        zz = w.hidden[r0:r0 + 480].float() @ w.w_vocab.float().T
+        lead[r0:r0 + 480] = torch.topk(zz, 2, dim=1).indices.cpu().numpy()
+        del zz
+    tok_h = synth.make_tokens(w.parent, lead, w.V, 4)
+    tok = torch.as_tensor(tok_h, device=dev)
+    parent = torch.as_tensor(w.parent, device=dev)
+    ws = torch.empty(int(mars.lib().mars_lmhead_workspace_bytes(w.B, w.N, w.V, w.d)), dtype=torch.uint8, device=dev)
+    out = mars.alloc_outputs(w.B, w.N, w.N - 1, dev)
+    flush = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=dev)
+
+    def step(h=None):
+        mars.lmhead_verify(w.hidden if h is None else h, w.w_vocab, None, tok, parent, w.theta,
+                           workspace=ws, out=out)
+
+    for _ in range(warm):
+        step()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier(world)
+    with ClockSampler(local) as clocks:
+        if args.profiler_range:
+            torch.cuda.profiler.start()
+        for a, b in evs:
+            flush.zero_()                      # L2 flush between timed steps (outside the events)
+            a.record()
+            step()
+            b.record()
+        torch.cuda.synchronize()
+        if args.profiler_range:
+            torch.cuda.profiler.stop()
+    barrier(world)
+    elapsed_ms = sum(a.elapsed_time(b) for a, b in evs)
+    total_ms, total_units = reduce_max_time_sum_units(elapsed_ms, float(M * steps), world)
+
+    e2e = None
+    if args.e2e_steps > 0:
+        h_hidden = torch.empty(w.hidden.shape, dtype=w.hidden.dtype, pin_memory=True).copy_(w.hidden)
+        h_tok, h_par = torch.as_tensor(tok_h).pin_memory(), torch.as_tensor(w.parent).pin_memory()
+        h_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype, pin_memory=True)
+                 for k in ("accept_len", "out_tokens", "out_len")}
+        d_hidden = torch.empty_like(w.hidden)
+
+        def e2e_step():
+            d_hidden.copy_(h_hidden, non_blocking=True)
+            tok.copy_(h_tok, non_blocking=True)
+            parent.copy_(h_par, non_blocking=True)
+            step(d_hidden)
+            for k, h in h_out.items():
+                h.copy_(out[k], non_blocking=True)
+        e2e_step()
+        torch.cuda.synchronize()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        f1.record()
+        torch.cuda.synchronize()
+        e_ms, e_units = reduce_max_time_sum_units(f0.elapsed_time(f1), float(M * args.e2e_steps), world)
+        e2e = {"value": e_units / (e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h_hidden.numel() * 2 + h_tok.numel() * 4 + h_par.numel() * 4,
+               "d2h_bytes_per_step": sum(h.numel() * h.element_size() for h in h_out.values()),
+               "steps": args.e2e_steps, "note": "W_vocab is a model weight and stays resident"}
+    if rank != 0:
+        return
+    status = out["seq_status"].cpu().numpy()
+    flops = 2.0 * M * w.d * w.V
+    ms = elapsed_ms / steps
+    tfs = flops / (ms * 1e-3) / 1e12
+    peak, src = measured_bf16_peak(sustained=False)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import mars_oracle as orc
+        hb = synth.to_numpy_bits(w.hidden[:w.N])
+        wb = synth.to_numpy_bits(w.w_vocab)
+        t0 = time.perf_counter()
+        orc.lmhead_verify_tree(hb, wb, None, tok_h[:1], w.parent[:1], w.theta)
+        dt = time.perf_counter() - t0
+        cpu = {"value": w.N / dt, "unit": UNIT, "cores": orc.usable_cores(), "kind": "oracle",
+               "sample": f"first sequence ({w.N} rows): numpy fp64 projection + C rule, {dt:.1f} s"}
+    print(json.dumps({
+        "metric": METRIC, "value": total_units / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": warm, "ms_per_step": total_ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "N": w.N, "V": w.V, "d": w.d, "theta": w.theta,
+                   "l2": "L2 flushed (252 MB write) before every timed step",
+                   "all_sequences_ok": bool((status == 0).all())},
+        "us_per_step": 1e3 * total_ms / steps, "tflops": tfs,
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 2 * steps,
+        "roofline": {"bound": "tensor", "achieved": tfs, "peak": peak, "unit": "TFLOP/s",
+                     "frac": tfs / peak, "traffic": None, "peak_source": src,
+                     "kernel": "mars::lmhead_top2_kernel", "algorithmic_flops_per_launch": flops},
+        "cpu_baseline": cpu}), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS) + ["cfg4"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profiler-range", action="store_true",
+                    help="cudaProfilerStart/Stop around the timed region (for ncu --profile-from-start off)")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the steps from a CUDA graph (device time of launch-bound workloads)")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences (smaller cases for profiler captures)")
     args = ap.parse_args()
@@ -205,6 +376,9 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
 
+    if args.workload == "cfg4":
+        lmhead_arm(args, rank, world, local)
+        return
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
@@ -252,16 +426,38 @@ def main():
         step(i)
     torch.cuda.synchronize()
 
+    graph = None
+    if args.graph:      # one graph = one pass over the rotating input copies
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(copies):
+                step(i)
+        replays = max(1, -(-args.steps // copies))
+        args.steps = replays * copies
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+
     # ---- timed region: K steps between two events on the launching stream ----
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(world)
     torch.cuda.synchronize()
     with ClockSampler(local) as clocks:
+        if args.profiler_range:
+            torch.cuda.profiler.start()
         e0.record()
-        for i in range(args.steps):
-            step(i)
+        if graph is not None:
+            for _ in range(replays):
+                graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
         e1.record()
         torch.cuda.synchronize()
+        if args.profiler_range:
+            torch.cuda.profiler.stop()
     barrier(world)
     elapsed_ms = e0.elapsed_time(e1)
     total_ms, total_units = reduce_max_time_sum_units(elapsed_ms, float(w.R * args.steps), world)
@@ -314,13 +510,7 @@ def main():
     # ---- roofline of the one kernel on the path (algorithmic bytes: every logit once) ----
     peak, peak_src = measured_hbm_peak()
     achieved = w.logits_bytes / (elapsed_ms / args.steps * 1e-3) / 1e9
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        try:
-            traffic = json.load(open(tpath)).get(args.workload)
-        except Exception:
-            traffic = None
+    traffic = ncu_traffic(args.workload) if not args.batch else None
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -340,6 +530,7 @@ def main():
                    "theta": w.theta, "rows_per_step": w.R, "logits_bytes_per_step": w.logits_bytes,
                    "l2": ("inputs larger than L2" if copies == 1 else
                           f"rotating over {copies} input copies, {copies * w.logits_bytes} B > L2"),
+                   "launch": "cuda graph replay" if graph is not None else "direct launches",
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "us_per_step": 1e3 * ms_per_step,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,

@@ -5,7 +5,7 @@
 // from HBM with 16-byte loads.  Each thread keeps an exact top-2 (values and token ids) in
 // registers, but touches it only for the few batches that can still change the answer:
 //
-//   - a batch of kU 16-byte vectors per thread is first reduced to its maximum with packed
+//   - a batch of kU (8) 16-byte vectors per thread is first reduced to its maximum with packed
 //     bf16x2 (or fp32) max instructions -- about one instruction per two bf16 elements;
 //   - the batch is skipped unless its maximum beats the thread's own runner-up AND is not
 //     below T2, a lower bound on the slice's runner-up value that the whole block shares
@@ -32,7 +32,8 @@
 namespace mars {
 
 constexpr int kThreads = 256;  // threads per block
-constexpr int kU = 4;          // 16-byte vectors per thread per batch (64 B in flight each)
+constexpr int kU = 8;          // 16-byte vectors per thread per batch (128 B in flight each)
+static_assert(kU >= 4 && (kU & (kU - 1)) == 0, "kU must be a power of two >= 4");
 constexpr int kTargetBlocks = 148 * 8;     // split rows until the grid has about this many blocks
 constexpr int kMinSliceBytes = 8 * 1024;   // ... but never below this many bytes per slice
 
@@ -45,6 +46,8 @@ struct Params {
     int L;   // elements per slice (multiple of 16)
     Rec *partial;        // [R*S]
     unsigned *counters;  // [B]
+    int stage_partials;  // last block copies the sequence's N*S records to shared memory first
+    int tail_smem_off;   // byte offset of that staging area in dynamic shared memory
     TailArgs tail;
 };
 
@@ -173,7 +176,14 @@ __device__ __forceinline__ float load_batch(const uint4 *vbase, int v0, int nvec
     }
 #pragma unroll
     for (int u = 0; u < kU; ++u) q[u] = E::vred(v[u]);
-    return E::to_float(E::pmax(E::pmax(q[0], q[1]), E::pmax(q[2], q[3])));
+    typename E::packed_t m[kU / 2];
+#pragma unroll
+    for (int u = 0; u < kU / 2; ++u) m[u] = E::pmax(q[2 * u], q[2 * u + 1]);
+#pragma unroll
+    for (int w = kU / 4; w > 0; w >>= 1)
+#pragma unroll
+        for (int u = 0; u < w; ++u) m[u] = E::pmax(m[u], m[u + w]);
+    return E::to_float(m[0]);
 }
 
 template <int DT>
@@ -267,10 +277,25 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
     __threadfence();
     const int S = p.S;
     const Rec *seq_partial = p.partial + (size_t)b * p.N * S;
-    verify_tail(p.tail, b, smem_dyn, [&](int i) {
+    unsigned char *tail_smem = smem_dyn;
+    const Rec *src = seq_partial;
+    if (p.stage_partials) {
+        // Bring all N*S records in with independent coalesced loads (one memory latency
+        // instead of S dependent ones per row), then merge out of shared memory.
+        Rec *s_part = reinterpret_cast<Rec *>(smem_dyn + p.tail_smem_off);
+        for (int f = tid; f < p.N * S; f += kThreads) {
+            int4 w = __ldcg(reinterpret_cast<const int4 *>(seq_partial + f));
+            *reinterpret_cast<int4 *>(s_part + f) = w;
+        }
+        __syncthreads();
+        src = s_part;
+    }
+    const bool staged = p.stage_partials != 0;
+    verify_tail(p.tail, b, tail_smem, [&](int i) {
         Rec acc = empty_rec();
         for (int k = 0; k < S; ++k) {
-            int4 w = __ldcg(reinterpret_cast<const int4 *>(seq_partial + (size_t)i * S + k));
+            const int4 *q = reinterpret_cast<const int4 *>(src + (size_t)i * S + k);
+            int4 w = staged ? *q : __ldcg(q);
             Rec r;
             r.z1 = __int_as_float(w.x); r.id1 = w.y; r.z2 = __int_as_float(w.z); r.id2 = w.w;
             acc = merge(acc, r);
@@ -351,7 +376,12 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (cudaMemsetAsync(p.counters, 0, (size_t)B * sizeof(unsigned), st) != cudaSuccess) return MARS_ERR_CUDA;
     const unsigned grid = (unsigned)(R * sp.S);
-    const size_t smem = tail_smem_bytes(N);
+    // dynamic shared memory: the tail's arrays, then (if it fits in 48 KB) room for N*S records
+    const size_t tail_bytes = (tail_smem_bytes(N) + 15) / 16 * 16;
+    const size_t stage_bytes = (size_t)N * sp.S * sizeof(Rec);
+    p.stage_partials = (sp.S > 1 && tail_bytes + stage_bytes <= 48 * 1024) ? 1 : 0;
+    p.tail_smem_off = (int)tail_bytes;
+    const size_t smem = tail_bytes + (p.stage_partials ? stage_bytes : 0);
     if (dt == MARS_BF16) verify_kernel<MARS_BF16><<<grid, kThreads, smem, st>>>(p);
     else verify_kernel<MARS_FP32><<<grid, kThreads, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
