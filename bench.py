@@ -415,12 +415,15 @@ def main():
     ws = torch.empty(mars.workspace_bytes(w.B, w.N, w.V, dt_code), dtype=torch.uint8, device=dev)
     out = mars.alloc_outputs(w.B, w.N, w.N - 1, dev)
 
+    ws.zero_()
+    fl = mars.COUNTERS_ZERO     # the workspace starts zeroed and every call leaves its counters at zero
+
     def step(i, lg=None):
         lg = logits[i % copies] if lg is None else lg
         if w.kind == "chain":
-            mars.verify_chain(lg, draft, w.theta, workspace=ws, out=out)
+            mars.verify_chain(lg, draft, w.theta, flags=fl, workspace=ws, out=out)
         else:
-            mars.verify_tree(lg, tok, parent, w.theta, workspace=ws, out=out)
+            mars.verify_tree(lg, tok, parent, w.theta, flags=fl, workspace=ws, out=out)
 
     for i in range(args.warmup):
         step(i)
@@ -531,6 +534,7 @@ def main():
                    "l2": ("inputs larger than L2" if copies == 1 else
                           f"rotating over {copies} input copies, {copies * w.logits_bytes} B > L2"),
                    "launch": "cuda graph replay" if graph is not None else "direct launches",
+                   "workspace": "zeroed once; MARS_COUNTERS_ZERO (counters reset by the kernel itself)",
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "us_per_step": 1e3 * ms_per_step,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,

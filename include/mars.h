@@ -50,6 +50,11 @@ typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
 /* flags */
 #define MARS_SIGN_LITERAL 1u  /* drop the z1 > 0 guard: relax whenever z2/z1 > theta          */
 #define MARS_SHARED_PARENT 2u /* `parent` is one [N] array shared by all sequences            */
+#define MARS_COUNTERS_ZERO 4u /* mars_verify_chain / _tree: the caller guarantees that the first
+                                 4*B bytes of `workspace` are zero, which holds after a
+                                 cudaMemset of the workspace and after every completed call of
+                                 these functions on it with at least B sequences; the library
+                                 then skips its own clearing of those bytes (one stream op less) */
 
 #define MARS_MAX_NODES 1024   /* cap on N (rows per sequence)                                 */
 

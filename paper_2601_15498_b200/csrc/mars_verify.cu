@@ -10,8 +10,9 @@
 //   - the batch is skipped unless its maximum beats the thread's own runner-up AND is not
 //     below T2, a lower bound on the slice's runner-up value that the whole block shares
 //     through shared memory (order-preserving integer encoding, atomicMax);
-//   - the bound is bootstrapped from the first batch with a warp-level top-2 of the batch
-//     maxima, so that no thread pays the exact path for its first batch.
+//   - the bound is bootstrapped from the first batch: each warp publishes the top-2 of its
+//     lanes' batch maxima, so that no thread pays the exact path for its whole first batch;
+//     the first batch's loads are issued before the block's set-up barrier.
 //
 // Why skipping is exact: threads visit their elements in increasing token id, so an element
 // equal to the thread's runner-up loses the id tie-break; and an element below a value that
@@ -34,8 +35,8 @@ namespace mars {
 constexpr int kThreads = 256;  // threads per block
 constexpr int kU = 8;          // 16-byte vectors per thread per batch (128 B in flight each)
 static_assert(kU >= 4 && (kU & (kU - 1)) == 0, "kU must be a power of two >= 4");
-constexpr int kTargetBlocks = 148 * 8;     // split rows until the grid has about this many blocks
-constexpr int kMinSliceBytes = 8 * 1024;   // ... but never below this many bytes per slice
+constexpr int kTargetBlocks = 148 * 4;      // resident blocks of this kernel on a B200
+constexpr int kMinSliceBytes = kThreads * kU * 16;   // a slice is at least one full batch
 
 struct Params {
     const void *logits;
@@ -215,20 +216,23 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
     const int ntail = max(hi - tlo, 0);
     const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
 
+    constexpr int kBatchVecs = kThreads * kU;
+    const int nfull = nvec / kBatchVecs;
+    uint4 v[kU];
+    typename E::packed_t q[kU];
+
+    // ---- batch 0: issue its loads first, so that the set-up below overlaps their latency ----
+    float bm = (nfull > 0) ? load_batch<DT, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, true>(vbase, tid, nvec, v, q);
     if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
     __syncthreads();
 
     Rec s = empty_rec();
     if (tid < nhead) insert<false>(s, E::scalar(rowp, lo + tid), lo + tid, sT);
 
-    constexpr int kBatchVecs = kThreads * kU;
-    const int nfull = nvec / kBatchVecs;
-    uint4 v[kU];
-    typename E::packed_t q[kU];
-
-    // ---- batch 0: bootstrap the shared bound from the batch maxima, then process ----
-    float bm = (nfull > 0) ? load_batch<DT, false>(vbase, tid, nvec, v, q)
-                           : load_batch<DT, true>(vbase, tid, nvec, v, q);
+    // Bootstrap the shared bound from the batch maxima: every warp publishes the top-2 of its
+    // lanes' maxima (distinct elements) and goes on without waiting for the other warps; it
+    // sees at least its own contribution.
     {
         float a1 = (bm == bm) ? bm : -INFINITY, a2 = -INFINITY;
 #pragma unroll
@@ -238,8 +242,8 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
             a1 = fmaxf(a1, b1);
         }
         if ((tid & 31) == 0) { publish(sT, a1); publish(sT, a2); }
+        __syncwarp();
     }
-    __syncthreads();
     float T2 = dec(*(volatile unsigned *)&sT[1]);
     process_batch<DT, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
 
@@ -316,7 +320,7 @@ static Split choose_split(long long R, int V, int dt)
     const char *force = getenv("MARS_FORCE_SPLIT");  // test hook: force slices per row
     int min_elems = kMinSliceBytes / es;
     if (force && atoi(force) >= 1) { S = atoi(force); min_elems = 64; }
-    else if (R < kTargetBlocks) S = (kTargetBlocks + R - 1) / R;
+    else if (R < kTargetBlocks) S = kTargetBlocks / R;   // never more blocks than fit at once
     long long smax = V / min_elems;
     if (smax < 1) smax = 1;
     if (S > smax) S = smax;
@@ -351,7 +355,7 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     if (ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
     if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
     if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
-    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT)) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_COUNTERS_ZERO)) return MARS_ERR_UNSUPPORTED;
     if (!sizes_supported(B, N, V, (int)dt)) return MARS_ERR_UNSUPPORTED;
     const int es = dt == MARS_BF16 ? 2 : 4;
     if ((uintptr_t)logits % es) return MARS_ERR_INVALID_ARG;
@@ -374,7 +378,11 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     p.tail.N = N; p.tail.Dcap = Dcap; p.tail.theta = theta; p.tail.flags = flags; p.tail.chain = chain;
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemsetAsync(p.counters, 0, (size_t)B * sizeof(unsigned), st) != cudaSuccess) return MARS_ERR_CUDA;
+    // Arrival counters start at zero.  Every sequence's last block puts its counter back to
+    // zero, so a caller that knows the counters are clean may skip the memset node.
+    if (!(flags & MARS_COUNTERS_ZERO) &&
+        cudaMemsetAsync(p.counters, 0, (size_t)B * sizeof(unsigned), st) != cudaSuccess)
+        return MARS_ERR_CUDA;
     const unsigned grid = (unsigned)(R * sp.S);
     // dynamic shared memory: the tail's arrays, then (if it fits in 48 KB) room for N*S records
     const size_t tail_bytes = (tail_smem_bytes(N) + 15) / 16 * 16;

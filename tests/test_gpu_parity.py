@@ -287,3 +287,23 @@ def test_workspace_reuse_and_non_default_stream():
     st.synchronize()
     for o in outs:
         assert_same(mars.to_host(o), ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "reuse")
+
+
+def test_counters_zero_flag_skips_the_memset_safely():
+    """With MARS_COUNTERS_ZERO the library does not clear the arrival counters itself; they
+    are zero after a memset of the workspace and after every completed call."""
+    big = synth.cfg2(DEV, seed=31, B=12)
+    small = synth.tree_workload("z", 5, 9, 3, 3, 40000, torch.float32, DEV, 32, 0.9, 3.0, 15.0, 30.0, 0.5)
+    need = max(mars.workspace_bytes(big.B, big.N, big.V, mars.BF16),
+               mars.workspace_bytes(small.B, small.N, small.V, mars.FP32))
+    ws = torch.zeros(need, dtype=torch.uint8, device=DEV)
+    ref_big = orc.verify_chain(synth.to_numpy_bits(big.logits), big.draft, 0.9)
+    ref_small = orc.verify_tree(synth.to_numpy_bits(small.logits), small.tok, small.parent, 0.9)
+    for _ in range(3):      # alternate shapes (split and unsplit rows) on the same workspace
+        out = mars.to_host(mars.verify_chain(big.logits, big.draft, 0.9, flags=mars.COUNTERS_ZERO,
+                                             debug=True, workspace=ws))
+        assert_same(out, ref_big, ("accept_len", "out_tokens", "out_len", "top2_id"), "flag chain")
+        out = mars.to_host(mars.verify_tree(small.logits, small.tok, small.parent, 0.9,
+                                            flags=mars.COUNTERS_ZERO, debug=True, workspace=ws))
+        assert_same(out, ref_small, KEYS_TREE, "flag tree")
+    assert int(ws[:256].to(torch.int32).sum()) == 0              # counters are back at zero
