@@ -134,3 +134,40 @@ def test_cfg4_full_size_sampled():
     assert mism < 0.02, mism
     assert ((out["accept_len"] >= 0) & (out["accept_len"] <= w.max_depth)).all()
     assert out["accept_len"].mean() > 0.5
+
+
+def test_flags_statuses_and_host_errors():
+    """Same tail as the stored-logits path: shared parents, padding, malformed trees, depth
+    cap, the literal-sign flag; and the host-side argument checks of the fused entry point."""
+    w, _, tok, z = make_case(6, 20, 3000, 128, seed=77, depth=5)
+    par, tk = w.parent.copy(), tok.copy()
+    par[1, 7] = -1          # absent node
+    tk[2, 3] = -4           # padding token
+    par[3, 0] = 0           # malformed
+    par[4, 5] = 5           # malformed
+    th = float(np.float32(0.9))
+    for flags, dcap in ((0, None), (mars.SIGN_LITERAL, None), (0, 1)):
+        out = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, None, tk, par, 0.9, flags=flags,
+                                              Dcap=dcap, debug=True))
+        ref = orc.verify_tree(z, tk, par, th, flags, dcap)
+        ref["logits"] = z
+        compare(out, ref, tk, par, 0.9)
+        assert out["seq_status"].tolist() == ref["seq_status"].tolist()
+        assert np.array_equal(out["node_flags"][3:5], ref["node_flags"][3:5])
+    assert out["seq_status"][3] == 1 and out["seq_status"][4] == 1
+    out = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, None, tok, w.parent[0], 0.9, debug=True))
+    ref = orc.verify_tree(z, tok, w.parent[0], th)
+    ref["logits"] = z
+    compare(out, ref, tok, np.tile(w.parent[0], (w.B, 1)), 0.9)
+    # host errors: nothing is launched
+    o = mars.alloc_outputs(w.B, w.N, w.N - 1, DEV)
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.lmhead_verify(w.hidden, w.w_vocab, None, tok, w.parent, float("nan"), out=o)
+    with pytest.raises(mars.MarsError, match="unsupported sizes"):      # d not a multiple of 64
+        mars.lmhead_verify(w.hidden[:, :96].contiguous(), w.w_vocab[:, :96].contiguous(), None, tok,
+                           w.parent, 0.9, out=o)
+    with pytest.raises(mars.MarsError, match="workspace"):
+        mars.lmhead_verify(w.hidden, w.w_vocab, None, tok, w.parent, 0.9, out=o,
+                           workspace=torch.empty(512, dtype=torch.uint8, device=DEV))
+    torch.cuda.synchronize()
+    assert (o["accept_len"].cpu().numpy() == -777).all()
