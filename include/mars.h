@@ -171,6 +171,41 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Vocabulary-parallel verification, step 1 of 2: top-2 of one vocabulary shard.
+ * When the logits are sharded over the vocabulary (a tensor-parallel LM head), each rank
+ * holds columns [id_offset, id_offset + V_local) of every row.  This call reduces the local
+ * shard to one 16-byte record {float z1; int32 id1; float z2; int32 id2} per row, with
+ * GLOBAL token ids (local id + id_offset), using the same streaming top-2 (Sec. 3.3 of the
+ * paper: top-2 tokens of a logits row) and the same total order as mars_verify_tree.  A
+ * record is "unfinished": a shard with fewer than two entries above -inf leaves
+ * id = 0x7fffffff in the unused slots; mars_verify_records completes rows after merging.
+ *
+ *   logits   [B*N, ld] local shard, `dt`; V_local >= 2 columns are read per row.
+ *   records  out, [B*N] records, 16-byte aligned device memory.
+ *   flags    0 or MARS_COUNTERS_ZERO.
+ *   workspace as mars_workspace_bytes(B, N, V_local, dt).
+ */
+mars_status_t mars_top2_shard(const void *logits, int64_t ld, mars_dtype_t dt, int B, int N,
+                              int V_local, int32_t id_offset, void *records, uint32_t flags,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Vocabulary-parallel verification, step 2 of 2: merge the G shard records of every row and
+ * verify (three-way rule of Sec. 3.4, tree resolution as mars_verify_tree).  The merge is
+ * associative and commutative under the total order, so outputs are bit-identical to
+ * mars_verify_tree on the unsharded logits.  Between the two steps the ranks exchange their
+ * record arrays (one all-gather of 16 bytes x B*N per rank) into LOCAL memory.
+ *
+ *   records  [G, B*N] records: shard g's array at records + g*B*N; any shard order.
+ *   Other arguments, outputs and statuses as mars_verify_tree (no workspace needed).
+ */
+mars_status_t mars_verify_records(const void *records, int G, const int32_t *tok,
+                                  const int32_t *parent, int B, int N, float theta, uint32_t flags,
+                                  int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
+                                  int32_t *out_len, int Dcap, int32_t *seq_status,
+                                  const mars_debug_out_t *dbg, void *cuda_stream);
+
+/*
  * mars_verify_tree for callers that must not allocate device memory.  (The paper has no
  * counterpart; this is a deployment convenience of the library.)
  *

@@ -47,6 +47,8 @@ struct Params {
     int L;   // elements per slice (multiple of 16)
     Rec *partial;        // [R*S]
     unsigned *counters;  // [B]
+    Rec *shard_out;      // non-null: emit merged per-row records [B*N] instead of verifying
+    int id_offset;       // ... with this offset added to the token ids (vocabulary shard)
     int stage_partials;  // last block copies the sequence's N*S records to shared memory first
     int tail_smem_off;   // byte offset of that staging area in dynamic shared memory
     TailArgs tail;
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
         src = s_part;
     }
     const bool staged = p.stage_partials != 0;
-    verify_tail(p.tail, b, tail_smem, [&](int i) {
+    auto merged_row = [&](int i) {
         Rec acc = empty_rec();
         for (int k = 0; k < S; ++k) {
             const int4 *q = reinterpret_cast<const int4 *>(src + (size_t)i * S + k);
@@ -304,8 +306,19 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
             r.z1 = __int_as_float(w.x); r.id1 = w.y; r.z2 = __int_as_float(w.z); r.id2 = w.w;
             acc = merge(acc, r);
         }
-        return finish_record(acc);
-    });
+        return acc;
+    };
+    if (p.shard_out) {
+        // vocabulary shard: hand the rows' records (global token ids, still unfinished) on
+        for (int i = tid; i < p.N; i += kThreads) {
+            Rec r = merged_row(i);
+            if (r.id1 != kNoId) r.id1 += p.id_offset;
+            if (r.id2 != kNoId) r.id2 += p.id_offset;
+            p.shard_out[(size_t)b * p.N + i] = r;
+        }
+    } else {
+        verify_tail(p.tail, b, tail_smem, [&](int i) { return finish_record(merged_row(i)); });
+    }
     if (tid == 0) p.counters[b] = 0;
 }
 
@@ -349,12 +362,15 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
                          uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
                          int32_t *path_nodes, int32_t *out_len, int Dcap, int32_t *seq_status,
                          const mars_debug_out_t *dbg, void *workspace, size_t workspace_bytes,
-                         void *cuda_stream)
+                         void *cuda_stream, Rec *shard_out = nullptr, int id_offset = 0)
 {
-    if (B < 1 || N < 1 || V < 2 || !logits || !accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
+    if (B < 1 || N < 1 || V < 2 || !logits) return MARS_ERR_INVALID_ARG;
     if (ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
-    if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
-    if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
+    if (!shard_out) {
+        if (!accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
+        if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
+        if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
+    }
     if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_COUNTERS_ZERO)) return MARS_ERR_UNSUPPORTED;
     if (!sizes_supported(B, N, V, (int)dt)) return MARS_ERR_UNSUPPORTED;
     const int es = dt == MARS_BF16 ? 2 : 4;
@@ -369,6 +385,7 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     p.logits = logits; p.ld = ld; p.V = V; p.N = N; p.S = sp.S; p.L = sp.L;
     p.counters = (unsigned *)workspace;
     p.partial = (Rec *)((char *)workspace + counters_bytes(B));
+    p.shard_out = shard_out; p.id_offset = id_offset;
     p.tail.tok = tok; p.tail.parent = parent;
     p.tail.accept_len = accept_len; p.tail.out_tokens = out_tokens; p.tail.path_nodes = path_nodes;
     p.tail.out_len = out_len; p.tail.seq_status = seq_status;
@@ -480,6 +497,17 @@ mars_status_t mars_verify_tree_static(const void *logits, int64_t ld, mars_dtype
     return mars::run(logits, ld, dt, tok, parent, 0, B, N, V, theta, flags, accept_len, out_tokens,
                      path_nodes, out_len, Dcap, seq_status, dbg, scratch, MARS_STATIC_SCRATCH_BYTES,
                      cuda_stream);
+}
+
+mars_status_t mars_top2_shard(const void *logits, int64_t ld, mars_dtype_t dt, int B, int N, int V_local,
+                              int32_t id_offset, void *records, uint32_t flags, void *workspace,
+                              size_t workspace_bytes, void *cuda_stream)
+{
+    if (!records || ((uintptr_t)records & 15) || id_offset < 0) return MARS_ERR_INVALID_ARG;
+    if (flags & ~MARS_COUNTERS_ZERO) return MARS_ERR_UNSUPPORTED;
+    return mars::run(logits, ld, dt, nullptr, nullptr, 0, B, N, V_local, 0.0f, flags, nullptr, nullptr,
+                     nullptr, nullptr, 0, nullptr, nullptr, workspace, workspace_bytes, cuda_stream,
+                     (mars::Rec *)records, id_offset);
 }
 
 const char *mars_status_string(mars_status_t s)

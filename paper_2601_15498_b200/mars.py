@@ -61,6 +61,11 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_tree_static.restype = i32
             L.mars_static_scratch_bytes.argtypes = []
             L.mars_static_scratch_bytes.restype = sz
+            L.mars_top2_shard.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, u32, vp, sz, vp]
+            L.mars_top2_shard.restype = i32
+            L.mars_verify_records.argtypes = [vp, i32, vp, vp, i32, i32, f32, u32, vp, vp, vp, vp, i32,
+                                              vp, ctypes.POINTER(_DebugOut), vp]
+            L.mars_verify_records.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -245,6 +250,54 @@ def lmhead_verify(hidden: torch.Tensor, w_vocab: torch.Tensor, bias, tok, parent
             workspace.numel(), _stream())
     _check(code, "mars_lmhead_verify")
     out["_keepalive"] = (tok, parent, workspace, bias)
+    return out
+
+
+def top2_shard(logits_local: torch.Tensor, B: int, N: int, id_offset: int, V_local: int | None = None,
+               flags: int = 0, workspace: torch.Tensor | None = None,
+               records: torch.Tensor | None = None) -> torch.Tensor:
+    """mars_top2_shard on the current stream: per-row records of one vocabulary shard as an
+    int32 [B*N, 4] tensor (z1 bits, global id1, z2 bits, global id2)."""
+    dev = logits_local.device
+    dt, ld, V_local = _logits_args(logits_local, B * N, V_local)
+    workspace, wbytes = _workspace(B, N, V_local, dt, dev, workspace)
+    if records is None:
+        records = torch.empty((B * N, 4), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_top2_shard(logits_local.data_ptr(), ld, dt, B, N, V_local, int(id_offset),
+                                     records.data_ptr(), flags, workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_top2_shard")
+    return records
+
+
+def verify_records(records: torch.Tensor, tok, parent, theta: float, flags: int = 0,
+                   Dcap: int | None = None, debug: bool = False, out: dict | None = None) -> dict:
+    """mars_verify_records on the current stream: records int32 [G, B*N, 4]."""
+    dev = records.device
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    if not (records.is_cuda and records.dtype == torch.int32 and records.is_contiguous()
+            and records.dim() == 3 and records.shape[1:] == (B * N, 4)):
+        raise MarsError("records must be a contiguous int32 [G, B*N, 4] device tensor")
+    G = records.shape[0]
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    if out is None:
+        out = alloc_outputs(B, N, Dcap, dev, debug)
+    dbg = None
+    if "top2_val" in out:
+        dbg = _DebugOut(out["top2_val"].data_ptr(), out["top2_id"].data_ptr(),
+                        out["node_flags"].data_ptr())
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_records(
+            records.data_ptr(), G, tok.data_ptr(), parent.data_ptr(), B, N, float(theta), flags,
+            out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(), out["path_nodes"].data_ptr(),
+            out["out_len"].data_ptr(), Dcap, out["seq_status"].data_ptr(),
+            ctypes.byref(dbg) if dbg is not None else None, _stream())
+    _check(code, "mars_verify_records")
+    out["_keepalive"] = (tok, parent, records)
     return out
 
 
