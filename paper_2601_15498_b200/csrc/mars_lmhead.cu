@@ -6,17 +6,20 @@
 // vocabulary tiles it sees; 16-byte records go to the workspace and a small second kernel
 // merges them per row and runs the verification tail.
 //
-// Kernel 1 (persistent, one block per SM, 192 threads, warp-specialised):
+// Kernel 1 comes in two forms with the same pipeline (192 threads, warp-specialised):
+//   lmhead_top2_kernel_pair  (default) clusters of two blocks sharing tcgen05.mma.cta_group::2,
+//                            M = 256 per pair; see the comment above that kernel.
+//   lmhead_top2_kernel       one block per SM, cta_group::1, M = 128 (test hook / fallback).
 //   warp 0      TMA producer: H tile [128 x 64] and W tile [256 x 64] (128-byte swizzle) per
-//               k-block into a 4-stage shared-memory ring, completion on mbarriers.
-//   warp 1      allocates the 512 TMEM columns and issues tcgen05.mma (M=128, N=256, K=16,
-//               kind::f16 with bf16 operands, fp32 accumulate); tcgen05.commit releases the
-//               ring stage / publishes the accumulator.
+//               k-block into a shared-memory ring, completion on mbarriers.
+//   warp 1      allocates the 512 TMEM columns and issues tcgen05.mma (N=256, K=16, kind::f16
+//               with bf16 operands, fp32 accumulate); tcgen05.commit releases the ring stage /
+//               publishes the accumulator.
 //   warps 2..5  epilogue: tcgen05.ld of the finished accumulator (double-buffered, so the next
 //               tile's MMAs overlap), bias, per-row running top-2.
-// Work item = (vocabulary chunk of kChunkTiles N-tiles, M-tile); items are dealt round-robin
-// with the M-tile index fastest, so the blocks that run together share W tiles through L2 and
-// W crosses HBM about once.
+// Work item = (vocabulary chunk of a few N-tiles, M-tile or pair of M-tiles); items are dealt
+// round-robin with the M index fastest, so the blocks that run together share W tiles through
+// L2 and W crosses HBM about once.
 //
 // Every wait on an mbarrier is bounded (clock64 budget).  A wait that gives up raises a
 // block-wide abort flag and a status word in the workspace; all roles then fall through to
@@ -38,7 +41,7 @@ constexpr int kBN = 256;          // vocabulary entries per tile = TMEM columns 
 constexpr int kBK = 64;           // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
 constexpr int kStages = 4;
-constexpr int kChunkTiles = 6;    // N-tiles per work item
+constexpr int kMaxChunkTiles = 16; // upper bound on N-tiles per work item
 constexpr int kLmThreads = 192;
 constexpr uint32_t kABytes = kBM * kBK * 2;   // 16 KB
 constexpr uint32_t kBBytes = kBN * kBK * 2;   // 32 KB
@@ -50,6 +53,7 @@ constexpr size_t kLmSmemBytes = (size_t)kStages * kStageBytes + 1024 /*align*/ +
 struct LmParams {
     int M, V, d;
     int n_mtiles, n_ntiles, n_chunks, n_items;
+    int chunk_tiles;     // N-tiles per work item
     const float *bias;   // [V] or null
     Rec *partial;        // [M, n_chunks]
     unsigned *status;    // workspace word: 0 ok, else MARS_SEQ_TIMEOUT
@@ -210,8 +214,8 @@ lmhead_top2_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
             bool ok = true;
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const int mt = item % p.n_mtiles, chunk = item / p.n_mtiles;
-                const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
-                for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+                const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
+                for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
                     for (int kb = 0; kb < kblocks; ++kb) {
                         if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                         const uint32_t fb = full0 + 8 * stage;
@@ -241,8 +245,8 @@ lmhead_top2_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
             bool ok = true;
             for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
                 const int chunk = item / p.n_mtiles;
-                const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
-                for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+                const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
+                for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
                     if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * kBN;
@@ -276,10 +280,10 @@ lmhead_top2_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
         bool ok = true;
         for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
             const int mt = item % p.n_mtiles, chunk = item / p.n_mtiles;
-            const int nt_end = min((chunk + 1) * kChunkTiles, p.n_ntiles);
+            const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
             const int row = mt * kBM + row_in_tile;
             Rec rec = empty_rec();
-            for (int nt = chunk * kChunkTiles; nt < nt_end && ok; ++nt) {
+            for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
                 // warp-uniform outcome: the TMEM loads below are warp-collective
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, p.status));
                 if (!ok) break;
@@ -322,6 +326,240 @@ lmhead_top2_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_const
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+
+// ----------------------------------------------------------------------------- 2-CTA variant
+//
+// Same pipeline with tcgen05 `cta_group::2`: two thread blocks of a cluster (two SMs) share one
+// MMA of M = 256 x N = 256.  Block r of the pair owns M-tile 2*pair + r: it loads its own
+// 128 x 64 slice of H and HALF of the W tile (128 of the 256 vocabulary rows) per k-block, the
+// leader block (rank 0) issues the MMAs, which read both blocks' shared memory and write each
+// block's 128 accumulator rows into that block's TMEM.  Per block and k-block 32 KB instead of
+// 48 KB come out of L2, and the ring has 6 stages instead of 4.
+//
+// Barriers (all in each block's own shared memory at identical offsets):
+//   full[s]    leader's copy only is used: armed by the leader's producer with the bytes of
+//              BOTH blocks; both producers' TMA loads complete on it.
+//   empty[s]   each block's own copy, released for both blocks by one multicast tcgen05.commit.
+//   tfull[a]   each block's own copy, published for both by one multicast tcgen05.commit.
+//   tempty[a]  leader's copy: 8 arrivals (4 epilogue warps of each block; the peer's warps
+//              arrive remotely).
+
+constexpr int kStages2 = 6;
+constexpr uint32_t kB2Bytes = (kBN / 2) * kBK * 2;          // 16 KB: this block's half of the W tile
+constexpr uint32_t kStage2Bytes = kABytes + kB2Bytes;        // 32 KB
+constexpr size_t kLm2SmemBytes = (size_t)kStages2 * kStage2Bytes + 1024 + 256;
+constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
+                             ((uint32_t)((2 * kBM) >> 4) << 24);
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t leader_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(leader_bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)   // same offset in both blocks
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((unsigned short)3)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair_local(uint32_t bar)   // this block's barrier only
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kLmThreads, 1)
+lmhead_top2_kernel_pair(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+                        const LmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t bars = tiles + kStages2 * kStage2Bytes;
+    const uint32_t full0 = bars, empty0 = bars + 8 * kStages2;
+    const uint32_t tfull0 = bars + 16 * kStages2, tempty0 = tfull0 + 16, drain = tempty0 + 16;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = leader
+    const int pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    const int kblocks = p.d / kBK;
+    const int n_mpairs = (p.n_mtiles + 1) / 2;
+    const int n_items = n_mpairs * p.n_chunks;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages2; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 8); }
+        mbar_init(drain, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    cluster_sync_all();            // both blocks' barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int *abort_flag = &s_abort;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both blocks)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int item = pair_id; item < n_items && ok; item += n_pairs) {
+                const int mt = 2 * (item % n_mpairs) + (int)rank, chunk = item / n_mpairs;
+                const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
+                for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                        const uint32_t leader_full = mapa_shared(full0 + 8 * stage, 0);
+                        if (rank == 0) mbar_expect_tx_cluster(leader_full, 2 * kStage2Bytes);
+                        const uint32_t a_dst = tiles + stage * kStage2Bytes;
+                        tma_load_2d_pair(a_dst, &map_h, kb * kBK, mt * kBM, leader_full);
+                        tma_load_2d_pair(a_dst + kABytes, &map_w, kb * kBK, nt * kBN + (int)rank * (kBN / 2),
+                                         leader_full);
+                        if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (*abort_flag) {     // let copies already issued by this block land (bounded)
+                const long long t0 = clock64();
+                while (clock64() - t0 < 20000000ll) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int item = pair_id; item < n_items && ok; item += n_pairs) {
+                const int chunk = item / n_mpairs;
+                const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
+                for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
+                    if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * kBN;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (!mbar_wait(full0 + 8 * stage, phase, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = tiles + stage * kStage2Bytes;
+                        const uint64_t adesc = umma_desc_k_sw128(a_addr);
+                        const uint64_t bdesc = umma_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBK / kUmmaK; ++k)
+                            tc_mma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc2, (kb | k) != 0 ? 1u : 0u);
+                        tc_commit_pair(empty0 + 8 * stage);      // frees the stage in both blocks
+                        if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit_pair(tfull0 + 8 * acc);            // accumulator complete in both blocks
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                }
+            }
+            tc_commit_pair_local(drain);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (both blocks)
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int item = pair_id; item < n_items && ok; item += n_pairs) {
+            const int mt = 2 * (item % n_mpairs) + (int)rank, chunk = item / n_mpairs;
+            const int nt_end = min((chunk + 1) * p.chunk_tiles, p.n_ntiles);
+            const int row = mt * kBM + row_in_tile;
+            Rec rec = empty_rec();
+            for (int nt = chunk * p.chunk_tiles; nt < nt_end && ok; ++nt) {
+                ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
+#pragma unroll 1
+                for (int c = 0; c < kBN / 32; ++c) {
+                    float v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    const int col0 = nt * kBN + c * 32;
+                    if (p.bias) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += (col0 + j < p.V) ? __ldg(p.bias + col0 + j) : 0.0f;
+                    }
+                    float m = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) m = fmaxf(m, v[j]);
+                    if (m > rec.z2) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float x = v[j];
+                            if (x > rec.z2 && col0 + j < p.V) {
+                                if (x > rec.z1) { rec.z2 = rec.z1; rec.id2 = rec.id1; rec.z1 = x; rec.id1 = col0 + j; }
+                                else { rec.z2 = x; rec.id2 = col0 + j; }
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(mapa_shared(tempty0 + 8 * acc, 0));   // leader's barrier
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (ok && row < p.M) p.partial[(size_t)row * p.n_chunks + chunk] = rec;
+        }
+    }
+
+    // The leader's MMAs write both blocks' TMEM: wait for them to retire, then meet the peer.
+    if (warp == 1 && lane == 0 && rank == 0) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(drain, 0) && clock64() - t0 < kWaitCycles) {}
+    }
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -388,15 +626,35 @@ static bool make_map(CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct LmShape { int n_mtiles, n_ntiles, n_chunks, n_items; };
+struct LmShape { int n_mtiles, n_ntiles, n_chunks, n_items, chunk_tiles; };
+
+// Work items are (vocabulary chunk, M-tile) pairs dealt round-robin to `blocks` persistent
+// blocks.  The chunk length is the one that wastes the least of the last round: cost =
+// rounds x tiles per item; ties go to the longer chunk (fewer records per row to merge).  Host-only and independent of the
+// device so that the workspace size is a pure function of the shapes.
+static bool lm_pair_mode()
+{
+    const char *e = getenv("MARS_LMHEAD_1CTA");    // test hook: force the single-block MMA kernel
+    return !(e && e[0] == '1');
+}
 
 static LmShape lm_shape(long long M, int V)
 {
+    const bool pair = lm_pair_mode();
     LmShape s;
     s.n_mtiles = (int)((M + kBM - 1) / kBM);
     s.n_ntiles = (V + kBN - 1) / kBN;
-    s.n_chunks = (s.n_ntiles + kChunkTiles - 1) / kChunkTiles;
-    s.n_items = s.n_mtiles * s.n_chunks;
+    const int blocks = pair ? 74 : 148;                          // schedulable units on a B200
+    const int m_units = pair ? (s.n_mtiles + 1) / 2 : s.n_mtiles;
+    long long best_cost = -1;
+    s.chunk_tiles = 1;
+    for (int c = 1; c <= kMaxChunkTiles && c <= s.n_ntiles; ++c) {
+        const long long items = (long long)m_units * ((s.n_ntiles + c - 1) / c);
+        const long long cost = ((items + blocks - 1) / blocks) * c;
+        if (best_cost < 0 || cost <= best_cost) { best_cost = cost; s.chunk_tiles = c; }
+    }
+    s.n_chunks = (s.n_ntiles + s.chunk_tiles - 1) / s.chunk_tiles;
+    s.n_items = m_units * s.n_chunks;
     return s;
 }
 
@@ -439,13 +697,14 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     LmParams p;
     p.M = (int)M; p.V = V; p.d = d;
     p.n_mtiles = s.n_mtiles; p.n_ntiles = s.n_ntiles; p.n_chunks = s.n_chunks; p.n_items = s.n_items;
+    p.chunk_tiles = s.chunk_tiles;
     p.bias = bias;
     p.status = (unsigned *)workspace;
     p.partial = (Rec *)((char *)workspace + 256);
 
     CUtensorMap map_h, map_w;
     if (!make_map(&map_h, hidden, (uint64_t)M, (uint64_t)d, kBM)) return MARS_ERR_CUDA;
-    if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, kBN)) return MARS_ERR_CUDA;
+    if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, lm_pair_mode() ? kBN / 2 : kBN)) return MARS_ERR_CUDA;
 
     TailArgs t;
     t.tok = tok; t.parent = parent; t.accept_len = accept_len; t.out_tokens = out_tokens;
@@ -463,13 +722,40 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     std::call_once(attr_once, [] {
         attr_err = cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)kLmSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(lmhead_top2_kernel_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kLm2SmemBytes);
     });
     if (attr_err != cudaSuccess) return MARS_ERR_CUDA;
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (cudaMemsetAsync(p.status, 0, 256, st) != cudaSuccess) return MARS_ERR_CUDA;
-    const int grid = s.n_items < sms ? s.n_items : sms;
-    lmhead_top2_kernel<<<grid, kLmThreads, kLmSmemBytes, st>>>(map_h, map_w, p);
+    if (lm_pair_mode()) {
+        // persistent pairs: never launch more clusters than can be resident together
+        static std::once_flag occ_once;
+        static int max_pairs = 0;
+        std::call_once(occ_once, [&] {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(sms / 2 * 2); cfg.blockDim = dim3(kLmThreads);
+            cfg.dynamicSmemBytes = kLm2SmemBytes;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, lmhead_top2_kernel_pair, &cfg) == cudaSuccess && n > 0)
+                max_pairs = n;
+            else
+                max_pairs = sms / 2;
+            (void)cudaGetLastError();
+        });
+        int pairs = max_pairs < sms / 2 ? max_pairs : sms / 2;
+        if (s.n_items < pairs) pairs = s.n_items;
+        lmhead_top2_kernel_pair<<<2 * pairs, kLmThreads, kLm2SmemBytes, st>>>(map_h, map_w, p);
+    } else {
+        const int grid = s.n_items < sms ? s.n_items : sms;
+        lmhead_top2_kernel<<<grid, kLmThreads, kLmSmemBytes, st>>>(map_h, map_w, p);
+    }
     if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
     lmhead_tail_kernel<<<B, 128, tail_smem_bytes(N), st>>>(p, t);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
