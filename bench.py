@@ -348,7 +348,7 @@ def lmhead_arm(args, rank: int, world: int, local: int):
         "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 2 * steps,
         "roofline": {"bound": "tensor", "achieved": tfs, "peak": peak, "unit": "TFLOP/s",
                      "frac": tfs / peak, "traffic": None, "peak_source": src,
-                     "kernel": "mars::lmhead_top2_kernel", "algorithmic_flops_per_launch": flops},
+                     "kernel": "mars::lmhead_top2_kernel_pair", "algorithmic_flops_per_launch": flops},
         "cpu_baseline": cpu}), flush=True)
     if world > 1:
         import torch.distributed as dist

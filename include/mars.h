@@ -171,6 +171,17 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Self-test of the bounded device-side wait used by mars_lmhead_verify's pipeline (the paper
+ * has no counterpart).  Launches one block that waits, with the pipeline's own wait routine,
+ * on a barrier that nothing ever signals; the wait must give up after `budget_cycles` SM
+ * clock cycles (1 .. 2e9) and the kernel must return normally.  Never faults or hangs.
+ *   scratch32  32 bytes of device memory, 8-byte aligned; after the stream has passed:
+ *              uint32 [0] = MARS_SEQ_TIMEOUT (the status the pipeline would report),
+ *              int64 at byte 8 = cycles actually waited, int64 at byte 16 = 0 (wait failed).
+ */
+mars_status_t mars_selftest_bounded_wait(int64_t budget_cycles, void *scratch32, void *cuda_stream);
+
+/*
  * Vocabulary-parallel verification, step 1 of 2: top-2 of one vocabulary shard.
  * When the logits are sharded over the vocabulary (a tensor-parallel LM head), each rank
  * holds columns [id_offset, id_offset + V_local) of every row.  This call reduces the local

@@ -90,7 +90,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 
 // Bounded wait.  Returns false if the budget ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          unsigned *status)
+                                          unsigned *status, long long budget = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > budget) {
             *abort_flag = 1;
             atomicExch(status, (unsigned)MARS_SEQ_TIMEOUT);
             return false;
@@ -563,6 +563,29 @@ lmhead_top2_kernel_pair(const __grid_constant__ CUtensorMap map_h, const __grid_
     }
 }
 
+// ----------------------------------------------------------------------------- wait self-test
+//
+// One block waits, with the pipeline's own bounded-wait routine, on an mbarrier that nothing
+// ever arrives on.  The wait must give up after `budget` cycles, raise the status word and let
+// the kernel return normally.  Used by mars_selftest_bounded_wait.
+__global__ void bounded_wait_selftest_kernel(unsigned *status, long long budget, long long *cycles_waited)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long t0 = clock64();
+        const bool ok = mbar_wait(smem_u32(&bar), 0, &s_abort, status, budget);
+        cycles_waited[0] = clock64() - t0;
+        cycles_waited[1] = ok ? 1 : 0;
+    }
+}
+
 // ----------------------------------------------------------------------------- tail kernel
 
 __global__ void __launch_bounds__(128) lmhead_tail_kernel(const LmParams p, const TailArgs t)
@@ -675,6 +698,17 @@ size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d)
     if (!mars::lm_supported(B, N, V, d)) return 0;
     const mars::LmShape s = mars::lm_shape((long long)B * N, V);
     return 256 + (size_t)B * N * s.n_chunks * sizeof(mars::Rec);
+}
+
+mars_status_t mars_selftest_bounded_wait(int64_t budget_cycles, void *scratch32, void *cuda_stream)
+{
+    if (!scratch32 || ((uintptr_t)scratch32 & 7) || budget_cycles < 1 || budget_cycles > 2000000000ll)
+        return MARS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(scratch32, 0, 32, st) != cudaSuccess) return MARS_ERR_CUDA;
+    mars::bounded_wait_selftest_kernel<<<1, 32, 0, st>>>((unsigned *)scratch32, (long long)budget_cycles,
+                                                         (long long *)((char *)scratch32 + 8));
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
 mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const float *bias, int d,

@@ -66,6 +66,8 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_records.argtypes = [vp, i32, vp, vp, i32, i32, f32, u32, vp, vp, vp, vp, i32,
                                               vp, ctypes.POINTER(_DebugOut), vp]
             L.mars_verify_records.restype = i32
+            L.mars_selftest_bounded_wait.argtypes = [i64, vp, vp]
+            L.mars_selftest_bounded_wait.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L

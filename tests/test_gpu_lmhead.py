@@ -171,3 +171,20 @@ def test_flags_statuses_and_host_errors():
                            workspace=torch.empty(512, dtype=torch.uint8, device=DEV))
     torch.cuda.synchronize()
     assert (o["accept_len"].cpu().numpy() == -777).all()
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait on a barrier that nothing signals runs out after its budget, sets the status
+    word and lets the kernel return; the context stays usable."""
+    lib = mars.lib()
+    scratch = torch.full((4,), -1, dtype=torch.int64, device=DEV)
+    budget = 2_000_000                                   # about a millisecond
+    code = lib.mars_selftest_bounded_wait(budget, scratch.data_ptr(), None)
+    assert code == 0
+    torch.cuda.synchronize()
+    h = scratch.cpu().numpy()
+    assert int(h[0]) & 0xFFFFFFFF == 3                   # MARS_SEQ_TIMEOUT
+    assert budget <= h[1] < 100 * budget and h[2] == 0
+    assert lib.mars_selftest_bounded_wait(0, scratch.data_ptr(), None) == 1
+    # the device still works
+    assert float(torch.ones(8, device=DEV).sum()) == 8.0
