@@ -307,3 +307,24 @@ def test_counters_zero_flag_skips_the_memset_safely():
                                             flags=mars.COUNTERS_ZERO, debug=True, workspace=ws))
         assert_same(out, ref_small, KEYS_TREE, "flag tree")
     assert int(ws[:256].to(torch.int32).sum()) == 0              # counters are back at zero
+
+
+def test_minimal_shapes_and_extreme_thetas():
+    """K = 1 chains (no drafts: only the bonus token), single-node trees, Dcap = 0, many short
+    sequences, and thresholds at the ends of the float range."""
+    g = torch.Generator(device="cpu"); g.manual_seed(3)
+    z = (torch.randn((40, 300), generator=g) * 3 + 5).to(DEV)
+    out, ref = run_chain(z, np.empty((40, 0), np.int32), 0.9)                 # K = 1
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "K=1")
+    assert (out["accept_len"] == 0).all() and (out["out_len"] == 1).all()
+    tok = np.full((40, 1), -1, np.int32)
+    par = np.full((40, 1), -1, np.int32)
+    out, ref = run_tree(z, tok, par, 0.9)                                     # N = 1
+    assert_same(out, ref, KEYS_TREE, "N=1")
+    w = synth.tree_workload("m", 2000, 4, 2, 2, 64, torch.bfloat16, DEV, 8, 0.9, 3.0, 15.0, 30.0, 0.5)
+    for theta in (0.9, float("inf"), float("-inf"), 3.0e38, -3.0e38, 0.0):
+        out, ref = run_tree(w.logits, w.tok, w.parent, theta)
+        assert_same(out, ref, KEYS_TREE, f"B=2000 theta={theta}")
+    out, ref = run_tree(w.logits, w.tok, w.parent, 0.5, Dcap=0)               # every accept overflows
+    assert_same(out, ref, KEYS_TREE, "Dcap=0")
+    assert set(out["seq_status"].tolist()) <= {0, 2} and 2 in out["seq_status"]
