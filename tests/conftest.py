@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """Compile libmars.so in-tree if it is missing or older than its sources (nvcc cross-compiles
+    without a GPU).  A failed build is reported by the tests that need the library."""
+    try:
+        from paper_2601_15498_b200 import build
+        build.build()
+    except Exception as e:  # pragma: no cover
+        print(f"libmars build skipped: {e}")
+    yield
