@@ -5,7 +5,7 @@
 // from HBM with 16-byte loads.  Each thread keeps an exact top-2 (values and token ids) in
 // registers, but touches it only for the few batches that can still change the answer:
 //
-//   - a batch of kU (8) 16-byte vectors per thread is first reduced to its maximum with packed
+//   - a batch of U (8, or 4 in the high-occupancy variant) 16-byte vectors per thread is first reduced to its maximum with packed
 //     bf16x2 (or fp32) max instructions -- about one instruction per two bf16 elements;
 //   - the batch is skipped unless its maximum beats the thread's own runner-up AND is not
 //     below T2, a lower bound on the slice's runner-up value that the whole block shares
@@ -34,7 +34,11 @@ namespace mars {
 
 constexpr int kThreads = 256;  // threads per block
 constexpr int kU = 8;          // 16-byte vectors per thread per batch (128 B in flight each)
-static_assert(kU >= 4 && (kU & (kU - 1)) == 0, "kU must be a power of two >= 4");
+// Large bf16 batches run a second instantiation with 4 vectors per batch and 8 resident blocks
+// per SM (32 registers): the same bytes in flight from twice the threads measured 1-1.5 %
+// faster there, and slower for fp32 and for batches of a few hundred rows.
+constexpr int kUDense = 4;
+constexpr int kDenseMinRows = 148 * 16;
 constexpr int kTargetBlocks = 148 * 4;      // resident blocks of this kernel on a B200
 constexpr int kMinSliceBytes = kThreads * kU * 16;   // a slice is at least one full batch
 
@@ -148,14 +152,14 @@ __device__ __forceinline__ void insert(Rec &s, float x, int idx, unsigned *sT)
     }
 }
 
-template <int DT, bool PUBLISH>
-__device__ __forceinline__ void process_batch(const uint4 (&v)[kU], const typename Elem<DT>::packed_t (&q)[kU],
+template <int DT, int U, bool PUBLISH>
+__device__ __forceinline__ void process_batch(const uint4 (&v)[U], const typename Elem<DT>::packed_t (&q)[U],
                                               float bm, float T2, int idx0, Rec &s, unsigned *sT)
 {
     typedef Elem<DT> E;
     if (bm > s.z2 && bm >= T2) {
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
+        for (int u = 0; u < U; ++u) {
             float qf = E::to_float(q[u]);
             if (qf > s.z2 && qf >= T2) {
                 int base = idx0 + u * kThreads * E::kVec;
@@ -166,31 +170,32 @@ __device__ __forceinline__ void process_batch(const uint4 (&v)[kU], const typena
     }
 }
 
-template <int DT, bool GUARD>
-__device__ __forceinline__ float load_batch(const uint4 *vbase, int v0, int nvec, uint4 (&v)[kU],
-                                            typename Elem<DT>::packed_t (&q)[kU])
+template <int DT, int U, bool GUARD>
+__device__ __forceinline__ float load_batch(const uint4 *vbase, int v0, int nvec, uint4 (&v)[U],
+                                            typename Elem<DT>::packed_t (&q)[U])
 {
     typedef Elem<DT> E;
+    static_assert(U >= 4 && (U & (U - 1)) == 0, "U must be a power of two >= 4");
 #pragma unroll
-    for (int u = 0; u < kU; ++u) {
+    for (int u = 0; u < U; ++u) {
         int vi = v0 + u * kThreads;
         if (!GUARD || vi < nvec) v[u] = ld_stream(vbase + vi);
         else v[u] = E::neg_inf();
     }
 #pragma unroll
-    for (int u = 0; u < kU; ++u) q[u] = E::vred(v[u]);
-    typename E::packed_t m[kU / 2];
+    for (int u = 0; u < U; ++u) q[u] = E::vred(v[u]);
+    typename E::packed_t m[U / 2];
 #pragma unroll
-    for (int u = 0; u < kU / 2; ++u) m[u] = E::pmax(q[2 * u], q[2 * u + 1]);
+    for (int u = 0; u < U / 2; ++u) m[u] = E::pmax(q[2 * u], q[2 * u + 1]);
 #pragma unroll
-    for (int w = kU / 4; w > 0; w >>= 1)
+    for (int w = U / 4; w > 0; w >>= 1)
 #pragma unroll
         for (int u = 0; u < w; ++u) m[u] = E::pmax(m[u], m[u + w]);
     return E::to_float(m[0]);
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
+template <int DT, int U, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
 {
     typedef Elem<DT> E;
     extern __shared__ __align__(16) unsigned char smem_dyn[];
@@ -218,14 +223,14 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
     const int ntail = max(hi - tlo, 0);
     const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
 
-    constexpr int kBatchVecs = kThreads * kU;
+    constexpr int kBatchVecs = kThreads * U;
     const int nfull = nvec / kBatchVecs;
-    uint4 v[kU];
-    typename E::packed_t q[kU];
+    uint4 v[U];
+    typename E::packed_t q[U];
 
     // ---- batch 0: issue its loads first, so that the set-up below overlaps their latency ----
-    float bm = (nfull > 0) ? load_batch<DT, false>(vbase, tid, nvec, v, q)
-                           : load_batch<DT, true>(vbase, tid, nvec, v, q);
+    float bm = (nfull > 0) ? load_batch<DT, U, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, U, true>(vbase, tid, nvec, v, q);
     if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
     __syncthreads();
 
@@ -247,18 +252,18 @@ __global__ void __launch_bounds__(kThreads) verify_kernel(const Params p)
         __syncwarp();
     }
     float T2 = dec(*(volatile unsigned *)&sT[1]);
-    process_batch<DT, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
+    process_batch<DT, U, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
 
     // ---- steady state ----
     for (int bi = 1; bi < nfull; ++bi) {
-        bm = load_batch<DT, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
+        bm = load_batch<DT, U, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
         T2 = dec(*(volatile unsigned *)&sT[1]);
-        process_batch<DT, true>(v, q, bm, T2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
+        process_batch<DT, U, true>(v, q, bm, T2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
     }
     if (nfull > 0 && nfull * kBatchVecs < nvec) {
-        bm = load_batch<DT, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        bm = load_batch<DT, U, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
         T2 = dec(*(volatile unsigned *)&sT[1]);
-        process_batch<DT, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
+        process_batch<DT, U, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
     }
     if (tid < ntail) insert<false>(s, E::scalar(rowp, tlo + tid), tlo + tid, sT);
 
@@ -407,8 +412,12 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     p.stage_partials = (sp.S > 1 && tail_bytes + stage_bytes <= 48 * 1024) ? 1 : 0;
     p.tail_smem_off = (int)tail_bytes;
     const size_t smem = tail_bytes + (p.stage_partials ? stage_bytes : 0);
-    if (dt == MARS_BF16) verify_kernel<MARS_BF16><<<grid, kThreads, smem, st>>>(p);
-    else verify_kernel<MARS_FP32><<<grid, kThreads, smem, st>>>(p);
+    if (dt == MARS_BF16 && sp.S == 1 && R >= kDenseMinRows)
+        verify_kernel<MARS_BF16, kUDense, 8><<<grid, kThreads, smem, st>>>(p);
+    else if (dt == MARS_BF16)
+        verify_kernel<MARS_BF16, kU, 4><<<grid, kThreads, smem, st>>>(p);
+    else
+        verify_kernel<MARS_FP32, kU, 4><<<grid, kThreads, smem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
