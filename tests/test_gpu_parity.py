@@ -328,3 +328,31 @@ def test_minimal_shapes_and_extreme_thetas():
     out, ref = run_tree(w.logits, w.tok, w.parent, 0.5, Dcap=0)               # every accept overflows
     assert_same(out, ref, KEYS_TREE, "Dcap=0")
     assert set(out["seq_status"].tolist()) <= {0, 2} and 2 in out["seq_status"]
+
+
+def test_cuda_graph_replay_with_changing_inputs():
+    """The calls only enqueue work (one optional memset, one kernel) and allocate nothing, so a
+    captured step can be replayed on new data written into the same buffers."""
+    ws_list = [synth.tree_workload("g", 4, 30, 5, 3, 50000, torch.bfloat16, DEV, 60 + i, 0.9, 3.0, 15.0,
+                                   30.0, 0.4) for i in range(3)]
+    w0 = ws_list[0]
+    logits = torch.empty_like(w0.logits)
+    tok = torch.zeros((w0.B, w0.N), dtype=torch.int32, device=DEV)
+    parent = torch.zeros((w0.B, w0.N), dtype=torch.int32, device=DEV)
+    work = torch.zeros(mars.workspace_bytes(w0.B, w0.N, w0.V, mars.BF16), dtype=torch.uint8, device=DEV)
+    out = mars.alloc_outputs(w0.B, w0.N, w0.N - 1, DEV, debug=True)
+    logits.copy_(w0.logits); tok.copy_(torch.as_tensor(w0.tok)); parent.copy_(torch.as_tensor(w0.parent))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        mars.verify_tree(logits, tok, parent, 0.9, workspace=work, out=out)     # warm-up outside capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        mars.verify_tree(logits, tok, parent, 0.9, workspace=work, out=out)
+    for w in ws_list[::-1]:
+        logits.copy_(w.logits); tok.copy_(torch.as_tensor(w.tok)); parent.copy_(torch.as_tensor(w.parent))
+        graph.replay()
+        got = mars.to_host(out)
+        ref = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, 0.9)
+        assert_same(got, ref, KEYS_TREE, "graph replay")
