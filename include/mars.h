@@ -56,6 +56,15 @@ typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
                                  these functions on it with at least B sequences; the library
                                  then skips its own clearing of those bytes (one stream op less) */
 
+/* Alternative indicators for the relaxation test (the paper's Sec. 3.3 discusses both as the
+ * alternatives to its logit ratio; the default, with neither bit set, is the paper's r > theta).
+ * With either bit the `theta` argument carries that indicator's threshold, the sign guard and
+ * MARS_SIGN_LITERAL do not apply, and everything else (exact match, stop at the first
+ * failure, tree resolution) is unchanged.  The two bits are mutually exclusive. */
+#define MARS_RULE_MARGIN 8u      /* relax iff Delta = z1 - z2 < theta (fixed logit margin, fp32) */
+#define MARS_RULE_PROB_RATIO 16u /* relax iff p2/p1 = exp(z2 - z1) > theta; evaluated as
+                                    z1 - z2 < (float)(-ln(theta)), theta <= 0 always relaxes  */
+
 #define MARS_MAX_NODES 1024   /* cap on N (rows per sequence)                                 */
 
 /* per-sequence status values written to seq_status */

@@ -48,6 +48,8 @@
 
 #define MARS_ORACLE_SIGN_LITERAL 1u
 #define MARS_ORACLE_SHARED_PARENT 2u
+#define MARS_ORACLE_RULE_MARGIN 8u
+#define MARS_ORACLE_RULE_PROB_RATIO 16u
 
 enum { ORACLE_BF16 = 0, ORACLE_FP32 = 1, ORACLE_FP64 = 2 };
 
@@ -118,15 +120,35 @@ static int beats_f64(double ax, int64_t aj, double bx, int64_t bj)
 DEFINE_TOP2(top2_row_f32, float, beats_f32, -INFINITY)
 DEFINE_TOP2(top2_row_f64, double, beats_f64, -INFINITY)
 
-/* Eq. 4 and the "Adaptive Relaxation" condition r > theta, one IEEE division. */
+/* Eq. 4 and the "Adaptive Relaxation" condition r > theta, one IEEE division.
+ * Variants (Sec. 3.3 names both as the alternatives to the logit ratio):
+ *   RULE_MARGIN      Delta = z(1) - z(2) < theta, the fixed-margin indicator (Delta as in Eq. 5);
+ *   RULE_PROB_RATIO  p2/p1 = exp(z(2) - z(1)) > theta, taken as Delta < (T)(-ln theta) with the
+ *                    logarithm in double; theta <= 0 always relaxes. */
 int mars_oracle_relax_f32(float z1, float z2, float theta, uint32_t flags)
 {
+    if (flags & MARS_ORACLE_RULE_PROB_RATIO) {
+        double t = (double)theta;
+        volatile float c = t > 0.0 ? (float)(-log(t)) : INFINITY;
+        volatile float d = z1 - z2;
+        return d < c;
+    }
+    if (flags & MARS_ORACLE_RULE_MARGIN) {
+        volatile float d = z1 - z2;
+        return d < theta;
+    }
     int guard = (flags & MARS_ORACLE_SIGN_LITERAL) ? 1 : (z1 > 0.0f);
     volatile float r = z2 / z1;
     return guard && (r > theta);
 }
 int mars_oracle_relax_f64(double z1, double z2, double theta, uint32_t flags)
 {
+    if (flags & MARS_ORACLE_RULE_PROB_RATIO) {
+        /* theta arrives as the fp32 threshold widened; the margin is rounded to fp32 as on the device */
+        double c = theta > 0.0 ? (double)(float)(-log(theta)) : INFINITY;
+        return (z1 - z2) < c;
+    }
+    if (flags & MARS_ORACLE_RULE_MARGIN) return (z1 - z2) < theta;
     int guard = (flags & MARS_ORACLE_SIGN_LITERAL) ? 1 : (z1 > 0.0);
     volatile double r = z2 / z1;
     return guard && (r > theta);

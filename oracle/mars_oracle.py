@@ -27,6 +27,8 @@ _lib = None
 
 SIGN_LITERAL = 1
 SHARED_PARENT = 2
+RULE_MARGIN = 8
+RULE_PROB_RATIO = 16
 
 _DT = {np.dtype(np.uint16): 0, np.dtype(np.float32): 1, np.dtype(np.float64): 2}
 

@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 
 namespace mars {
@@ -72,12 +73,29 @@ __device__ __forceinline__ Rec finish_record(Rec r)
     return r;
 }
 
-// Adaptive-relaxation bit of one row: sign guard, then r = z2/z1 > theta with one IEEE
-// round-to-nearest division (Eq. 4; strict comparison as in Sec. 3.4 / Algorithm 1).
+// Adaptive-relaxation bit of one row.  Default: sign guard, then r = z2/z1 > theta with one
+// IEEE round-to-nearest division (Eq. 4; strict comparison as in Sec. 3.4 / Algorithm 1).
+// With flag bit 3 (fixed-margin variant) the test is Delta = z1 - z2 < theta instead, one fp32
+// subtraction (Delta as defined with Eq. 5); the probability-ratio variant is mapped onto it
+// on the host, see rule_threshold().
 __device__ __forceinline__ bool relax_bit(float z1, float z2, float theta, uint32_t flags)
 {
+    if (flags & 8u) return __fsub_rn(z1, z2) < theta;
     bool guard = (flags & 1u) ? true : (z1 > 0.0f);
     return guard && (__fdiv_rn(z2, z1) > theta);
+}
+
+// Host: p2/p1 = exp(z2 - z1) > theta  <=>  z1 - z2 < -ln(theta)  (Sec. 3.3: the probability
+// ratio is the exponentiated logit difference).  Rewrites the probability-ratio variant
+// (flag bit 4) as a fixed margin c = -ln(theta), computed in double and rounded once;
+// theta <= 0 accepts every runner-up (c = +inf).
+inline void rule_threshold(float *theta, uint32_t *flags)
+{
+    if (*flags & 16u) {
+        const double t = (double)*theta;
+        *theta = t > 0.0 ? (float)(-log(t)) : INFINITY;
+        *flags = (*flags & ~16u) | 8u;
+    }
 }
 
 struct TailArgs {

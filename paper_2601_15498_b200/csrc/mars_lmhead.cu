@@ -721,7 +721,10 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     if (!hidden || !w_vocab || !tok || !parent || !accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
     if (B < 1 || N < 1 || V < 2 || d < 1 || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
     if (((uintptr_t)hidden & 15) || ((uintptr_t)w_vocab & 15)) return MARS_ERR_INVALID_ARG;
-    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT)) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO))
+        return MARS_ERR_UNSUPPORTED;
+    if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
+    rule_threshold(&theta, &flags);
     if (!lm_supported(B, N, V, d)) return MARS_ERR_UNSUPPORTED;
     const size_t need = mars_lmhead_workspace_bytes(B, N, V, d);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;

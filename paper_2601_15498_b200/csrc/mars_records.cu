@@ -39,7 +39,10 @@ extern "C" mars_status_t mars_verify_records(const void *records, int G, const i
     if (!records || ((uintptr_t)records & 15) || !tok || !parent || !accept_len || !out_tokens || !out_len)
         return MARS_ERR_INVALID_ARG;
     if (G < 1 || B < 1 || N < 1 || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
-    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT)) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO))
+        return MARS_ERR_UNSUPPORTED;
+    if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
+    rule_threshold(&theta, &flags);
     if (N > MARS_MAX_NODES || G > 4096) return MARS_ERR_UNSUPPORTED;
     TailArgs t;
     t.tok = tok; t.parent = parent; t.accept_len = accept_len; t.out_tokens = out_tokens;

@@ -376,7 +376,11 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
         if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
         if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
     }
-    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_COUNTERS_ZERO)) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_COUNTERS_ZERO | MARS_RULE_MARGIN |
+                  MARS_RULE_PROB_RATIO))
+        return MARS_ERR_UNSUPPORTED;
+    if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
+    rule_threshold(&theta, &flags);
     if (!sizes_supported(B, N, V, (int)dt)) return MARS_ERR_UNSUPPORTED;
     const int es = dt == MARS_BF16 ? 2 : 4;
     if ((uintptr_t)logits % es) return MARS_ERR_INVALID_ARG;

@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 BF16, FP32 = 0, 1
-SIGN_LITERAL, SHARED_PARENT, COUNTERS_ZERO = 1, 2, 4
+SIGN_LITERAL, SHARED_PARENT, COUNTERS_ZERO, RULE_MARGIN, RULE_PROB_RATIO = 1, 2, 4, 8, 16
 MAX_NODES = 1024
 
 _lock = threading.Lock()

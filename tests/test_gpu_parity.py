@@ -356,3 +356,30 @@ def test_cuda_graph_replay_with_changing_inputs():
         got = mars.to_host(out)
         ref = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, 0.9)
         assert_same(got, ref, KEYS_TREE, "graph replay")
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_rule_variants_margin_and_probability_ratio(dtype):
+    w = synth.tree_workload("rv", 12, 40, 5, 3, 30000, dtype, DEV, 70, 0.9, 3.0, 15.0, 30.0, 0.5)
+    bits = synth.to_numpy_bits(w.logits)
+    seen = set()
+    for flags, thetas in ((mars.RULE_MARGIN, (0.0, 0.5, 1.0, 2.5, 100.0)),
+                          (mars.RULE_PROB_RATIO, (-1.0, 0.0, 0.05, 0.3, 0.6, 1.0))):
+        for theta in thetas:
+            out = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, theta, flags, debug=True))
+            ref = orc.verify_tree(bits, w.tok, w.parent, theta, flags)
+            assert_same(out, ref, KEYS_TREE, f"flags={flags} theta={theta}")
+            seen.add(tuple(out["accept_len"].tolist()))
+    assert len(seen) >= 3                       # the thresholds really change decisions
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.verify_tree(w.logits, w.tok, w.parent, 0.5, mars.RULE_MARGIN | mars.RULE_PROB_RATIO)
+    # chain entry point and the records path take the same flags
+    c = synth.cfg2(DEV, seed=71, B=6)
+    out = mars.to_host(mars.verify_chain(c.logits, c.draft, 1.0, mars.RULE_MARGIN, debug=True))
+    ref = orc.verify_chain(synth.to_numpy_bits(c.logits), c.draft, 1.0, orc.RULE_MARGIN)
+    assert_same(out, ref, ("accept_len", "out_tokens", "out_len", "top2_id"), "chain margin")
+    rec = mars.top2_shard(w.logits, w.B, w.N, 0)
+    out = mars.to_host(mars.verify_records(rec[None].contiguous(), w.tok, w.parent, 0.3,
+                                           mars.RULE_PROB_RATIO, debug=True))
+    ref = orc.verify_tree(bits, w.tok, w.parent, 0.3, orc.RULE_PROB_RATIO)
+    assert_same(out, ref, KEYS_TREE, "records prob ratio")

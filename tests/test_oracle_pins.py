@@ -473,3 +473,65 @@ def test_lmhead_small_against_hand_fp64():
     want = M - 1 if (z[2, order[2, 0]] > 0 and r2 > 0.0) else 2
     assert out["accept_len"][0] == want
     assert (out["top2_id"] == order[:, :2]).all()
+
+
+# --------------------------------------------------------------------------- rule variants
+
+def test_margin_variant_one_ulp_and_through_chain():
+    """Fixed-margin indicator: relax iff Delta = z1 - z2 < c (strict), one fp32 subtraction."""
+    c = F32(0.5)
+    z1 = F32(8.0)
+    on = F32(7.5)                                           # Delta == c exactly
+    closer = np.nextafter(on, F32(np.inf), dtype=F32)       # Delta just below c
+    farther = np.nextafter(on, F32(-np.inf), dtype=F32)
+    assert orc.relax(z1, closer, c, orc.RULE_MARGIN)
+    assert not orc.relax(z1, on, c, orc.RULE_MARGIN)
+    assert not orc.relax(z1, farther, c, orc.RULE_MARGIN)
+    assert orc.relax(-3.0, -3.25, c, orc.RULE_MARGIN)       # no sign guard for this indicator
+    assert not orc.relax(5.0, -np.inf, c, orc.RULE_MARGIN)
+    for z2, want in ((closer, 1), (on, 0)):
+        z = np.full((2, 8), -1.0, F32)
+        z[:, 2] = z1
+        z[:, 5] = z2
+        out = orc.verify_chain(z, np.array([[5]], np.int32), float(c), orc.RULE_MARGIN)
+        assert out["accept_len"][0] == want
+        out = orc.verify_chain(z, np.array([[2]], np.int32), float(c), orc.RULE_MARGIN)
+        assert out["accept_len"][0] == 1                     # exact match is unaffected
+
+
+def test_prob_ratio_variant_against_softmax_definition():
+    """p2/p1 > theta with p = softmax(z) (Eq. 3) evaluated in fp64 on whole rows, away from
+    the boundary; and the limits theta <= 0 (always) / theta >= 1 (never for distinct logits)."""
+    rng = np.random.default_rng(21)
+    n = 0
+    for _ in range(3000):
+        z = rng.normal(0, 3, 50).astype(np.float32)
+        theta = F32(rng.uniform(0.05, 0.95))
+        zs = np.sort(z.astype(np.float64))[::-1]
+        p = np.exp(zs - zs[0]); p /= p.sum()
+        ratio = p[1] / p[0]
+        if abs(ratio - float(theta)) < 1e-4:
+            continue
+        n += 1
+        assert orc.relax(zs[0], zs[1], theta, orc.RULE_PROB_RATIO) == (ratio > float(theta))
+    assert n > 2500
+    assert orc.relax(3.0, -40.0, 0.0, orc.RULE_PROB_RATIO) and orc.relax(3.0, -40.0, -1.0, orc.RULE_PROB_RATIO)
+    assert not orc.relax(3.0, 2.999, 1.0, orc.RULE_PROB_RATIO)
+    assert not orc.relax(3.0, 3.0, 1.0, orc.RULE_PROB_RATIO)      # p2/p1 == 1 is not > 1
+    # equal to the margin variant at c = -ln(theta)
+    for theta in (0.3, 0.6, 0.9):
+        c = F32(-np.log(np.float64(F32(theta))))
+        for z2 in np.linspace(1.0, 3.0, 41):
+            assert orc.relax(3.0, z2, theta, orc.RULE_PROB_RATIO) == orc.relax(3.0, z2, c, orc.RULE_MARGIN)
+
+
+def test_variants_only_change_relaxed_accepts():
+    rng = np.random.default_rng(22)
+    z, draft = planted_chain(rng, 300, 6, 64)
+    strict = orc.verify_chain(z, draft, 1.5)["accept_len"]
+    for flags, th in ((orc.RULE_MARGIN, 0.0), (orc.RULE_PROB_RATIO, 1.0)):      # nothing relaxes
+        assert (orc.verify_chain(z, draft, th, flags)["accept_len"] == strict).all()
+    loose = orc.verify_chain(z, draft, 100.0, orc.RULE_MARGIN)["accept_len"]    # every runner-up relaxes
+    assert (loose >= strict).all() and (loose > strict).any()
+    mid = orc.verify_chain(z, draft, 2.0, orc.RULE_MARGIN)["accept_len"]        # planted gaps 0..3
+    assert (mid >= strict).all() and (mid <= loose).all() and (mid != loose).any() and (mid != strict).any()
