@@ -383,3 +383,27 @@ def test_rule_variants_margin_and_probability_ratio(dtype):
                                            mars.RULE_PROB_RATIO, debug=True))
     ref = orc.verify_tree(bits, w.tok, w.parent, 0.3, orc.RULE_PROB_RATIO)
     assert_same(out, ref, KEYS_TREE, "records prob ratio")
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_sorted_rows_worst_case_for_the_filter(dtype):
+    """Ascending rows make every batch beat the running bound (the exact path runs all the
+    time); descending rows decide everything in the first batch.  Both must stay exact,
+    including the many ties that bf16 rounding creates in a ramp."""
+    V = 151936
+    ramp = torch.linspace(-20.0, 20.0, V)
+    rows = torch.stack([ramp, ramp.flip(0), ramp * 0.5 + 3, (ramp * 0.25).flip(0), ramp.abs(), -ramp.abs()])
+    z = rows.repeat(4, 1).to(dtype).to(DEV)                     # 24 rows -> rows are split
+    N = 6
+    parent = np.tile(np.arange(-1, N - 1, dtype=np.int32), (4, 1))
+    ids = orc.top2(synth.to_numpy_bits(z))[1].reshape(4, N, 2)
+    tok = np.full((4, N), -1, np.int32)
+    tok[:, 1:] = ids[:, :-1, 1]                                 # always draft the runner-up
+    for theta in (0.9, 0.9999):
+        out, ref = run_tree(z, tok, parent, theta)
+        assert_same(out, ref, KEYS_TREE, f"sorted rows theta={theta}")
+    big = rows[:2].repeat(1300, 1).to(dtype).to(DEV)            # 2600 rows: one block per row
+    val, idx = orc.top2(synth.to_numpy_bits(big[:2]))
+    out = mars.to_host(mars.verify_chain(big, np.zeros((1300, 1), np.int32), 0.9, debug=True))
+    assert np.array_equal(out["top2_id"][:2], idx) and np.array_equal(out["top2_id"][-2:], idx)
+    assert np.array_equal(out["top2_val"][:2].view(np.uint32), val.view(np.uint32))
