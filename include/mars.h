@@ -180,6 +180,22 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Telemetry: histograms of the top-2 statistics that the paper plots for its target models
+ * (Fig. 3: top-1 logit values, logit ratios z2/z1, probability ratios p2/p1; Fig. 1 scatters
+ * the same quantities), from the [rows, 2] top-2 values a verification call wrote to
+ * mars_debug_out_t.top2_val.  No logits are read again.
+ *   hist      out, uint32 [3, nbins] (1 <= nbins <= 256), cleared by the call:
+ *             [0] z1 over [z1_lo, z1_hi) in nbins equal bins;
+ *             [1] r = z2/z1 over [0, 1] for rows with z1 > 0 (r == 1 goes to the last bin);
+ *             [2] p2/p1 = exp(z2 - z1) over (0, 1]: bin k holds k/nbins <= p2/p1 < (k+1)/nbins,
+ *                 decided as a comparison of z1 - z2 with (float)(-ln(k/nbins)).
+ *   outliers  out, uint32 [3]: rows outside the range of the respective histogram (z1 outside
+ *             [z1_lo, z1_hi) or not finite; z1 <= 0 or r outside [0, 1] or NaN; z1 - z2 NaN).
+ */
+mars_status_t mars_top2_histograms(const float *top2_val, int64_t rows, float z1_lo, float z1_hi,
+                                   int nbins, uint32_t *hist, uint32_t *outliers, void *cuda_stream);
+
+/*
  * Self-test of the bounded device-side wait used by mars_lmhead_verify's pipeline (the paper
  * has no counterpart).  Launches one block that waits, with the pipeline's own wait routine,
  * on a barrier that nothing ever signals; the wait must give up after `budget_cycles` SM

@@ -331,3 +331,48 @@ void mars_oracle_verify_chain(const void *logits, int dtype, int64_t ld, const i
         out_len[b] = n;
     }
 }
+
+/*
+ * Histograms of the top-2 statistics plotted in the paper's Fig. 3 (top-1 logit, logit ratio
+ * z2/z1, probability ratio p2/p1 = exp(z2 - z1) by Eq. 3), from [rows, 2] fp32 top-2 values.
+ * Bin rules (all fp32, one operation at a time):
+ *   z1:     [lo, hi) in nbins equal bins, bin = floor((z1 - lo) * (nbins / (hi - lo)));
+ *   ratio:  rows with z1 > 0 and 0 <= r <= 1, bin = min(nbins-1, floor(r * nbins));
+ *   p2/p1:  bin k holds k/nbins <= p2/p1 < (k+1)/nbins, decided in the logit-difference domain:
+ *           bin = #{k in 1..nbins-1 : z1 - z2 <= (float)(-ln(k/nbins))}.
+ * Rows outside a histogram's range are counted in outliers[which].
+ */
+void mars_oracle_histograms(const float *val, int64_t rows, float lo, float hi, int nbins,
+                            uint32_t *hist, uint32_t *outliers)
+{
+    memset(hist, 0, sizeof(uint32_t) * 3 * (size_t)nbins);
+    memset(outliers, 0, sizeof(uint32_t) * 3);
+    volatile float inv_w = (float)nbins / (hi - lo);
+    for (int64_t r = 0; r < rows; ++r) {
+        float z1 = val[2 * r], z2 = val[2 * r + 1];
+        if (z1 >= lo && z1 < hi) {
+            volatile float d = z1 - lo;
+            volatile float t = d * inv_w;
+            int b = (int)floorf(t);
+            if (b < 0) b = 0;
+            if (b > nbins - 1) b = nbins - 1;
+            hist[b]++;
+        } else outliers[0]++;
+        volatile float ratio = z2 / z1;
+        if (z1 > 0.0f && ratio >= 0.0f && ratio <= 1.0f) {
+            volatile float t = ratio * (float)nbins;
+            int b = (int)floorf(t);
+            if (b > nbins - 1) b = nbins - 1;
+            hist[nbins + b]++;
+        } else outliers[1]++;
+        volatile float delta = z1 - z2;
+        if (delta >= 0.0f) {
+            int b = 0;
+            for (int k = 1; k < nbins; ++k) {
+                float e = (float)(-log((double)k / (double)nbins));
+                if (delta <= e) b++;
+            }
+            hist[2 * nbins + b]++;
+        } else outliers[2]++;
+    }
+}

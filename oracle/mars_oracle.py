@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
             L.mars_oracle_verify_tree.restype = None
             L.mars_oracle_verify_chain.argtypes = [vp, i32, i64, vp, i32, i32, i64, f64, u32] + [vp] * 7
             L.mars_oracle_verify_chain.restype = None
+            L.mars_oracle_histograms.argtypes = [vp, i64, ctypes.c_float, ctypes.c_float, i32, vp, vp]
+            L.mars_oracle_histograms.restype = None
             _lib = L
     return _lib
 
@@ -213,3 +215,12 @@ def lmhead_verify_tree(hidden_bits, w_bits, bias, tok, parent, theta, flags: int
     out = verify_tree(z, tok, parent, float(np.float32(theta)), flags, Dcap)
     out["logits"] = z
     return out
+
+
+def histograms(top2_val: np.ndarray, lo: float, hi: float, nbins: int):
+    """Histograms of z1, z2/z1 and p2/p1 from [rows, 2] fp32 top-2 values; see mars_oracle.c."""
+    v = np.ascontiguousarray(top2_val, np.float32)
+    hist = np.zeros((3, nbins), np.uint32)
+    outl = np.zeros(3, np.uint32)
+    lib().mars_oracle_histograms(_p(v), v.shape[0], float(lo), float(hi), int(nbins), _p(hist), _p(outl))
+    return hist, outl

@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_records.restype = i32
             L.mars_selftest_bounded_wait.argtypes = [i64, vp, vp]
             L.mars_selftest_bounded_wait.restype = i32
+            L.mars_top2_histograms.argtypes = [vp, i64, f32, f32, i32, vp, vp, vp]
+            L.mars_top2_histograms.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -301,6 +303,23 @@ def verify_records(records: torch.Tensor, tok, parent, theta: float, flags: int 
     _check(code, "mars_verify_records")
     out["_keepalive"] = (tok, parent, records)
     return out
+
+
+def top2_histograms(top2_val: torch.Tensor, z1_lo: float, z1_hi: float, nbins: int):
+    """mars_top2_histograms on the current stream: returns (hist uint32-as-int32 [3, nbins],
+    outliers [3]) device tensors."""
+    if not (top2_val.is_cuda and top2_val.dtype == torch.float32 and top2_val.is_contiguous()
+            and top2_val.dim() == 2 and top2_val.shape[1] == 2):
+        raise MarsError("top2_val must be a contiguous float32 [rows, 2] device tensor")
+    dev = top2_val.device
+    hist = torch.empty((3, nbins), dtype=torch.int32, device=dev)
+    outl = torch.empty((3,), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_top2_histograms(top2_val.data_ptr(), top2_val.shape[0], float(z1_lo),
+                                          float(z1_hi), int(nbins), hist.data_ptr(), outl.data_ptr(),
+                                          _stream())
+    _check(code, "mars_top2_histograms")
+    return hist, outl
 
 
 def alloc_outputs(B: int, N: int, Dcap: int, device, debug: bool = False) -> dict:

@@ -535,3 +535,32 @@ def test_variants_only_change_relaxed_accepts():
     assert (loose >= strict).all() and (loose > strict).any()
     mid = orc.verify_chain(z, draft, 2.0, orc.RULE_MARGIN)["accept_len"]        # planted gaps 0..3
     assert (mid >= strict).all() and (mid <= loose).all() and (mid != loose).any() and (mid != strict).any()
+
+
+# --------------------------------------------------------------------------- telemetry
+
+def test_histograms_against_numpy_histogram():
+    """z1, z2/z1 and p2/p1 = exp(z2 - z1) binned by numpy in fp64, on values kept away from
+    the bin edges; plus hand rows for the edge conventions."""
+    rng = np.random.default_rng(31)
+    nb, lo, hi = 20, 0.0, 40.0
+    z1 = rng.uniform(0.5, 39.5, 20000)
+    r = rng.uniform(0.0, 1.0, 20000)
+    z2 = z1 * r
+    v = np.stack([z1, z2], 1).astype(np.float32)
+    z1f, z2f = v[:, 0].astype(np.float64), v[:, 1].astype(np.float64)
+    q = [(z1f - lo) / (hi - lo) * nb, z2f / z1f * nb, np.exp(z2f - z1f) * nb]
+    keep = np.ones(len(v), bool)
+    for x in q:
+        keep &= np.abs(x - np.round(x)) > 1e-3
+    v = v[keep]
+    hist, outl = orc.histograms(v, lo, hi, nb)
+    z1f, z2f = v[:, 0].astype(np.float64), v[:, 1].astype(np.float64)
+    assert (hist[0] == np.histogram(z1f, nb, (lo, hi))[0]).all()
+    assert (hist[1] == np.histogram(z2f / z1f, nb, (0.0, 1.0))[0]).all()
+    assert (hist[2] == np.histogram(np.exp(z2f - z1f), nb, (0.0, 1.0))[0]).all()
+    assert outl.tolist() == [0, 0, 0] and hist.sum(1).tolist() == [len(v)] * 3
+    hand = np.array([[10, 9], [20, 5], [5, 5], [-1, -2], [3, -np.inf], [np.nan, np.nan], [40, 1]], np.float32)
+    hist, outl = orc.histograms(hand, 0, 30, 6)
+    assert hist[0].tolist() == [1, 1, 1, 0, 1, 0] and hist[1].tolist() == [1, 1, 0, 0, 0, 2]
+    assert hist[2].tolist() == [3, 0, 2, 0, 0, 1] and outl.tolist() == [3, 3, 1]
