@@ -99,7 +99,12 @@ def test_cfg3_full_size_sampled(dtype):
     checks a sample of whole sequences, every sequence is checked for validity."""
     w = synth.cfg3(DEV, dtype=dtype)
     assert w.R == 15360
-    out = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, debug=True))
+    # as the benchmark launches it: workspace zeroed once, counters left to the kernel's own reset
+    work = torch.zeros(mars.workspace_bytes(w.B, w.N, w.V, mars.BF16 if dtype == torch.bfloat16 else mars.FP32),
+                       dtype=torch.uint8, device=DEV)
+    mars.verify_tree(w.logits, w.tok, w.parent, w.theta, flags=mars.COUNTERS_ZERO, workspace=work)
+    out = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, flags=mars.COUNTERS_ZERO,
+                                        debug=True, workspace=work))
     rng = np.random.default_rng(0)
     sample = sorted(set(rng.choice(w.B, 10, replace=False).tolist()) | {0, w.B - 1})
     rows = np.concatenate([np.arange(b * w.N, (b + 1) * w.N) for b in sample])
