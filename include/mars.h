@@ -180,6 +180,22 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Exact top-k of logits rows with token ids (1 <= k <= 32, k <= V): the selection a drafter
+ * makes when it expands a token tree with the k best continuations of a node (the paper's
+ * setup builds its draft trees with top-k = 10, Sec. 4.1).  Same streaming read of each row
+ * and the same total order as the verification calls (larger value first, lower id first
+ * among equal values, NaN counts as -inf, -0 reported as +0); rows with fewer than k entries
+ * above -inf are completed with the lowest unused ids at value -inf.
+ *   logits    [rows, ld] of `dt`, first V columns of each row are read.
+ *   out_val   float [rows, k], out_id int32 [rows, k]: best first.
+ *   workspace mars_topk_workspace_bytes(rows, V, dt, k) bytes, 256-byte aligned.
+ */
+size_t mars_topk_workspace_bytes(int64_t rows, int V, mars_dtype_t dt, int k);
+mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, int64_t rows, int V,
+                             int k, float *out_val, int32_t *out_id, void *workspace,
+                             size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Telemetry: histograms of the top-2 statistics that the paper plots for its target models
  * (Fig. 3: top-1 logit values, logit ratios z2/z1, probability ratios p2/p1; Fig. 1 scatters
  * the same quantities), from the [rows, 2] top-2 values a verification call wrote to

@@ -376,3 +376,42 @@ void mars_oracle_histograms(const float *val, int64_t rows, float lo, float hi, 
         } else outliers[2]++;
     }
 }
+
+/*
+ * Exact top-k of each row under the total order (value descending, token id ascending, NaN as
+ * -inf): one sequential pass per row keeping a sorted list of the k best so far.  Used for the
+ * draft-tree expansion with the k best continuations (the paper's setup: top-k = 10, Sec. 4.1).
+ *   val [R,k] (float for dtype 0/1, double for 2), id [R,k], best first.
+ */
+void mars_oracle_topk(const void *logits, int dtype, int64_t ld, int64_t R, int64_t V, int k,
+                      void *val, int32_t *id)
+{
+    size_t e = dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < R; ++r) {
+        const char *row = (const char *)logits + (size_t)r * (size_t)ld * e;
+        double bx[64];
+        int64_t bj[64];
+        int n = 0;
+        for (int64_t j = 0; j < V; ++j) {
+            double x;
+            if (dtype == ORACLE_BF16) x = (double)bf16_to_f32(((const uint16_t *)row)[j]);
+            else if (dtype == ORACLE_FP32) x = (double)((const float *)row)[j];
+            else x = ((const double *)row)[j];
+            if (x != x) x = -INFINITY;
+            /* position of (x, j) in the sorted list: behind everything that beats it */
+            int pos = n;
+            while (pos > 0 && beats_f64(x, j, bx[pos - 1], bj[pos - 1])) --pos;
+            if (pos >= k) continue;
+            int last = n < k ? n : k - 1;
+            for (int t = last; t > pos; --t) { bx[t] = bx[t - 1]; bj[t] = bj[t - 1]; }
+            bx[pos] = x; bj[pos] = j;
+            if (n < k) ++n;
+        }
+        for (int t = 0; t < k; ++t) {
+            if (dtype == ORACLE_FP64) ((double *)val)[r * k + t] = bx[t] + 0.0;
+            else ((float *)val)[r * k + t] = (float)bx[t] + 0.0f;
+            id[r * k + t] = (int32_t)bj[t];
+        }
+    }
+}

@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
             L.mars_oracle_verify_chain.restype = None
             L.mars_oracle_histograms.argtypes = [vp, i64, ctypes.c_float, ctypes.c_float, i32, vp, vp]
             L.mars_oracle_histograms.restype = None
+            L.mars_oracle_topk.argtypes = [vp, i32, i64, i64, i64, i32, vp, vp]
+            L.mars_oracle_topk.restype = None
             _lib = L
     return _lib
 
@@ -224,3 +226,18 @@ def histograms(top2_val: np.ndarray, lo: float, hi: float, nbins: int):
     outl = np.zeros(3, np.uint32)
     lib().mars_oracle_histograms(_p(v), v.shape[0], float(lo), float(hi), int(nbins), _p(hist), _p(outl))
     return hist, outl
+
+
+def topk(logits: np.ndarray, k: int, V: int | None = None):
+    """Exact top-k per row (values [R,k], ids [R,k], best first) under the library's total order."""
+    if logits.ndim != 2 or not logits.flags.c_contiguous or logits.dtype not in _DT:
+        raise ValueError("logits must be a C-contiguous [R, ld] array of uint16/float32/float64")
+    dt = _DT[logits.dtype]
+    V = logits.shape[1] if V is None else int(V)
+    if not (1 <= k <= 64 and k <= V <= logits.shape[1]):
+        raise ValueError("need 1 <= k <= min(64, V) and V <= ld")
+    R, ld = logits.shape
+    val = np.empty((R, k), np.float64 if dt == 2 else np.float32)
+    idx = np.empty((R, k), np.int32)
+    lib().mars_oracle_topk(_p(logits), dt, ld, R, V, int(k), _p(val), _p(idx))
+    return val, idx

@@ -70,6 +70,10 @@ def lib() -> ctypes.CDLL:
             L.mars_selftest_bounded_wait.restype = i32
             L.mars_top2_histograms.argtypes = [vp, i64, f32, f32, i32, vp, vp, vp]
             L.mars_top2_histograms.restype = i32
+            L.mars_topk_workspace_bytes.argtypes = [i64, i32, i32, i32]
+            L.mars_topk_workspace_bytes.restype = sz
+            L.mars_topk_rows.argtypes = [vp, i64, i32, i64, i32, i32, vp, vp, vp, sz, vp]
+            L.mars_topk_rows.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -320,6 +324,26 @@ def top2_histograms(top2_val: torch.Tensor, z1_lo: float, z1_hi: float, nbins: i
                                           _stream())
     _check(code, "mars_top2_histograms")
     return hist, outl
+
+
+def topk_rows(logits: torch.Tensor, k: int, V: int | None = None,
+              workspace: torch.Tensor | None = None):
+    """mars_topk_rows on the current stream: (values float32 [rows, k], ids int32 [rows, k])."""
+    dev = logits.device
+    dt, ld, V = _logits_args(logits, logits.shape[0], V)
+    rows = logits.shape[0]
+    need = int(lib().mars_topk_workspace_bytes(rows, V, dt, int(k)))
+    if need == 0:
+        raise MarsError("unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    val = torch.empty((rows, k), dtype=torch.float32, device=dev)
+    idx = torch.empty((rows, k), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_topk_rows(logits.data_ptr(), ld, dt, rows, V, int(k), val.data_ptr(),
+                                    idx.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream())
+    _check(code, "mars_topk_rows")
+    return val, idx
 
 
 def alloc_outputs(B: int, N: int, Dcap: int, device, debug: bool = False) -> dict:

@@ -1,0 +1,70 @@
+"""Exact top-k of logits rows on the device against the oracle: ids and value bits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mars_oracle as orc
+from paper_2601_15498_b200 import mars, synth
+from tests.test_gpu_parity import special_rows
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def check(logits, k, V=None):
+    val, idx = mars.topk_rows(logits, k, V=V)
+    torch.cuda.synchronize()
+    src = logits if V is None else logits[:, :V].contiguous()
+    rv, ri = orc.topk(synth.to_numpy_bits(src), k)
+    assert np.array_equal(idx.cpu().numpy(), ri), f"ids k={k}"
+    assert np.array_equal(val.cpu().numpy().view(np.uint32), rv.view(np.uint32)), f"values k={k}"
+
+
+@pytest.fixture(autouse=True)
+def _no_forced_split(monkeypatch):
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+
+
+@pytest.mark.parametrize("k", [1, 2, 10, 32])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_topk_qwen_and_vicuna_sized_rows(k, dtype):
+    g = torch.Generator(device=DEV); g.manual_seed(k)
+    for R, V in ((60, 151936), (700, 32000), (10, 32000)):       # split rows, whole rows, few rows
+        z = (torch.randn((R, V), generator=g, device=DEV) * 3).to(dtype)
+        check(z, k)
+
+
+@pytest.mark.parametrize("V", [1, 2, 9, 33, 257, 4099, 18437])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_topk_odd_sizes_and_degenerate_rows(V, dtype):
+    g = torch.Generator(device="cpu"); g.manual_seed(V)
+    z = (torch.randn((5, V), generator=g) * 3).to(dtype).to(DEV)
+    for k in sorted({1, min(2, V), min(10, V), min(32, V)}):
+        check(z, k)
+    if V >= 9:
+        s = special_rows(V, dtype)
+        for k in (2, min(9, V)):
+            check(s, k)
+
+
+@pytest.mark.parametrize("S", [2, 5, 64])
+def test_topk_forced_split_and_unaligned(monkeypatch, S):
+    monkeypatch.setenv("MARS_FORCE_SPLIT", str(S))
+    g = torch.Generator(device=DEV); g.manual_seed(S)
+    big = torch.full((9, 40007 + 11), 3.0e38, dtype=torch.bfloat16, device=DEV)     # canaries around
+    view = big[1:-1, 3:3 + 40007]
+    view.copy_((torch.randn((7, 40007), generator=g, device=DEV) * 3).to(torch.bfloat16))
+    view[2] = torch.round(view[2].float()).to(torch.bfloat16)                      # heavy ties
+    val, idx = mars.topk_rows(view, 10)
+    torch.cuda.synchronize()
+    rv, ri = orc.topk(synth.to_numpy_bits(view.contiguous()), 10)
+    assert np.array_equal(idx.cpu().numpy(), ri) and np.array_equal(val.cpu().numpy(), rv)
+    asc = torch.linspace(-5, 5, 40007, device=DEV).repeat(3, 1).to(torch.bfloat16)   # worst case for the filter
+    check(asc, 10)
+
+
+def test_topk_host_errors():
+    z = torch.zeros((4, 100), device=DEV)
+    for k in (0, 33, 101):
+        with pytest.raises(mars.MarsError):
+            mars.topk_rows(z, k)

@@ -564,3 +564,28 @@ def test_histograms_against_numpy_histogram():
     hist, outl = orc.histograms(hand, 0, 30, 6)
     assert hist[0].tolist() == [1, 1, 1, 0, 1, 0] and hist[1].tolist() == [1, 1, 0, 0, 0, 2]
     assert hist[2].tolist() == [3, 0, 2, 0, 0, 1] and outl.tolist() == [3, 3, 1]
+
+
+# --------------------------------------------------------------------------- top-k
+
+@pytest.mark.parametrize("k", [1, 2, 10, 32])
+def test_topk_matches_library_sort_and_top2(k):
+    rng = np.random.default_rng(40 + k)
+    V = 500
+    z = rng.normal(0, 3, size=(12, V)).astype(np.float32)
+    z[2] = np.round(z[2])                   # ties
+    z[3] = 2.0                              # constant
+    z[4, ::3] = np.nan
+    z[5] = -np.inf
+    z[5, [7, 400]] = [1.0, 1.0]             # only two entries above -inf
+    for a in (z, bf16_bits(z), z.astype(np.float64)):
+        val, idx = orc.topk(a, k)
+        x = widen(a).astype(np.float64)
+        x = np.where(np.isnan(x), -np.inf, x)
+        for r in range(len(a)):
+            order = np.lexsort((np.arange(V), -x[r]))[:k]
+            assert idx[r].tolist() == order.tolist(), (r, k)
+            assert (val[r] == x[r][order]).all()
+        if k == 2:
+            v2, i2 = orc.top2(a)
+            assert (i2 == idx).all() and (v2 == val).all()
