@@ -242,6 +242,24 @@ mars_status_t mars_top2_shard(const void *logits, int64_t ld, mars_dtype_t dt, i
                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Vocabulary-parallel verification, step 1 of 2, fused form: the output projection of one
+ * vocabulary shard (Eq. 2 of the paper restricted to rows [id_offset, id_offset + V_local) of
+ * W_o) reduced to per-row top-2 records inside the GEMM epilogue, as mars_lmhead_verify does,
+ * but handed on as records with GLOBAL token ids for mars_verify_records.  Every logit is the
+ * same fp32 sum as in the unsharded call, so the merged result is bit-identical to it.
+ *   hidden      bf16 [B*N, d] (replicated on every rank); w_shard bf16 [V_local, d];
+ *               bias_shard fp32 [V_local] or NULL; d a multiple of 64.
+ *   records     out, [B*N] 16-byte records {z1, id1, z2, id2}, 16-byte aligned.
+ *   workspace   mars_lmhead_workspace_bytes(B, N, V_local, d) bytes.  After a device-side
+ *               timeout (see mars_lmhead_verify) all records are empty (ids 0x7fffffff) and the
+ *               first uint32 of the workspace holds MARS_SEQ_TIMEOUT.
+ */
+mars_status_t mars_lmhead_top2_shard(const void *hidden, const void *w_shard, const float *bias_shard,
+                                     int d, int B, int N, int V_local, int32_t id_offset,
+                                     void *records, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream);
+
+/*
  * Vocabulary-parallel verification, step 2 of 2: merge the G shard records of every row and
  * verify (three-way rule of Sec. 3.4, tree resolution as mars_verify_tree).  The merge is
  * associative and commutative under the total order, so outputs are bit-identical to

@@ -614,6 +614,22 @@ __global__ void __launch_bounds__(128) lmhead_tail_kernel(const LmParams p, cons
     });
 }
 
+// Vocabulary shard: merge a row's per-chunk records into one record with global token ids
+// (local id + id_offset), left unfinished for mars_verify_records.  One thread per row.
+__global__ void __launch_bounds__(128) lmhead_records_kernel(const LmParams p, int id_offset, Rec *records)
+{
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= p.M) return;
+    Rec acc = empty_rec();
+    if (*(volatile unsigned *)p.status == 0) {
+        const Rec *base = p.partial + (size_t)row * p.n_chunks;
+        for (int k = 0; k < p.n_chunks; ++k) acc = merge(acc, base[k]);
+        if (acc.id1 != kNoId) acc.id1 += id_offset;
+        if (acc.id2 != kNoId) acc.id2 += id_offset;
+    }
+    records[row] = acc;     // after a device-side timeout every record stays empty
+}
+
 // ----------------------------------------------------------------------------- host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -689,6 +705,71 @@ static bool lm_supported(int B, int N, int V, int d)
     return true;
 }
 
+// Shapes, tensor maps and launch of the GEMM + top-2 kernel; fills *pout for the kernels that
+// consume the per-chunk records.
+static mars_status_t lm_launch_gemm(const void *hidden, const void *w_vocab, const float *bias, int d,
+                                    int B, int N, int V, void *workspace, cudaStream_t st, LmParams *pout)
+{
+    const long long M = (long long)B * N;
+    const LmShape s = lm_shape(M, V);
+    LmParams p;
+    p.M = (int)M; p.V = V; p.d = d;
+    p.n_mtiles = s.n_mtiles; p.n_ntiles = s.n_ntiles; p.n_chunks = s.n_chunks; p.n_items = s.n_items;
+    p.chunk_tiles = s.chunk_tiles;
+    p.bias = bias;
+    p.status = (unsigned *)workspace;
+    p.partial = (Rec *)((char *)workspace + 256);
+
+    CUtensorMap map_h, map_w;
+    if (!make_map(&map_h, hidden, (uint64_t)M, (uint64_t)d, kBM)) return MARS_ERR_CUDA;
+    if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, lm_pair_mode() ? kBN / 2 : kBN)) return MARS_ERR_CUDA;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MARS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MARS_ERR_CUDA;
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)kLmSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(lmhead_top2_kernel_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kLm2SmemBytes);
+    });
+    if (attr_err != cudaSuccess) return MARS_ERR_CUDA;
+
+    if (cudaMemsetAsync(p.status, 0, 256, st) != cudaSuccess) return MARS_ERR_CUDA;
+    if (lm_pair_mode()) {
+        // persistent pairs: never launch more clusters than can be resident together
+        static std::once_flag occ_once;
+        static int max_pairs = 0;
+        std::call_once(occ_once, [&] {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(sms / 2 * 2); cfg.blockDim = dim3(kLmThreads);
+            cfg.dynamicSmemBytes = kLm2SmemBytes;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, lmhead_top2_kernel_pair, &cfg) == cudaSuccess && n > 0)
+                max_pairs = n;
+            else
+                max_pairs = sms / 2;
+            (void)cudaGetLastError();
+        });
+        int pairs = max_pairs < sms / 2 ? max_pairs : sms / 2;
+        if (s.n_items < pairs) pairs = s.n_items;
+        lmhead_top2_kernel_pair<<<2 * pairs, kLmThreads, kLm2SmemBytes, st>>>(map_h, map_w, p);
+    } else {
+        const int grid = s.n_items < sms ? s.n_items : sms;
+        lmhead_top2_kernel<<<grid, kLmThreads, kLmSmemBytes, st>>>(map_h, map_w, p);
+    }
+    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    *pout = p;
+    return MARS_OK;
+}
+
 }  // namespace mars
 
 extern "C" {
@@ -698,6 +779,25 @@ size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d)
     if (!mars::lm_supported(B, N, V, d)) return 0;
     const mars::LmShape s = mars::lm_shape((long long)B * N, V);
     return 256 + (size_t)B * N * s.n_chunks * sizeof(mars::Rec);
+}
+
+mars_status_t mars_lmhead_top2_shard(const void *hidden, const void *w_shard, const float *bias_shard, int d,
+                                     int B, int N, int V_local, int32_t id_offset, void *records,
+                                     void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    using namespace mars;
+    if (!hidden || !w_shard || !records || ((uintptr_t)records & 15) || id_offset < 0) return MARS_ERR_INVALID_ARG;
+    if (B < 1 || N < 1 || V_local < 2 || d < 1) return MARS_ERR_INVALID_ARG;
+    if (((uintptr_t)hidden & 15) || ((uintptr_t)w_shard & 15)) return MARS_ERR_INVALID_ARG;
+    if (!lm_supported(B, N, V_local, d)) return MARS_ERR_UNSUPPORTED;
+    const size_t need = mars_lmhead_workspace_bytes(B, N, V_local, d);
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    LmParams p;
+    const mars_status_t gs = lm_launch_gemm(hidden, w_shard, bias_shard, d, B, N, V_local, workspace, st, &p);
+    if (gs != MARS_OK) return gs;
+    lmhead_records_kernel<<<(p.M + 127) / 128, 128, 0, st>>>(p, id_offset, (Rec *)records);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
 mars_status_t mars_selftest_bounded_wait(int64_t budget_cycles, void *scratch32, void *cuda_stream)
@@ -729,19 +829,10 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     const size_t need = mars_lmhead_workspace_bytes(B, N, V, d);
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;
 
-    const long long M = (long long)B * N;
-    const LmShape s = lm_shape(M, V);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
     LmParams p;
-    p.M = (int)M; p.V = V; p.d = d;
-    p.n_mtiles = s.n_mtiles; p.n_ntiles = s.n_ntiles; p.n_chunks = s.n_chunks; p.n_items = s.n_items;
-    p.chunk_tiles = s.chunk_tiles;
-    p.bias = bias;
-    p.status = (unsigned *)workspace;
-    p.partial = (Rec *)((char *)workspace + 256);
-
-    CUtensorMap map_h, map_w;
-    if (!make_map(&map_h, hidden, (uint64_t)M, (uint64_t)d, kBM)) return MARS_ERR_CUDA;
-    if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, lm_pair_mode() ? kBN / 2 : kBN)) return MARS_ERR_CUDA;
+    const mars_status_t gs = lm_launch_gemm(hidden, w_vocab, bias, d, B, N, V, workspace, st, &p);
+    if (gs != MARS_OK) return gs;
 
     TailArgs t;
     t.tok = tok; t.parent = parent; t.accept_len = accept_len; t.out_tokens = out_tokens;
@@ -751,49 +842,6 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     t.dbg_flags = dbg ? dbg->node_flags : nullptr;
     t.N = N; t.Dcap = Dcap; t.theta = theta; t.flags = flags; t.chain = 0;
 
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MARS_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MARS_ERR_CUDA;
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kLmSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(lmhead_top2_kernel_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kLm2SmemBytes);
-    });
-    if (attr_err != cudaSuccess) return MARS_ERR_CUDA;
-
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    if (cudaMemsetAsync(p.status, 0, 256, st) != cudaSuccess) return MARS_ERR_CUDA;
-    if (lm_pair_mode()) {
-        // persistent pairs: never launch more clusters than can be resident together
-        static std::once_flag occ_once;
-        static int max_pairs = 0;
-        std::call_once(occ_once, [&] {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(sms / 2 * 2); cfg.blockDim = dim3(kLmThreads);
-            cfg.dynamicSmemBytes = kLm2SmemBytes;
-            cudaLaunchAttribute at[1];
-            at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-            cfg.attrs = at; cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, lmhead_top2_kernel_pair, &cfg) == cudaSuccess && n > 0)
-                max_pairs = n;
-            else
-                max_pairs = sms / 2;
-            (void)cudaGetLastError();
-        });
-        int pairs = max_pairs < sms / 2 ? max_pairs : sms / 2;
-        if (s.n_items < pairs) pairs = s.n_items;
-        lmhead_top2_kernel_pair<<<2 * pairs, kLmThreads, kLm2SmemBytes, st>>>(map_h, map_w, p);
-    } else {
-        const int grid = s.n_items < sms ? s.n_items : sms;
-        lmhead_top2_kernel<<<grid, kLmThreads, kLmSmemBytes, st>>>(map_h, map_w, p);
-    }
-    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
     lmhead_tail_kernel<<<B, 128, tail_smem_bytes(N), st>>>(p, t);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }

@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
             L.mars_topk_workspace_bytes.restype = sz
             L.mars_topk_rows.argtypes = [vp, i64, i32, i64, i32, i32, vp, vp, vp, sz, vp]
             L.mars_topk_rows.restype = i32
+            L.mars_lmhead_top2_shard.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
+            L.mars_lmhead_top2_shard.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -275,6 +277,35 @@ def top2_shard(logits_local: torch.Tensor, B: int, N: int, id_offset: int, V_loc
         code = lib().mars_top2_shard(logits_local.data_ptr(), ld, dt, B, N, V_local, int(id_offset),
                                      records.data_ptr(), flags, workspace.data_ptr(), wbytes, _stream())
     _check(code, "mars_top2_shard")
+    return records
+
+
+def lmhead_top2_shard(hidden: torch.Tensor, w_shard: torch.Tensor, bias_shard, B: int, N: int,
+                      id_offset: int, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """mars_lmhead_top2_shard on the current stream: records int32 [B*N, 4] of one vocabulary
+    shard of the output projection (hidden bf16 [B*N, d], w_shard bf16 [V_local, d])."""
+    dev = hidden.device
+    if not (hidden.is_cuda and w_shard.is_cuda and hidden.dtype == torch.bfloat16
+            and w_shard.dtype == torch.bfloat16 and hidden.is_contiguous() and w_shard.is_contiguous()):
+        raise MarsError("hidden and w_shard must be contiguous bfloat16 device tensors")
+    M, d = hidden.shape
+    V_local = w_shard.shape[0]
+    if M != B * N or w_shard.shape[1] != d:
+        raise MarsError("shape mismatch")
+    if bias_shard is not None:
+        bias_shard = bias_shard.to(device=dev, dtype=torch.float32).contiguous()
+    need = int(lib().mars_lmhead_workspace_bytes(B, N, V_local, d))
+    if need == 0:
+        raise MarsError("unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    records = torch.empty((M, 4), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_lmhead_top2_shard(
+            hidden.data_ptr(), w_shard.data_ptr(), bias_shard.data_ptr() if bias_shard is not None else None,
+            d, B, N, V_local, int(id_offset), records.data_ptr(), workspace.data_ptr(), workspace.numel(),
+            _stream())
+    _check(code, "mars_lmhead_top2_shard")
     return records
 
 

@@ -62,3 +62,23 @@ def test_degenerate_rows_sharded(dtype):
             out = sharded(z, tok, parent, 0.9, ranges, flags)
             ref = orc.verify_tree(synth.to_numpy_bits(z), tok, parent, 0.9, flags)
             assert_same(out, ref, KEYS_TREE, f"which={which} flags={flags}")
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_lm_head_equals_unsharded_bit_for_bit(world):
+    """Each logit is the same fp32 accumulation whichever shard computes it, so the sharded
+    output projection followed by the record merge must reproduce mars_lmhead_verify exactly."""
+    w = synth.cfg4_operands(DEV, seed=50 + world, B=4, N=30, V=20000 + 8 * world, d=512, depth=4)
+    g = torch.Generator(device="cpu"); g.manual_seed(world)
+    bias = (torch.randn(w.V, generator=g) * 0.5).to(DEV)
+    zz = w.hidden.float() @ w.w_vocab.float().T + bias
+    lead = torch.topk(zz, 2, dim=1).indices.cpu().numpy()
+    tok = synth.make_tokens(w.parent, lead, w.V, 9)
+    ref = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, bias, tok, w.parent, 0.9, debug=True))
+    recs = []
+    for lo, hi in vocab_parallel.shard_ranges(w.V, world):
+        recs.append(mars.lmhead_top2_shard(w.hidden, w.w_vocab[lo:hi].contiguous(), bias[lo:hi].contiguous(),
+                                           w.B, w.N, lo))
+    out = mars.to_host(mars.verify_records(torch.stack(recs), tok, w.parent, 0.9, debug=True))
+    assert_same(out, ref, KEYS_TREE, f"lm head world={world}")
+    assert (out["seq_status"] == 0).all() and out["accept_len"].max() >= 1
