@@ -168,6 +168,8 @@ size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d);
  *   Remaining arguments, outputs and per-sequence statuses are those of mars_verify_tree.
  *   Accumulation order differs from a sequential sum, so near-ties may resolve differently
  *   from an fp64 evaluation; decisions are still taken in fp32 on the accumulated values.
+ *   The first call in a process sets function attributes and queries cluster occupancy
+ *   (host-side, once); make that first call outside any stream capture.
  *   If a bounded device-side wait gives up (which indicates a fault in the pipeline, not a
  *   property of the data), every sequence gets MARS_SEQ_TIMEOUT, accept_len 0, out_len 0 and
  *   out_tokens / path_nodes filled with -1.
