@@ -11,6 +11,9 @@
  *   - logits from the output projection z = W_o h + b_o                 (Eq. 2; logits
  *     are produced by the Python wrapper with an fp64 matmul, the rule below then
  *     runs on double rows)
+ *   - stochastic (T > 0) verification: Eq. 1 acceptance, residual draw     (Sec. 2.2, Eq. 3;
+ *     its composition with the relaxation is a reading of this repository, PARITY
+ *     UNPINNED by the paper -- see the block comment above that function)
  *
  * Only tests, the smoke check and the benchmark's CPU-baseline leg may call this file.
  * It shares no code, header, table or helper with the CUDA library.
@@ -413,5 +416,210 @@ void mars_oracle_topk(const void *logits, int dtype, int64_t ld, int64_t R, int6
             else ((float *)val)[r * k + t] = (float)bx[t] + 0.0f;
             id[r * k + t] = (int32_t)bj[t];
         }
+    }
+}
+
+/* ======================================================================================
+ * Stochastic (temperature T > 0) verification.
+ *
+ * What the paper fixes (Sec. 2.2): in stochastic decoding a drafted token is accepted with
+ * probability min(1, P_target / P_draft) (Eq. 1); on rejection the corrected token is drawn
+ * from a residual distribution that compensates for the draft; tree-based methods extend the
+ * same logic to a token tree; the target probabilities are the softmax of the logits (Eq. 3).
+ * Sec. 2.2 also says that MARS changes only the accept/reject decision and applies on top of
+ * sampling-based verification, and Sec. 4.1 that draft trees are built from the drafter's k
+ * best continuations.  HOW the relaxation composes with Eq. 1 is not stated anywhere.
+ *
+ * Reading taken here (a convention of this repository; the composition is PARITY UNPINNED by
+ * the paper, the pieces are pinned, see below):
+ *   - P(v) = exp(z_v / T) / sum_u exp(z_u / T) per row, evaluated in fp64 as
+ *     exp((z_v - m) / T) with m the row maximum (the same number); NaN logits count as -inf.
+ *   - Candidates are deterministic (a top-k expansion), so the draft distribution at a node is
+ *     a point mass on the candidate and Eq. 1 reads "accept x with probability P(x)".  The
+ *     children of the current node are tried in node order.  When child x is rejected, the
+ *     target distribution is replaced by its residual, which for a point-mass draft is P with
+ *     x removed and renormalised; the next sibling is judged against that residual, i.e. it
+ *     is accepted iff u * rem < e_x, where e_x is x's unnormalised mass, rem the mass that is
+ *     left, and u the node's uniform in [0, 1).  If no child is accepted the walk stops
+ *     and the next token is drawn from the residual by inverting its CDF in token-id order with
+ *     the sequence's uniform uniform[b, 0]: the smallest id j with sum_{k <= j} w_k > u * W.
+ *     At a leaf nothing was removed and the draw is from P itself (the bonus token).
+ *   - Composition with MARS (flags): by default a child that passes the three-way rule of
+ *     Sec. 3.4 on the current row (exact match, or runner-up with r > theta) is accepted
+ *     outright, and only the others take the Eq. 1 test; STOCH_RELAX_ONLY keeps Eq. 1 for the
+ *     top-1 as well and adds only the relaxed runner-up; STOCH_PLAIN is Eq. 1 alone (standard
+ *     speculative sampling, which preserves the target distribution exactly).
+ *   - A row whose maximum is not finite, or a residual without mass, has no distribution to
+ *     draw from: the walk stops there, the row's top-1 is emitted and the status is 4.
+ *   Pinned by tests: softmax against a library routine; CDF inversion against cumsum +
+ *   searchsorted; exact preservation of the target distribution for the first and second
+ *   emitted token in STOCH_PLAIN (the theorem behind Eq. 1); T -> 0 equals strict greedy;
+ *   u -> 1 in the default mode equals Algorithm 1 on chains; invariance under scaling logits
+ *   and T by a power of two.
+ * ==================================================================================== */
+#define MARS_ORACLE_STOCH_PLAIN 32u
+#define MARS_ORACLE_STOCH_RELAX_ONLY 64u
+
+static double row_get(const void *row, int dtype, int64_t j)
+{
+    double x;
+    if (dtype == ORACLE_BF16) x = (double)bf16_to_f32(((const uint16_t *)row)[j]);
+    else if (dtype == ORACLE_FP32) x = (double)((const float *)row)[j];
+    else x = ((const double *)row)[j];
+    return (x != x) ? -INFINITY : x;
+}
+
+/* Row maximum and softmax denominator sum_j exp((z_j - m)/T) (Eq. 3 with temperature). */
+static void row_softmax_stats(const void *row, int dtype, int64_t V, double T, double *m_out,
+                              double *S_out)
+{
+    double m = -INFINITY;
+    for (int64_t j = 0; j < V; ++j) { double x = row_get(row, dtype, j); if (x > m) m = x; }
+    double S = 0.0;
+    if (isfinite(m))
+        for (int64_t j = 0; j < V; ++j) S += exp((row_get(row, dtype, j) - m) / T);
+    *m_out = m;
+    *S_out = S;
+}
+
+/*
+ *   uniform   float [B,N]: uniform[b,i] (i > 0) judges node i; uniform[b,0] draws the final token
+ *   node_prob double [B,N] or NULL: P(tok[i]) under the PARENT's row (plain softmax, nothing removed);
+ *             0 for the root, padding nodes and ids outside [0,V)
+ *   node_how  uint8 [B,N] or NULL: 0 not visited, 1 exact match, 2 relaxed runner-up, 3 accepted by
+ *             Eq. 1, 4 rejected
+ *   margin    double [B,2] or NULL: [0] the smallest |e_x - u*rem| / S over the Eq. 1 tests taken,
+ *             [1] the distance of u*W from the nearer edge of the drawn token's CDF interval, / W
+ *             (how close each decision was to flipping; +inf where no such decision was taken)
+ */
+void mars_oracle_verify_tree_stochastic(const void *logits, int dtype, int64_t ld, const int32_t *tok,
+                                        const int32_t *parent, const float *uniform, int B, int N,
+                                        int64_t V, double theta, double temperature, uint32_t flags,
+                                        int Dcap, int32_t *accept_len, int32_t *out_tokens,
+                                        int32_t *path_nodes, int32_t *out_len, int32_t *status,
+                                        double *node_prob, uint8_t *node_how, double *margin)
+{
+    size_t e = dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8;
+    const double T = temperature;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const int32_t *par = (flags & MARS_ORACLE_SHARED_PARENT) ? parent : parent + (size_t)b * N;
+        const int32_t *tk = tok + (size_t)b * N;
+        const float *u = uniform + (size_t)b * N;
+        int32_t *otok = out_tokens + (size_t)b * (Dcap + 1);
+        int32_t *opath = path_nodes ? path_nodes + (size_t)b * (Dcap + 1) : NULL;
+        double *nprob = node_prob ? node_prob + (size_t)b * N : NULL;
+        uint8_t *nhow = node_how ? node_how + (size_t)b * N : NULL;
+        double mg_test = INFINITY, mg_draw = INFINITY;
+        fill(otok, Dcap + 1, -1);
+        fill(opath, Dcap + 1, -1);
+        if (nhow) memset(nhow, 0, (size_t)N);
+        if (nprob) for (int i = 0; i < N; ++i) nprob[i] = 0.0;
+
+        int st = 0;
+        if (par[0] != -1) st = 1;
+        for (int i = 1; i < N && !st; ++i)
+            if (par[i] >= i || par[i] < -1) st = 1;
+
+        /* plain softmax probability of every node's token under its parent's row */
+        if (nprob && !st) {
+            for (int i = 1; i < N; ++i) {
+                int p = par[i];
+                if (p < 0 || tk[i] < 0 || tk[i] >= V) continue;
+                const char *row = (const char *)logits + ((size_t)b * N + p) * (size_t)ld * e;
+                double m, S;
+                row_softmax_stats(row, dtype, V, T, &m, &S);
+                if (isfinite(m) && S > 0.0) nprob[i] = exp((row_get(row, dtype, tk[i]) - m) / T) / S;
+            }
+        }
+
+        int cur = 0, a = 0, bad_dist = 0;
+        int32_t removed[1024];
+        int nrem = 0;
+        float v2[2];
+        int32_t id2[2] = {0, 1};
+        double m = 0, S = 0;
+        const char *row = NULL;
+        if (opath) opath[0] = 0;
+        while (!st) {
+            row = (const char *)logits + ((size_t)b * N + cur) * (size_t)ld * e;
+            top2_row_f32(row, dtype, V, v2, id2);
+            int relax = mars_oracle_relax_f32(v2[0], v2[1], (float)theta, flags);
+            row_softmax_stats(row, dtype, V, T, &m, &S);
+            nrem = 0;
+            if (!isfinite(m) || !(S > 0.0)) { bad_dist = 1; break; }
+            double rem = S;
+            int next = -1;
+            for (int i = cur + 1; i < N && next < 0; ++i) {
+                if (par[i] != cur || tk[i] < 0) continue;
+                int32_t x = tk[i];
+                int gone = 0;
+                for (int k = 0; k < nrem; ++k) if (removed[k] == x) gone = 1;
+                double ex = (x < V && !gone) ? exp((row_get(row, dtype, x) - m) / T) : 0.0;
+                int how = (flags & MARS_ORACLE_STOCH_PLAIN) ? 0 : rule(x, id2, relax);
+                if ((flags & MARS_ORACLE_STOCH_RELAX_ONLY) && how == 1) how = 0;
+                if (how == 0) {
+                    double lhs = (double)u[i] * rem;          /* Eq. 1 on the running residual */
+                    double d = fabs(ex - lhs) / S;
+                    if (d < mg_test) mg_test = d;
+                    how = (lhs < ex) ? 3 : 4;
+                }
+                if (nhow) nhow[i] = (uint8_t)how;
+                if (how == 4) {
+                    if (ex > 0.0 && nrem < 1024) {
+                        rem -= ex; if (rem < 0.0) rem = 0.0;
+                        removed[nrem++] = x;
+                    }
+                } else next = i;
+            }
+            if (next < 0) break;
+            cur = next; ++a;
+            if (a <= Dcap) { otok[a - 1] = tk[cur]; if (opath) opath[a] = cur; }
+        }
+        if (!st && a > Dcap) st = 2;
+        if (st) {   /* malformed tree or path deeper than the outputs: accept nothing, emit the root's top-1 */
+            fill(otok, Dcap + 1, -1);
+            fill(opath, Dcap + 1, -1);
+            if (nhow) memset(nhow, 0, (size_t)N);
+            row = (const char *)logits + ((size_t)b * N) * (size_t)ld * e;
+            top2_row_f32(row, dtype, V, v2, id2);
+            accept_len[b] = 0; out_len[b] = 1; otok[0] = id2[0];
+            if (opath) opath[0] = 0;
+            if (status) status[b] = st;
+            if (margin) { margin[2 * b] = INFINITY; margin[2 * b + 1] = INFINITY; }
+            continue;
+        }
+        /* the next token: a draw from the residual of row `cur` (nothing removed at a leaf) */
+        int32_t drawn = id2[0];
+        if (!bad_dist) {
+            double W = 0.0;
+            for (int64_t j = 0; j < V; ++j) {
+                int gone = 0;
+                for (int k = 0; k < nrem; ++k) if (removed[k] == j) gone = 1;
+                if (!gone) W += exp((row_get(row, dtype, j) - m) / T);
+            }
+            if (!(W > 0.0)) bad_dist = 1;
+            else {
+                double target = (double)u[0] * W, c = 0.0, lo = 0.0;
+                int64_t pick = -1, last = -1;
+                for (int64_t j = 0; j < V && pick < 0; ++j) {
+                    int gone = 0;
+                    for (int k = 0; k < nrem; ++k) if (removed[k] == j) gone = 1;
+                    double w = gone ? 0.0 : exp((row_get(row, dtype, j) - m) / T);
+                    if (w > 0.0) last = j;
+                    lo = c;
+                    c += w;
+                    if (c > target) pick = j;
+                }
+                if (pick < 0) { pick = last; }
+                drawn = (int32_t)pick;
+                double d0 = (target - lo) / W, d1 = (c - target) / W;
+                mg_draw = d0 < d1 ? d0 : d1;
+            }
+        }
+        otok[a] = drawn;
+        accept_len[b] = a; out_len[b] = a + 1;
+        if (status) status[b] = bad_dist ? 4 : 0;
+        if (margin) { margin[2 * b] = mg_test; margin[2 * b + 1] = mg_draw; }
     }
 }

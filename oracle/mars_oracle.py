@@ -71,6 +71,9 @@ def lib() -> ctypes.CDLL:
             L.mars_oracle_histograms.restype = None
             L.mars_oracle_topk.argtypes = [vp, i32, i64, i64, i64, i32, vp, vp]
             L.mars_oracle_topk.restype = None
+            L.mars_oracle_verify_tree_stochastic.argtypes = [vp, i32, i64, vp, vp, vp, i32, i32, i64, f64,
+                                                             f64, u32, i32] + [vp] * 8
+            L.mars_oracle_verify_tree_stochastic.restype = None
             _lib = L
     return _lib
 
@@ -241,3 +244,45 @@ def topk(logits: np.ndarray, k: int, V: int | None = None):
     idx = np.empty((R, k), np.int32)
     lib().mars_oracle_topk(_p(logits), dt, ld, R, V, int(k), _p(val), _p(idx))
     return val, idx
+
+
+STOCH_PLAIN = 32
+STOCH_RELAX_ONLY = 64
+
+
+def verify_tree_stochastic(logits, tok, parent, uniform, theta, temperature, flags: int = 0,
+                           Dcap: int | None = None, V: int | None = None) -> dict:
+    """Stochastic (T > 0) tree verification; see the block comment in mars_oracle.c.
+    ``uniform`` is float32 [B, N]: [b, i>0] judges node i, [b, 0] draws the final token."""
+    dt, V = _check_logits(logits, V)
+    tok = np.ascontiguousarray(tok, np.int32)
+    parent = np.ascontiguousarray(parent, np.int32)
+    uniform = np.ascontiguousarray(uniform, np.float32)
+    B, N = tok.shape
+    if parent.ndim == 1:
+        flags |= SHARED_PARENT
+    if logits.shape[0] != B * N or parent.shape[-1] != N or uniform.shape != (B, N):
+        raise ValueError("shape mismatch")
+    if not (temperature > 0 and np.isfinite(temperature)):
+        raise ValueError("temperature must be positive and finite")
+    if N > 1024:
+        raise ValueError("N <= 1024")
+    if Dcap is None:
+        Dcap = N - 1
+    out = {
+        "accept_len": np.empty(B, np.int32),
+        "out_tokens": np.empty((B, Dcap + 1), np.int32),
+        "path_nodes": np.empty((B, Dcap + 1), np.int32),
+        "out_len": np.empty(B, np.int32),
+        "seq_status": np.empty(B, np.int32),
+        "node_prob": np.empty((B, N), np.float64),
+        "node_how": np.empty((B, N), np.uint8),
+        "margin": np.empty((B, 2), np.float64),
+    }
+    L = lib()
+    L.mars_oracle_verify_tree_stochastic(
+        _p(logits), dt, logits.shape[1], _p(tok), _p(parent), _p(uniform), B, N, V, float(theta),
+        float(temperature), flags, Dcap, _p(out["accept_len"]), _p(out["out_tokens"]),
+        _p(out["path_nodes"]), _p(out["out_len"]), _p(out["seq_status"]), _p(out["node_prob"]),
+        _p(out["node_how"]), _p(out["margin"]))
+    return out
