@@ -65,6 +65,12 @@ typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
 #define MARS_RULE_PROB_RATIO 16u /* relax iff p2/p1 = exp(z2 - z1) > theta; evaluated as
                                     z1 - z2 < (float)(-ln(theta)), theta <= 0 always relaxes  */
 
+/* Stochastic verification only (mars_verify_tree_stochastic / _chain_stochastic): how the margin
+ * rule composes with the acceptance test of Eq. 1.  With neither bit a child that passes the
+ * three-way rule is accepted outright and the others take the Eq. 1 test.  Mutually exclusive. */
+#define MARS_STOCH_PLAIN 32u      /* Eq. 1 alone: standard speculative sampling, no relaxation  */
+#define MARS_STOCH_RELAX_ONLY 64u /* Eq. 1, plus the relaxed runner-up (top-1 is not automatic)  */
+
 #define MARS_MAX_NODES 1024   /* cap on N (rows per sequence)                                 */
 
 /* per-sequence status values written to seq_status */
@@ -72,6 +78,8 @@ typedef enum { MARS_BF16 = 0, MARS_FP32 = 1 } mars_dtype_t;
 #define MARS_SEQ_BAD_TREE 1   /* parent[0] != -1, or for i>0 parent[i] >= i or parent[i] < -1 */
 #define MARS_SEQ_DEPTH_CAP 2  /* the accepted path is deeper than Dcap                          */
 #define MARS_SEQ_TIMEOUT 3    /* a bounded device-side wait gave up (mars_lmhead_verify only)  */
+#define MARS_SEQ_BAD_DISTRIBUTION 4 /* stochastic calls: a row on the walk has no softmax (its
+                                       maximum is not finite) or its residual has no mass      */
 
 /* Optional extra outputs; the struct lives in HOST memory, its members are device
  * pointers, any of which may be NULL. */
@@ -276,6 +284,69 @@ mars_status_t mars_verify_records(const void *records, int G, const int32_t *tok
                                   int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
                                   int32_t *out_len, int Dcap, int32_t *seq_status,
                                   const mars_debug_out_t *dbg, void *cuda_stream);
+
+/*
+ * Stochastic (temperature T > 0) verification of token trees.
+ *
+ * From the paper: Sec. 2.2 -- a drafted token is accepted with probability
+ * min(1, P_target / P_draft) (Eq. 1), a rejection draws the corrected token from the residual
+ * distribution, tree-based methods apply the same logic to a token tree, and MARS "modifies only
+ * the accept/reject decision" and applies on top of sampling-based verification; Eq. 3 -- P is
+ * the softmax of the logits; Sec. 4.1 -- draft trees are top-k expansions.  The paper does not
+ * say how the relaxation composes with Eq. 1; the reading implemented here:
+ *
+ *   - P(v) = softmax(z / T)(v) of a row; NaN logits count as -inf.
+ *   - Candidates are deterministic, so the draft distribution at a node is a point mass and
+ *     Eq. 1 reads "accept x with probability P(x)".  Starting at the root, the children of the
+ *     current node are tried in node order against the current node's row.  A child x is
+ *     accepted iff the composition mode accepts it outright (default: x is the row's top-1, or
+ *     its runner-up with r > theta -- the three-way rule of Sec. 3.4; see MARS_STOCH_*), or
+ *     uniform[b, child] * rem < e_x, where e_x = exp((z_x - max z) / T) and rem is the
+ *     unnormalised mass left after removing the siblings rejected so far (the residual of a
+ *     point-mass draft is P without that token, renormalised).  The first accepted child
+ *     becomes the current node; a repeated sibling token has no mass left.
+ *   - When no child is accepted (or the node is a leaf) the next token is drawn from the
+ *     residual of the current node's row by inverting its CDF in token-id order with
+ *     uniform[b, 0]: the smallest id j with (sum of residual weights of ids <= j) > u * W.
+ *   - Arithmetic is fp32 (2^x by the hardware approximation): probabilities carry a relative
+ *     error of order 1e-6, so a decision can differ from an exact evaluation only when
+ *     |e_x - u * rem| or the distance of u * W to a CDF step is that small relative to the
+ *     row's total mass.
+ *
+ *   logits, tok, parent, B, N, V, theta, Dcap, accept_len, out_tokens, path_nodes, out_len:
+ *              as mars_verify_tree; out_tokens[b, a] is the drawn token.
+ *   uniform    float [B, N], values in [0, 1): [b, i] judges node i (i > 0), [b, 0] draws the
+ *              next token.  Supplied by the caller, so results are reproducible.
+ *   temperature T > 0, finite.
+ *   flags      MARS_SIGN_LITERAL, MARS_SHARED_PARENT, MARS_RULE_*, MARS_STOCH_*.
+ *   seq_status MARS_SEQ_BAD_TREE / MARS_SEQ_DEPTH_CAP: safe output as mars_verify_tree (accept
+ *              nothing, emit the root row's top-1).  MARS_SEQ_BAD_DISTRIBUTION: the path so far
+ *              is kept and the top-1 of the row where the walk stopped is emitted.
+ *   node_prob  float [B, N] or NULL: softmax probability of tok[b, i] under its parent's row
+ *              (nothing removed); 0 for the root, absent nodes and ids outside [0, V).
+ *   node_how   uint8 [B, N] or NULL: 0 not visited, 1 exact match, 2 relaxed runner-up,
+ *              3 accepted by Eq. 1, 4 rejected.
+ *   workspace  mars_stochastic_workspace_bytes(B, N, V, dt) bytes, 256-byte aligned; contents
+ *              need not be initialised.  Two kernels are enqueued; nothing is allocated.
+ *
+ * mars_verify_chain_stochastic is the chain form (K rows, K-1 drafts, uniform [B, K] with
+ * [b, i] judging draft i-1 and [b, 0] drawing the correction or bonus token).
+ */
+size_t mars_stochastic_workspace_bytes(int B, int N, int V, mars_dtype_t dt);
+mars_status_t mars_verify_tree_stochastic(const void *logits, int64_t ld, mars_dtype_t dt,
+                                          const int32_t *tok, const int32_t *parent,
+                                          const float *uniform, int B, int N, int V, float theta,
+                                          float temperature, uint32_t flags, int32_t *accept_len,
+                                          int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len,
+                                          int Dcap, int32_t *seq_status, float *node_prob,
+                                          uint8_t *node_how, void *workspace, size_t workspace_bytes,
+                                          void *cuda_stream);
+mars_status_t mars_verify_chain_stochastic(const void *logits, int64_t ld, mars_dtype_t dt,
+                                           const int32_t *draft, const float *uniform, int B, int K,
+                                           int V, float theta, float temperature, uint32_t flags,
+                                           int32_t *accept_len, int32_t *out_tokens, int32_t *out_len,
+                                           int32_t *seq_status, float *node_prob, uint8_t *node_how,
+                                           void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * mars_verify_tree for callers that must not allocate device memory.  (The paper has no

@@ -1,0 +1,637 @@
+// libmars: stochastic (temperature T > 0) verification.
+//
+// Sec. 2.2 of the paper: a drafted token is accepted with probability min(1, P_target/P_draft)
+// (Eq. 1), a rejection draws the correction from the residual distribution, and tree methods
+// apply the same logic to a token tree; P is the softmax of the logits (Eq. 3).  Draft trees are
+// top-k expansions (Sec. 4.1), so a candidate's draft distribution is a point mass and Eq. 1
+// reads "accept x with probability P(x)" under the running residual (P with the rejected
+// siblings removed).  How the margin rule composes with Eq. 1 is a reading of this library,
+// selected by flags (see mars.h).
+//
+// Two kernels per call:
+//
+//   stoch_stream_kernel   one pass over every logits row, as in the deterministic path (16-byte
+//       streaming loads, filtered exact top-2 in registers), that also accumulates the softmax
+//       denominator online: every thread keeps a reference `ref` (its largest batch maximum
+//       times c = log2(e)/T) and sum = SUM 2^(z*c - ref); the reference only moves when a
+//       batch maximum exceeds it, which the top-2 filter computes anyway.  One 32-byte record
+//       {z1, id1, z2, id2, ref, sum} per slice.
+//   stoch_tail_kernel     one block per sequence: merges slice records, gathers the logit of
+//       every node's token from its parent's row (one scalar load per node, all in parallel),
+//       walks the tree (Eq. 1 on the running residual, or the margin rule), then draws the next
+//       token from the residual of the row where the walk stopped by inverting its CDF in
+//       token-id order: the row is summed by contiguous warp segments, the segment holding
+//       u*W is split again, and so on down to one 32-lane tile and one element (partial sums
+//       and the running target in fp64, so that the pick depends on the weights alone).
+#include "mars_top2_stream.cuh"
+
+#include <cmath>
+
+#include "mars.h"
+
+namespace mars {
+
+struct __align__(16) SRec {
+    float z1; int id1; float z2; int id2;
+    float ref;   // scaled reference: weights are 2^(z*c - ref)
+    float sum;   // SUM of those weights over the slice
+    int pad0, pad1;
+};
+
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// (ref, sum) of the union of two disjoint element sets.
+__device__ __forceinline__ void soft_merge(float &ref, float &sum, float ref_b, float sum_b)
+{
+    const float r = fmaxf(ref, ref_b);
+    if (r == -INFINITY) { ref = r; sum = 0.0f; return; }
+    sum = sum * ex2f(ref - r) + sum_b * ex2f(ref_b - r);
+    ref = r;
+}
+
+// One element joins (ref, sum); NaN counts as -inf (weight 0), +inf makes the sum infinite.
+__device__ __forceinline__ void soft_add_scalar(float &ref, float &sum, float x, float c)
+{
+    if (!(x == x)) return;
+    const float xc = x * c;
+    if (xc > ref) { sum *= ex2f(ref - xc); ref = xc; }
+    if (ref > -INFINITY) {
+        const float t = fmaf(x, c, -ref);
+        sum += (t == t) ? ex2f(t) : INFINITY;
+    }
+}
+
+// NaN -> -inf on the packed representation (one instruction per 16-byte word pair for bf16).
+template <int DT> __device__ __forceinline__ uint4 nan_to_neg_inf(const uint4 &v);
+template <> __device__ __forceinline__ uint4 nan_to_neg_inf<MARS_BF16>(const uint4 &v)
+{
+    return make_uint4(bmax2(v.x, 0xff80ff80u), bmax2(v.y, 0xff80ff80u), bmax2(v.z, 0xff80ff80u),
+                      bmax2(v.w, 0xff80ff80u));
+}
+template <> __device__ __forceinline__ uint4 nan_to_neg_inf<MARS_FP32>(const uint4 &v)
+{
+    return make_uint4(__float_as_uint(fmaxf(__uint_as_float(v.x), -INFINITY)),
+                      __float_as_uint(fmaxf(__uint_as_float(v.y), -INFINITY)),
+                      __float_as_uint(fmaxf(__uint_as_float(v.z), -INFINITY)),
+                      __float_as_uint(fmaxf(__uint_as_float(v.w), -INFINITY)));
+}
+
+// A batch joins (ref, sum).  bm is the batch maximum (NaN operands ignored by the packed max).
+// NaN logits are mapped to -inf (weight 0) before the exponential; a +inf logit makes the
+// reference infinite and the sum NaN or infinite, which the tail reports as a row without a
+// distribution.
+template <int DT, int U>
+__device__ __forceinline__ void soft_batch(const uint4 (&v)[U], float bm, float c, float &ref, float &sum)
+{
+    typedef Elem<DT> E;
+    const float bmc = bm * c;
+    if (bmc > ref) { sum *= ex2f(ref - bmc); ref = bmc; }
+    if (!(ref > -INFINITY)) return;          // nothing above -inf seen so far: all weights are 0
+    const float nref = -ref;
+    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint4 w = nan_to_neg_inf<DT>(v[u]);
+#pragma unroll
+        for (int k = 0; k < E::kVec; k += 4) {
+            a0 += ex2f(fmaf(E::elem(w, k + 0), c, nref));
+            a1 += ex2f(fmaf(E::elem(w, k + 1), c, nref));
+            a2 += ex2f(fmaf(E::elem(w, k + 2), c, nref));
+            a3 += ex2f(fmaf(E::elem(w, k + 3), c, nref));
+        }
+    }
+    sum += (a0 + a1) + (a2 + a3);
+}
+
+struct StreamParams {
+    const void *logits;
+    long long ld;
+    int V;
+    int S;       // slices per row
+    int L;       // elements per slice (multiple of 16)
+    float c;     // log2(e) / T
+    SRec *partial;   // [R*S]
+};
+
+template <int DT, int U, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const StreamParams p)
+{
+    typedef Elem<DT> E;
+    __shared__ unsigned sT[2];
+    __shared__ Rec s_warp[kThreads / 32];
+    __shared__ float2 s_soft[kThreads / 32];
+
+    const int tid = threadIdx.x;
+    const long long blk = blockIdx.x;
+    const long long row = blk / p.S;
+    const int slice = (int)(blk - row * p.S);
+    const float c = p.c;
+
+    const int lo = slice * p.L;
+    const int hi = min(p.V, lo + p.L);
+    const char *rowp = (const char *)p.logits + (size_t)row * (size_t)p.ld * E::kBytes;
+
+    // [lo, hi) = head scalars | 16-byte vectors | tail scalars
+    const uintptr_t a0 = (uintptr_t)(rowp + (size_t)lo * E::kBytes);
+    int nhead = (int)(((16 - (a0 & 15)) & 15) / E::kBytes);
+    nhead = min(nhead, max(hi - lo, 0));
+    const int vlo = lo + nhead;
+    const int nvec = max(hi - vlo, 0) / E::kVec;
+    const int tlo = vlo + nvec * E::kVec;
+    const int ntail = max(hi - tlo, 0);
+    const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
+
+    constexpr int kBatchVecs = kThreads * U;
+    const int nfull = nvec / kBatchVecs;
+    uint4 v[U];
+    typename E::packed_t q[U];
+
+    float bm = (nfull > 0) ? load_batch<DT, U, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, U, true>(vbase, tid, nvec, v, q);
+    if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
+    __syncthreads();
+
+    Rec s = empty_rec();
+    float ref = -INFINITY, sum = 0.0f;
+    if (tid < nhead) {
+        const float x = E::scalar(rowp, lo + tid);
+        insert<false>(s, x, lo + tid, sT);
+        soft_add_scalar(ref, sum, x, c);
+    }
+    {   // bootstrap of the shared runner-up bound from the first batch's maxima
+        float a1 = (bm == bm) ? bm : -INFINITY, a2 = -INFINITY;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            float b1 = __shfl_xor_sync(0xffffffffu, a1, m), b2 = __shfl_xor_sync(0xffffffffu, a2, m);
+            a2 = fmaxf(fminf(a1, b1), fmaxf(a2, b2));
+            a1 = fmaxf(a1, b1);
+        }
+        if ((tid & 31) == 0) { publish(sT, a1); publish(sT, a2); }
+        __syncwarp();
+    }
+    float T2 = dec(*(volatile unsigned *)&sT[1]);
+    soft_batch<DT, U>(v, bm, c, ref, sum);
+    process_batch<DT, U, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
+
+    for (int bi = 1; bi < nfull; ++bi) {
+        bm = load_batch<DT, U, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
+        T2 = dec(*(volatile unsigned *)&sT[1]);
+        soft_batch<DT, U>(v, bm, c, ref, sum);
+        process_batch<DT, U, true>(v, q, bm, T2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
+    }
+    if (nfull > 0 && nfull * kBatchVecs < nvec) {
+        bm = load_batch<DT, U, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        T2 = dec(*(volatile unsigned *)&sT[1]);
+        soft_batch<DT, U>(v, bm, c, ref, sum);
+        process_batch<DT, U, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
+    }
+    if (tid < ntail) {
+        const float x = E::scalar(rowp, tlo + tid);
+        insert<false>(s, x, tlo + tid, sT);
+        soft_add_scalar(ref, sum, x, c);
+    }
+
+    // ---- block merge: top-2 under the total order, (ref, sum) by rescaling ----
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        s = merge(s, shfl_xor_rec(s, m));
+        const float rb = __shfl_xor_sync(0xffffffffu, ref, m), sb = __shfl_xor_sync(0xffffffffu, sum, m);
+        soft_merge(ref, sum, rb, sb);
+    }
+    if ((tid & 31) == 0) { s_warp[tid >> 5] = s; s_soft[tid >> 5] = make_float2(ref, sum); }
+    __syncthreads();
+    if (tid == 0) {
+        Rec r = s_warp[0];
+        float rr = s_soft[0].x, ss = s_soft[0].y;
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) {
+            r = merge(r, s_warp[w]);
+            soft_merge(rr, ss, s_soft[w].x, s_soft[w].y);
+        }
+        SRec o;
+        o.z1 = r.z1; o.id1 = r.id1; o.z2 = r.z2; o.id2 = r.id2; o.ref = rr; o.sum = ss; o.pad0 = 0; o.pad1 = 0;
+        p.partial[blk] = o;
+    }
+}
+
+// ------------------------------------------------------------------------------- tail
+
+constexpr int kTailThreads = 512;
+constexpr int kTailWarps = kTailThreads / 32;
+
+struct StochTailParams {
+    const void *logits;
+    long long ld;
+    int V, N, S;
+    float c, theta;
+    uint32_t flags;
+    int chain;
+    int Dcap;
+    const SRec *partial;     // [B*N*S]
+    const int32_t *tok;      // tree [B,N]; chain: draft [B,N-1]
+    const int32_t *parent;   // tree [B,N] or [N]
+    const float *uniform;    // [B,N]
+    int32_t *accept_len, *out_tokens, *path_nodes, *out_len, *seq_status;
+    float *node_prob;        // [B,N] or null
+    uint8_t *node_how;       // [B,N] or null
+};
+
+__host__ __device__ inline size_t stoch_tail_smem_bytes(int N)
+{
+    return (size_t)N * (9 * 4 + 2) + 64;
+}
+
+// Weights 2^(z*c - ref) of the kVec elements that `lane` owns in 32-lane tile `tile` of a row
+// (element j0 = (tile*32 + lane)*kVec onwards), zero beyond V and for removed tokens.
+template <int DT>
+__device__ __forceinline__ void tile_weights(const char *rowp, bool aligned, int V, long long tile, int lane,
+                                             float c, float nref, const int32_t *removed, int nrem,
+                                             float (&w)[Elem<DT>::kVec])
+{
+    typedef Elem<DT> E;
+    const long long j0 = (tile * 32 + lane) * E::kVec;
+    if (aligned && j0 + E::kVec <= V) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)j0 * E::kBytes));
+#pragma unroll
+        for (int k = 0; k < E::kVec; ++k) w[k] = E::elem(v, k);
+    } else {
+#pragma unroll
+        for (int k = 0; k < E::kVec; ++k) w[k] = (j0 + k < V) ? E::scalar(rowp, (int)(j0 + k)) : -INFINITY;
+    }
+#pragma unroll
+    for (int k = 0; k < E::kVec; ++k) {
+        const float x = w[k];
+        const float t = fmaf(x, c, nref);
+        w[k] = (x == x && t == t) ? ex2f(t) : 0.0f;
+    }
+    for (int r = 0; r < nrem; ++r) {
+        const long long d = (long long)removed[r] - j0;
+        if (d >= 0 && d < E::kVec) {
+#pragma unroll
+            for (int k = 0; k < E::kVec; ++k) if (k == (int)d) w[k] = 0.0f;
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kTailThreads, 1) stoch_tail_kernel(const StochTailParams p)
+{
+    typedef Elem<DT> E;
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    const int N = p.N, V = p.V, S = p.S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x;
+
+    int32_t *s_id1 = reinterpret_cast<int32_t *>(smem_dyn);
+    int32_t *s_id2 = s_id1 + N;
+    int32_t *s_par = s_id2 + N;
+    int32_t *s_tok = s_par + N;
+    int32_t *s_removed = s_tok + N;
+    float *s_ref = reinterpret_cast<float *>(s_removed + N);
+    float *s_sum = s_ref + N;
+    float *s_e = s_sum + N;
+    float *s_u = s_e + N;
+    unsigned char *s_relax = reinterpret_cast<unsigned char *>(s_u + N);
+    unsigned char *s_how = s_relax + N;
+
+    __shared__ double s_part[kTailWarps];
+    __shared__ int s_ctl[8];     // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token
+    __shared__ double s_target;
+    __shared__ long long s_range[2];
+
+    const int32_t *par_g = p.chain ? nullptr : ((p.flags & MARS_SHARED_PARENT) ? p.parent : p.parent + (size_t)b * N);
+    int bad = 0;
+    for (int i = tid; i < N; i += kTailThreads) {
+        // merge the row's slice records
+        const SRec *src = p.partial + ((size_t)b * N + i) * S;
+        Rec acc = empty_rec();
+        float ref = -INFINITY, sum = 0.0f;
+        for (int k = 0; k < S; ++k) {
+            const int4 a = __ldcg(reinterpret_cast<const int4 *>(src + k));
+            const int4 bq = __ldcg(reinterpret_cast<const int4 *>(src + k) + 1);
+            Rec r;
+            r.z1 = __int_as_float(a.x); r.id1 = a.y; r.z2 = __int_as_float(a.z); r.id2 = a.w;
+            acc = merge(acc, r);
+            soft_merge(ref, sum, __int_as_float(bq.x), __int_as_float(bq.y));
+        }
+        acc = finish_record(acc);
+        s_id1[i] = acc.id1;
+        s_id2[i] = acc.id2;
+        s_relax[i] = relax_bit(acc.z1, acc.z2, p.theta, p.flags) ? 1 : 0;
+        s_ref[i] = ref;
+        s_sum[i] = sum;
+        int pa, tk;
+        if (p.chain) {
+            pa = i - 1;
+            tk = i > 0 ? p.tok[(size_t)b * (N - 1) + (i - 1)] : -1;
+        } else {
+            pa = par_g[i];
+            tk = p.tok[(size_t)b * N + i];
+            if (i == 0 ? (pa != -1) : (pa >= i || pa < -1)) bad = 1;
+        }
+        s_par[i] = pa;
+        s_tok[i] = tk;
+        s_u[i] = p.uniform[(size_t)b * N + i];
+        s_how[i] = 0;
+    }
+    bad = __syncthreads_or(bad);
+
+    // every node's token under its parent's row: unnormalised mass, plain softmax probability
+    for (int i = tid; i < N; i += kTailThreads) {
+        float e = 0.0f, prob = 0.0f;
+        const int pa = s_par[i], tk = s_tok[i];
+        if (!bad && i > 0 && pa >= 0 && tk >= 0 && tk < V) {
+            const float ref = s_ref[pa], sum = s_sum[pa];
+            if (ref > -INFINITY && ref < INFINITY && sum > 0.0f && sum < INFINITY) {
+                const char *rowp = (const char *)p.logits + ((size_t)b * N + pa) * (size_t)p.ld * E::kBytes;
+                const float x = E::scalar(rowp, tk);
+                const float t = fmaf(x, p.c, -ref);
+                e = (x == x && t == t) ? ex2f(t) : 0.0f;
+                prob = __fdiv_rn(e, sum);
+            }
+        }
+        s_e[i] = e;
+        if (p.node_prob) p.node_prob[(size_t)b * N + i] = prob;
+    }
+    __syncthreads();
+
+    // ---- the walk (one thread; at most N node visits) ----
+    if (tid == 0) {
+        int cur = 0, a = 0, status = bad ? 1 : 0, nrem = 0, draw = 0;
+        const int W = p.Dcap + 1;
+        int32_t *o_tok = p.out_tokens + (size_t)b * W;
+        int32_t *o_path = p.path_nodes ? p.path_nodes + (size_t)b * W : nullptr;
+        for (int k = 0; k < W; ++k) { o_tok[k] = -1; if (o_path) o_path[k] = -1; }
+        if (o_path) o_path[0] = 0;
+        while (status == 0) {
+            const float ref = s_ref[cur], sum = s_sum[cur];
+            nrem = 0;
+            if (!(ref > -INFINITY && ref < INFINITY && sum > 0.0f && sum < INFINITY)) { status = 4; break; }
+            float rem = sum;
+            int next = -1;
+            for (int i = cur + 1; i < N && next < 0; ++i) {
+                if (s_par[i] != cur || s_tok[i] < 0) continue;
+                const int x = s_tok[i];
+                bool gone = false;
+                for (int k = 0; k < nrem; ++k) gone |= (s_removed[k] == x);
+                const float ex = gone ? 0.0f : s_e[i];
+                int how = 0;
+                if (!(p.flags & MARS_STOCH_PLAIN)) {
+                    if (x == s_id1[cur]) how = (p.flags & MARS_STOCH_RELAX_ONLY) ? 0 : 1;
+                    else if (x == s_id2[cur] && s_relax[cur]) how = 2;
+                }
+                if (how == 0) how = (__fmul_rn(s_u[i], rem) < ex) ? 3 : 4;   // Eq. 1 on the running residual
+                s_how[i] = (unsigned char)how;
+                if (how == 4) {
+                    if (ex > 0.0f) { rem = fmaxf(__fsub_rn(rem, ex), 0.0f); s_removed[nrem++] = x; }
+                } else next = i;
+            }
+            if (next < 0) { draw = 1; break; }
+            cur = next; ++a;
+            if (a <= p.Dcap) { o_tok[a - 1] = s_tok[cur]; if (o_path) o_path[a] = cur; }
+        }
+        if ((status == 0 || status == 4) && a > p.Dcap) status = 2;
+        if (status == 1 || status == 2) {
+            for (int k = 0; k < W; ++k) { o_tok[k] = -1; if (o_path) o_path[k] = -1; }
+            if (o_path) o_path[0] = 0;
+            for (int i = 0; i < N; ++i) s_how[i] = 0;
+            cur = 0; a = 0; draw = 0; nrem = 0;
+        }
+        s_ctl[0] = cur; s_ctl[1] = a; s_ctl[2] = status; s_ctl[3] = nrem; s_ctl[4] = draw;
+        s_ctl[5] = s_id1[cur];
+    }
+    __syncthreads();
+
+    // ---- the next token: CDF inversion over the residual of row `cur` ----
+    const int cur = s_ctl[0];
+    if (s_ctl[4]) {
+        const int nrem = s_ctl[3];
+        const char *rowp = (const char *)p.logits + ((size_t)b * N + cur) * (size_t)p.ld * E::kBytes;
+        const bool aligned = (((uintptr_t)rowp) & 15) == 0;
+        const float nref = -s_ref[cur];
+        const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
+        long long t0 = 0, t1 = ntiles;
+        bool first = true, ok = true;
+        while (t1 - t0 > 1) {
+            const long long len = (t1 - t0 + kTailWarps - 1) / kTailWarps;
+            const long long w0 = min(t1, t0 + warp * len), w1 = min(t1, w0 + len);
+            double acc = 0.0;
+            for (long long t = w0; t < w1; ++t) {
+                float w[E::kVec];
+                tile_weights<DT>(rowp, aligned, V, t, lane, p.c, nref, s_removed, nrem, w);
+                float ls = 0.0f;
+#pragma unroll
+                for (int k = 0; k < E::kVec; ++k) ls += w[k];
+                acc += (double)ls;
+            }
+#pragma unroll
+            for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+            if (lane == 0) s_part[warp] = acc;
+            __syncthreads();
+            if (tid == 0) {
+                double target;
+                bool good = true;
+                if (first) {
+                    double Wt = 0.0;
+                    for (int k = 0; k < kTailWarps; ++k) Wt += s_part[k];
+                    good = (Wt > 0.0 && Wt < (double)INFINITY);
+                    target = (double)s_u[0] * Wt;
+                } else target = s_target;
+                int pick = -1, lastpos = -1;
+                double cum = 0.0, before = 0.0;
+                for (int k = 0; k < kTailWarps && pick < 0; ++k) {
+                    if (s_part[k] > 0.0) lastpos = k;
+                    before = cum;
+                    cum += s_part[k];
+                    if (cum > target) pick = k;
+                }
+                if (pick < 0) {   // rounding pushed the target past the total: the last part with mass
+                    pick = lastpos;
+                    before = 0.0;
+                    for (int k = 0; k < pick; ++k) before += s_part[k];
+                }
+                if (!good || pick < 0) { s_ctl[2] = 4; s_range[0] = 0; s_range[1] = 0; }
+                else {
+                    s_target = fmax(target - before, 0.0);
+                    s_range[0] = min(t1, t0 + pick * len);
+                    s_range[1] = min(t1, s_range[0] + len);
+                }
+            }
+            __syncthreads();
+            t0 = s_range[0]; t1 = s_range[1];
+            first = false;
+            if (t1 <= t0) { ok = false; break; }
+        }
+        if (ok && warp == 0) {
+            // one tile left: lane prefix, then the element inside the lane
+            float w[E::kVec];
+            tile_weights<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem, w);
+            double ls = 0.0;
+#pragma unroll
+            for (int k = 0; k < E::kVec; ++k) ls += (double)w[k];
+            double inc = ls;
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const double o = __shfl_up_sync(0xffffffffu, inc, m);
+                if (lane >= m) inc += o;
+            }
+            const double total = __shfl_sync(0xffffffffu, inc, 31);
+            double target;
+            bool good = true;
+            if (first) {   // the whole row is one tile
+                good = (total > 0.0 && total < (double)INFINITY);
+                target = (double)s_u[0] * total;
+            } else target = s_target;
+            const unsigned hit = __ballot_sync(0xffffffffu, inc > target);
+            const unsigned pos = __ballot_sync(0xffffffffu, ls > 0.0);
+            int src = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
+            if (!good || src < 0) { if (lane == 0) s_ctl[2] = 4; }
+            else if (lane == src) {
+                const double tl = fmax(target - (inc - ls), 0.0);
+                int pick = -1, lastpos = -1;
+                double cum = 0.0;
+#pragma unroll
+                for (int k = 0; k < E::kVec; ++k) {
+                    if (w[k] > 0.0f) lastpos = k;
+                    cum += (double)w[k];
+                    if (pick < 0 && cum > tl) pick = k;
+                }
+                if (pick < 0) pick = lastpos;
+                s_ctl[5] = (int)((t0 * 32 + lane) * E::kVec) + pick;
+            }
+        }
+        __syncthreads();
+    }
+
+    if (tid == 0) {
+        const int a = s_ctl[1], status = s_ctl[2];
+        p.out_tokens[(size_t)b * (p.Dcap + 1) + a] = (status == 4) ? s_id1[cur] : s_ctl[5];
+        p.accept_len[b] = a;
+        p.out_len[b] = a + 1;
+        if (p.seq_status) p.seq_status[b] = status;
+    }
+    if (p.node_how)
+        for (int i = tid; i < N; i += kTailThreads) p.node_how[(size_t)b * N + i] = s_how[i];
+}
+
+// ------------------------------------------------------------------------------- host
+
+static size_t stoch_ws_bytes(long long R, int S) { return ((size_t)R * S * sizeof(SRec) + 255) / 256 * 256; }
+
+static bool stoch_sizes_supported(int B, int N, int V, int dt)
+{
+    if (B < 1 || N < 1 || V < 2) return false;
+    if (dt != MARS_BF16 && dt != MARS_FP32) return false;
+    if (N > MARS_MAX_NODES || V > (1 << 30)) return false;
+    if ((long long)B * N > (1ll << 40)) return false;
+    return true;
+}
+
+static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
+                                    const int32_t *parent, const float *uniform, int chain, int B, int N,
+                                    int V, float theta, float temperature, uint32_t flags,
+                                    int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
+                                    int32_t *out_len, int Dcap, int32_t *seq_status, float *node_prob,
+                                    uint8_t *node_how, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream)
+{
+    if (B < 1 || N < 1 || V < 2 || !logits || !uniform) return MARS_ERR_INVALID_ARG;
+    if (ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !(temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
+    if (!accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
+    if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
+    if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO |
+                  MARS_STOCH_PLAIN | MARS_STOCH_RELAX_ONLY))
+        return MARS_ERR_UNSUPPORTED;
+    if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
+    if ((flags & MARS_STOCH_PLAIN) && (flags & MARS_STOCH_RELAX_ONLY)) return MARS_ERR_INVALID_ARG;
+    rule_threshold(&theta, &flags);
+    if (!stoch_sizes_supported(B, N, V, (int)dt)) return MARS_ERR_UNSUPPORTED;
+    const int es = dt == MARS_BF16 ? 2 : 4;
+    if ((uintptr_t)logits % es) return MARS_ERR_INVALID_ARG;
+    const double cd = 1.4426950408889634074 / (double)temperature;   // log2(e) / T
+    if (!(cd < 3.0e38)) return MARS_ERR_INVALID_ARG;
+    const long long R = (long long)B * N;
+    const Split sp = choose_split(R, V, (int)dt);
+    if (R * sp.S > 0x7fffffffll) return MARS_ERR_UNSUPPORTED;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < stoch_ws_bytes(R, sp.S))
+        return MARS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    StreamParams sp1;
+    sp1.logits = logits; sp1.ld = ld; sp1.V = V; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
+    sp1.partial = (SRec *)workspace;
+    const unsigned grid = (unsigned)(R * sp.S);
+    // Launch shape: bf16 is bound by the exponential unit and runs best with short batches and
+    // many resident warps (4 vectors per batch, 6 blocks per SM); fp32 has half the elements
+    // per byte and keeps the deterministic path's shape (8 vectors, 4 blocks per SM).
+    // MARS_STOCH_VARIANT (test / tuning hook) forces one of the four instantiations.
+    const char *var = getenv("MARS_STOCH_VARIANT");
+    const int variant = var ? atoi(var) : (dt == MARS_BF16 ? 3 : 1);
+#define MARS_STOCH_LAUNCH(DT)                                                                    \
+    switch (variant) {                                                                           \
+    case 0: stoch_stream_kernel<DT, 8, 3><<<grid, kThreads, 0, st>>>(sp1); break;                \
+    case 1: stoch_stream_kernel<DT, 8, 4><<<grid, kThreads, 0, st>>>(sp1); break;                \
+    case 2: stoch_stream_kernel<DT, 4, 4><<<grid, kThreads, 0, st>>>(sp1); break;                \
+    default: stoch_stream_kernel<DT, 4, 6><<<grid, kThreads, 0, st>>>(sp1); break;               \
+    }
+    if (dt == MARS_BF16) { MARS_STOCH_LAUNCH(MARS_BF16) } else { MARS_STOCH_LAUNCH(MARS_FP32) }
+#undef MARS_STOCH_LAUNCH
+    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+
+    StochTailParams tp;
+    tp.logits = logits; tp.ld = ld; tp.V = V; tp.N = N; tp.S = sp.S; tp.c = (float)cd; tp.theta = theta;
+    tp.flags = flags; tp.chain = chain; tp.Dcap = Dcap; tp.partial = (const SRec *)workspace;
+    tp.tok = tok; tp.parent = parent; tp.uniform = uniform;
+    tp.accept_len = accept_len; tp.out_tokens = out_tokens; tp.path_nodes = path_nodes;
+    tp.out_len = out_len; tp.seq_status = seq_status; tp.node_prob = node_prob; tp.node_how = node_how;
+    const size_t smem = stoch_tail_smem_bytes(N);
+    if (dt == MARS_BF16) stoch_tail_kernel<MARS_BF16><<<(unsigned)B, kTailThreads, smem, st>>>(tp);
+    else stoch_tail_kernel<MARS_FP32><<<(unsigned)B, kTailThreads, smem, st>>>(tp);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+}
+
+}  // namespace mars
+
+extern "C" {
+
+size_t mars_stochastic_workspace_bytes(int B, int N, int V, mars_dtype_t dt)
+{
+    if (!mars::stoch_sizes_supported(B, N, V, (int)dt)) return 0;
+    const long long R = (long long)B * N;
+    return mars::stoch_ws_bytes(R, mars::choose_split(R, V, (int)dt).S);
+}
+
+mars_status_t mars_verify_tree_stochastic(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
+                                          const int32_t *parent, const float *uniform, int B, int N, int V,
+                                          float theta, float temperature, uint32_t flags,
+                                          int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
+                                          int32_t *out_len, int Dcap, int32_t *seq_status, float *node_prob,
+                                          uint8_t *node_how, void *workspace, size_t workspace_bytes,
+                                          void *cuda_stream)
+{
+    return mars::run_stochastic(logits, ld, dt, tok, parent, uniform, 0, B, N, V, theta, temperature, flags,
+                                accept_len, out_tokens, path_nodes, out_len, Dcap, seq_status, node_prob,
+                                node_how, workspace, workspace_bytes, cuda_stream);
+}
+
+mars_status_t mars_verify_chain_stochastic(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *draft,
+                                           const float *uniform, int B, int K, int V, float theta,
+                                           float temperature, uint32_t flags, int32_t *accept_len,
+                                           int32_t *out_tokens, int32_t *out_len, int32_t *seq_status,
+                                           float *node_prob, uint8_t *node_how, void *workspace,
+                                           size_t workspace_bytes, void *cuda_stream)
+{
+    if (flags & MARS_SHARED_PARENT) return MARS_ERR_INVALID_ARG;
+    return mars::run_stochastic(logits, ld, dt, draft, nullptr, uniform, 1, B, K, V, theta, temperature, flags,
+                                accept_len, out_tokens, nullptr, out_len, K - 1, seq_status, node_prob,
+                                node_how, workspace, workspace_bytes, cuda_stream);
+}
+
+}  // extern "C"

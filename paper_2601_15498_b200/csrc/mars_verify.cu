@@ -21,8 +21,7 @@
 // Finished slices meet in global memory: the block writes its 16-byte record, bumps the
 // sequence's arrival counter, and the block that arrives last (nobody waits, nobody spins)
 // merges the records of the sequence and runs the verification tail of mars_common.cuh.
-#include "mars_common.cuh"
-#include "mars_stream.cuh"
+#include "mars_top2_stream.cuh"
 
 #include <cmath>
 #include <cstdlib>
@@ -32,16 +31,6 @@
 #include "mars.h"
 
 namespace mars {
-
-constexpr int kThreads = 256;  // threads per block
-constexpr int kU = 8;          // 16-byte vectors per thread per batch (128 B in flight each)
-// Large bf16 batches run a second instantiation with 4 vectors per batch and 8 resident blocks
-// per SM (32 registers): the same bytes in flight from twice the threads measured 1-1.5 %
-// faster there, and slower for fp32 and for batches of a few hundred rows.
-constexpr int kUDense = 4;
-constexpr int kDenseMinRows = 148 * 16;
-constexpr int kTargetBlocks = 148 * 4;      // resident blocks of this kernel on a B200
-constexpr int kMinSliceBytes = kThreads * kU * 16;   // a slice is at least one full batch
 
 struct Params {
     const void *logits;
@@ -58,83 +47,6 @@ struct Params {
     int tail_smem_off;   // byte offset of that staging area in dynamic shared memory
     TailArgs tail;
 };
-
-// ---- order-preserving float <-> uint encoding for the shared bound ----------------------
-__device__ __forceinline__ unsigned enc(float x)
-{
-    unsigned b = __float_as_uint(x + 0.0f);
-    return b ^ ((unsigned)((int)b >> 31) | 0x80000000u);
-}
-__device__ __forceinline__ float dec(unsigned e)
-{
-    return __uint_as_float(e ^ ((e & 0x80000000u) ? 0x80000000u : 0xffffffffu));
-}
-
-// Insert one element's value into the block-wide multiset top-2 {T1 >= T2}.  Every element
-// is published at most once, so T2 never exceeds the slice's true runner-up value.
-__device__ __forceinline__ void publish(unsigned *sT, float x)
-{
-    unsigned e = enc(x);
-    if (e > *(volatile unsigned *)&sT[1]) {
-        unsigned old = atomicMax(&sT[0], e);
-        unsigned y = min(old, e);
-        if (y > *(volatile unsigned *)&sT[1]) atomicMax(&sT[1], y);
-    }
-}
-
-// Exact insert of one element into the thread's top-2.  Valid because a thread sees its
-// elements in increasing token id: equality never displaces.
-template <bool PUBLISH>
-__device__ __forceinline__ void insert(Rec &s, float x, int idx, unsigned *sT)
-{
-    if (x > s.z2) {
-        if (x > s.z1) { s.z2 = s.z1; s.id2 = s.id1; s.z1 = x; s.id1 = idx; }
-        else { s.z2 = x; s.id2 = idx; }
-        if (PUBLISH) publish(sT, x);
-    }
-}
-
-template <int DT, int U, bool PUBLISH>
-__device__ __forceinline__ void process_batch(const uint4 (&v)[U], const typename Elem<DT>::packed_t (&q)[U],
-                                              float bm, float T2, int idx0, Rec &s, unsigned *sT)
-{
-    typedef Elem<DT> E;
-    if (bm > s.z2 && bm >= T2) {
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float qf = E::to_float(q[u]);
-            if (qf > s.z2 && qf >= T2) {
-                int base = idx0 + u * kThreads * E::kVec;
-#pragma unroll
-                for (int k = 0; k < E::kVec; ++k) insert<PUBLISH>(s, E::elem(v[u], k), base + k, sT);
-            }
-        }
-    }
-}
-
-template <int DT, int U, bool GUARD>
-__device__ __forceinline__ float load_batch(const uint4 *vbase, int v0, int nvec, uint4 (&v)[U],
-                                            typename Elem<DT>::packed_t (&q)[U])
-{
-    typedef Elem<DT> E;
-    static_assert(U >= 4 && (U & (U - 1)) == 0, "U must be a power of two >= 4");
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        int vi = v0 + u * kThreads;
-        if (!GUARD || vi < nvec) v[u] = ld_stream(vbase + vi);
-        else v[u] = E::neg_inf();
-    }
-#pragma unroll
-    for (int u = 0; u < U; ++u) q[u] = E::vred(v[u]);
-    typename E::packed_t m[U / 2];
-#pragma unroll
-    for (int u = 0; u < U / 2; ++u) m[u] = E::pmax(q[2 * u], q[2 * u + 1]);
-#pragma unroll
-    for (int w = U / 4; w > 0; w >>= 1)
-#pragma unroll
-        for (int u = 0; u < w; ++u) m[u] = E::pmax(m[u], m[u + w]);
-    return E::to_float(m[0]);
-}
 
 template <int DT, int U, int MINB>
 __global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
@@ -270,27 +182,6 @@ __global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
 }
 
 // ------------------------------------------------------------------------- host side
-
-struct Split { int S; int L; };
-
-static Split choose_split(long long R, int V, int dt)
-{
-    const int es = dt == MARS_BF16 ? 2 : 4;
-    long long S = 1;
-    const char *force = getenv("MARS_FORCE_SPLIT");  // test hook: force slices per row
-    int min_elems = kMinSliceBytes / es;
-    if (force && atoi(force) >= 1) { S = atoi(force); min_elems = 64; }
-    else if (R < kTargetBlocks) S = kTargetBlocks / R;   // never more blocks than fit at once
-    long long smax = V / min_elems;
-    if (smax < 1) smax = 1;
-    if (S > smax) S = smax;
-    long long L = (V + S - 1) / S;
-    L = (L + 15) / 16 * 16;
-    Split sp;
-    sp.L = (int)L;
-    sp.S = (int)((V + L - 1) / L);
-    return sp;
-}
 
 static size_t counters_bytes(int B) { return ((size_t)B * sizeof(unsigned) + 255) / 256 * 256; }
 

@@ -16,6 +16,7 @@ from . import build as _build
 
 BF16, FP32 = 0, 1
 SIGN_LITERAL, SHARED_PARENT, COUNTERS_ZERO, RULE_MARGIN, RULE_PROB_RATIO = 1, 2, 4, 8, 16
+STOCH_PLAIN, STOCH_RELAX_ONLY = 32, 64
 MAX_NODES = 1024
 
 _lock = threading.Lock()
@@ -76,6 +77,14 @@ def lib() -> ctypes.CDLL:
             L.mars_topk_rows.restype = i32
             L.mars_lmhead_top2_shard.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, sz, vp]
             L.mars_lmhead_top2_shard.restype = i32
+            L.mars_stochastic_workspace_bytes.argtypes = [i32, i32, i32, i32]
+            L.mars_stochastic_workspace_bytes.restype = sz
+            L.mars_verify_tree_stochastic.argtypes = [vp, i64, i32, vp, vp, vp, i32, i32, i32, f32, f32, u32,
+                                                      vp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+            L.mars_verify_tree_stochastic.restype = i32
+            L.mars_verify_chain_stochastic.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, f32, u32,
+                                                       vp, vp, vp, vp, vp, vp, vp, sz, vp]
+            L.mars_verify_chain_stochastic.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -260,6 +269,91 @@ def lmhead_verify(hidden: torch.Tensor, w_vocab: torch.Tensor, bias, tok, parent
             workspace.numel(), _stream())
     _check(code, "mars_lmhead_verify")
     out["_keepalive"] = (tok, parent, workspace, bias)
+    return out
+
+
+def _dev_f32(x, device) -> torch.Tensor:
+    t = torch.as_tensor(x)
+    if t.dtype != torch.float32 or t.device != device or not t.is_contiguous():
+        t = t.to(device=device, dtype=torch.float32).contiguous()
+    return t
+
+
+def alloc_stochastic_outputs(B: int, N: int, Dcap: int, device, debug: bool = False) -> dict:
+    out = alloc_outputs(B, N, Dcap, device)
+    if debug:
+        out["node_prob"] = torch.full((B, N), float("nan"), dtype=torch.float32, device=device)
+        out["node_how"] = torch.full((B, N), 255, dtype=torch.uint8, device=device)
+    return out
+
+
+def _stoch_workspace(B, N, V, dt, device, workspace):
+    need = int(lib().mars_stochastic_workspace_bytes(B, N, V, dt))
+    if need == 0:
+        raise MarsError("unsupported sizes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    return workspace, workspace.numel() * workspace.element_size()
+
+
+def verify_tree_stochastic(logits: torch.Tensor, tok, parent, uniform, theta: float, temperature: float,
+                           flags: int = 0, Dcap: int | None = None, V: int | None = None,
+                           debug: bool = False, workspace: torch.Tensor | None = None,
+                           out: dict | None = None) -> dict:
+    """mars_verify_tree_stochastic on the current stream; `uniform` is float32 [B, N]."""
+    dev = logits.device
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    uniform = _dev_f32(uniform, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    if tuple(uniform.shape) != (B, N):
+        raise MarsError("uniform must be [B, N]")
+    dt, ld, V = _logits_args(logits, B * N, V)
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    workspace, wbytes = _stoch_workspace(B, N, V, dt, dev, workspace)
+    if out is None:
+        out = alloc_stochastic_outputs(B, N, Dcap, dev, debug)
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_tree_stochastic(
+            logits.data_ptr(), ld, dt, tok.data_ptr(), parent.data_ptr(), uniform.data_ptr(), B, N, V,
+            float(theta), float(temperature), flags, out["accept_len"].data_ptr(),
+            out["out_tokens"].data_ptr(), out["path_nodes"].data_ptr(), out["out_len"].data_ptr(), Dcap,
+            out["seq_status"].data_ptr(),
+            out["node_prob"].data_ptr() if "node_prob" in out else None,
+            out["node_how"].data_ptr() if "node_how" in out else None,
+            workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_verify_tree_stochastic")
+    out["_keepalive"] = (tok, parent, uniform, workspace)
+    return out
+
+
+def verify_chain_stochastic(logits: torch.Tensor, draft, uniform, theta: float, temperature: float,
+                            flags: int = 0, V: int | None = None, debug: bool = False,
+                            workspace: torch.Tensor | None = None, out: dict | None = None) -> dict:
+    """mars_verify_chain_stochastic on the current stream: K rows, K-1 drafts, uniform [B, K]."""
+    dev = logits.device
+    draft = _dev_i32(draft, dev)
+    uniform = _dev_f32(uniform, dev)
+    B, Km1 = draft.shape
+    K = Km1 + 1
+    if tuple(uniform.shape) != (B, K):
+        raise MarsError("uniform must be [B, K]")
+    dt, ld, V = _logits_args(logits, B * K, V)
+    workspace, wbytes = _stoch_workspace(B, K, V, dt, dev, workspace)
+    if out is None:
+        out = alloc_stochastic_outputs(B, K, K - 1, dev, debug)
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_chain_stochastic(
+            logits.data_ptr(), ld, dt, draft.data_ptr() if Km1 > 0 else None, uniform.data_ptr(), B, K, V,
+            float(theta), float(temperature), flags, out["accept_len"].data_ptr(),
+            out["out_tokens"].data_ptr(), out["out_len"].data_ptr(), out["seq_status"].data_ptr(),
+            out["node_prob"].data_ptr() if "node_prob" in out else None,
+            out["node_how"].data_ptr() if "node_how" in out else None,
+            workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_verify_chain_stochastic")
+    out["_keepalive"] = (draft, uniform, workspace)
     return out
 
 

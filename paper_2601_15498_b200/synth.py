@@ -239,3 +239,12 @@ def to_numpy_bits(t: torch.Tensor) -> np.ndarray:
     if t.dtype == torch.bfloat16:
         return t.view(torch.int16).numpy().view(np.uint16)
     return t.numpy()
+
+
+def make_uniforms(B: int, N: int, seed: int) -> np.ndarray:
+    """float32 uniforms in [0, 1) for stochastic verification: [b, i > 0] judges node i,
+    [b, 0] draws the next token.  They are inputs of the method, drawn here so that the oracle
+    and the library consume the same numbers."""
+    rng = np.random.Generator(np.random.Philox(key=[seed, 0x0A11CE]))
+    u = rng.random((B, N), dtype=np.float32)
+    return np.minimum(u, np.float32(1.0) - np.float32(2.0 ** -24))

@@ -1,0 +1,329 @@
+"""Parity of stochastic (T > 0) verification with the CPU oracle, through the C ABI.
+
+The oracle evaluates the softmax in fp64, the library in fp32 with the hardware 2^x; the
+uniforms are inputs shared by both.  Bar:
+  * top-2 based decisions (exact match, relaxed runner-up) are bit-exact as everywhere else;
+  * node probabilities agree within PROB_RTOL;
+  * a sequence whose every Eq. 1 test was decided by more than DECISION_TOL (of the row's total
+    mass; the oracle reports the smallest such margin) must have the same walk: accepted length,
+    path, per-node decisions, accepted tokens; closer ones may differ, are counted, bounded,
+    and must still be valid walks;
+  * where the walk is the same the drawn token must be the oracle's, or else u*W must lie within
+    DRAW_TOL * W of the fp64 CDF interval of the token the library drew (a neighbouring step).
+Where the tolerances come from: an fp32 weight 2^(z*c - ref) carries the rounding of its
+exponent (|z*c - ref| up to about 2^6 where it matters, so about 2^-18 * ln 2 absolute, 3e-6
+relative) and 2 ulp of the approximation; the denominator is an fp32 sum of up to 151 936 such
+terms in a tree of partial sums (about 1e-6 relative); the draw accumulates in fp64, so its
+position error is that of the weights.  DECISION_TOL = 2e-5 and DRAW_TOL = 1e-5 leave a margin
+of several times over these and flag only a few decisions in 10^5.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mars_oracle as orc
+from paper_2601_15498_b200 import mars, synth
+
+pytestmark = pytest.mark.gpu
+DEV = os.environ.get("MARS_TEST_DEVICE", "cuda:0")
+PROB_RTOL = 2e-5
+DECISION_TOL = 2e-5
+DRAW_TOL = 1e-5
+WALK_KEYS = ("accept_len", "path_nodes", "out_len", "seq_status", "node_how")
+STATS = {"close": 0, "draw_neighbour": 0, "sequences": 0, "max_draw_dist": 0.0}
+
+
+@pytest.fixture(autouse=True)
+def _no_hooks(monkeypatch):
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    monkeypatch.delenv("MARS_STOCH_VARIANT", raising=False)
+
+
+def check_walk_is_valid(got, tok, parent, b):
+    a = int(got["accept_len"][b])
+    path = got["path_nodes"][b, :a + 1]
+    assert path[0] == 0 and got["out_len"][b] == a + 1
+    par = parent if parent.ndim == 1 else parent[b]
+    for d in range(1, a + 1):
+        c = int(path[d])
+        assert par[c] == path[d - 1] and got["node_how"][b, c] in (1, 2, 3)
+        assert got["out_tokens"][b, d - 1] == tok[b, c]
+    assert got["out_tokens"][b, a] >= 0
+
+
+def draw_distance(row_f64, T, removed, u0, token):
+    """Distance (in units of the residual mass W) of u0*W from the CDF interval of `token`."""
+    w = np.exp((row_f64 - np.max(row_f64[np.isfinite(row_f64)])) / T)
+    w[np.isnan(w)] = 0.0
+    w[list(removed)] = 0.0
+    c = np.cumsum(w)
+    W = c[-1]
+    lo, hi = (c[token - 1] if token > 0 else 0.0), c[token]
+    t = float(u0) * W
+    if w[token] <= 0.0:
+        return np.inf
+    return max(lo - t, t - hi, 0.0) / W
+
+
+def compare(got, ref, tok, parent, logits_host, u, T, what="", max_close_frac=0.02):
+    """logits_host: float64 [R, V] view of the rows (exact widening)."""
+    B, N = tok.shape
+    n_close = n_neigh = 0
+    for b in range(B):
+        par = parent if parent.ndim == 1 else parent[b]
+        a = int(ref["accept_len"][b])
+        same_walk = all(np.array_equal(got[k][b], ref[k][b]) for k in WALK_KEYS) and \
+            np.array_equal(got["out_tokens"][b, :a], ref["out_tokens"][b, :a])
+        if not same_walk:
+            if ref["margin"][b, 0] < DECISION_TOL:
+                n_close += 1
+                if got["seq_status"][b] == 0:
+                    check_walk_is_valid(got, tok, parent, b)
+                continue
+            diff = {k: (got[k][b].tolist(), ref[k][b].tolist()) for k in WALK_KEYS + ("out_tokens",)
+                    if not np.array_equal(got[k][b], ref[k][b])}
+            raise AssertionError(f"{what}: sequence {b} differs (margins {ref['margin'][b]}): {diff}")
+        g, r = int(got["out_tokens"][b, a]), int(ref["out_tokens"][b, a])
+        assert (got["out_tokens"][b, a + 1:] == -1).all()
+        if g != r:
+            assert ref["seq_status"][b] == 0, (what, b)
+            cur = int(ref["path_nodes"][b, a])
+            removed = {int(tok[b, i]) for i in range(1, N) if par[i] == cur and ref["node_how"][b, i] == 4
+                       and 0 <= tok[b, i] < logits_host.shape[1]}
+            d = draw_distance(logits_host[b * N + cur], T, removed, u[b, 0], g)
+            STATS["max_draw_dist"] = max(STATS["max_draw_dist"], float(d))
+            assert d <= DRAW_TOL, (what, b, g, r, d)
+            n_neigh += 1
+    ok = ref["seq_status"] != 1
+    np.testing.assert_allclose(got["node_prob"][ok], ref["node_prob"][ok], rtol=PROB_RTOL, atol=1e-30,
+                               err_msg=what)
+    STATS["close"] += n_close
+    STATS["draw_neighbour"] += n_neigh
+    STATS["sequences"] += B
+    assert n_close <= max(2, int(max_close_frac * B)), (what, n_close, B)
+    assert n_neigh <= max(2, int(0.1 * B)), (what, n_neigh, B)
+    return n_close, n_neigh
+
+
+def host_f64(logits, V=None):
+    x = logits.detach().float().cpu().numpy().astype(np.float64)
+    return x if V is None else x[:, :V]
+
+
+def run_and_compare(logits, tok, parent, u, theta, T, flags=0, Dcap=None, what="", **kw):
+    got = mars.to_host(mars.verify_tree_stochastic(logits, tok, parent, u, theta, T, flags, Dcap, debug=True))
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(logits), tok, parent, u, theta, T, flags, Dcap)
+    compare(got, ref, tok, parent, host_f64(logits), u, T, what, **kw)
+    return got, ref
+
+
+def third_candidates(w, seed, delta=1.5, frac=0.3):
+    """Input construction for these tests: plants a third logit at z1 - delta in every row and
+    aims a fraction of the draft tokens at it, so that candidates which are neither the top-1 nor
+    the runner-up carry a visible probability and the Eq. 1 test decides both ways."""
+    rng = np.random.default_rng(seed)
+    top = torch.topk(w.logits[:, :w.V].float(), 2, dim=1)
+    ids3 = torch.as_tensor(rng.integers(0, w.V, w.R), device=w.logits.device)
+    clash = (ids3 == top.indices[:, 0]) | (ids3 == top.indices[:, 1])
+    ids3 = torch.where(clash, (top.indices.max(dim=1).values + 1) % w.V, ids3)
+    clash = (ids3 == top.indices[:, 0]) | (ids3 == top.indices[:, 1])
+    ids3 = torch.where(clash, (ids3 + 1) % w.V, ids3)
+    rows = torch.arange(w.R, device=w.logits.device)
+    w.logits[rows, ids3] = (top.values[:, 0] - delta).to(w.logits.dtype)
+    ids3 = ids3.cpu().numpy().reshape(w.B, w.N)
+    par = w.parent if w.parent.ndim == 2 else np.tile(w.parent, (w.B, 1))
+    for b in range(w.B):
+        for i in range(1, w.N):
+            if par[b, i] >= 0 and rng.random() < frac:
+                w.tok[b, i] = ids3[b, par[b, i]]
+    return w
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY])
+@pytest.mark.parametrize("T", [0.7, 1.0, 2.0])
+def test_small_trees(dtype, flags, T):
+    """Rows of several tiles with a ragged tail; candidates of every kind."""
+    w = third_candidates(synth.tree_workload("t", 48, 20, 4, 3, 33333, dtype, DEV, 21, 0.9, 1.0, 9.0, 16.0, 0.4), 21)
+    u = synth.make_uniforms(w.B, w.N, 21)
+    got, ref = run_and_compare(w.logits, w.tok, w.parent, u, w.theta, T, flags, what=f"{dtype} flags={flags} T={T}")
+    how = ref["node_how"]
+    assert (how == 4).any()
+    if T <= 1.0:
+        assert (how == 3).any() and ref["accept_len"].max() >= 1
+    if flags == mars.STOCH_PLAIN:
+        assert not ((how == 1) | (how == 2)).any()
+
+
+def test_cfg1_one_tree_rows_split_over_blocks():
+    w = synth.cfg1(DEV)
+    for seed in range(4):
+        u = synth.make_uniforms(w.B, w.N, 100 + seed)
+        run_and_compare(w.logits, w.tok, w.parent, u, w.theta, 1.0, what=f"cfg1 seed {seed}")
+
+
+def test_cfg3_slice_of_the_serving_batch():
+    w = synth.cfg3(DEV, B=12)
+    u = synth.make_uniforms(w.B, w.N, 3)
+    for flags in (0, mars.STOCH_PLAIN):
+        run_and_compare(w.logits, w.tok, w.parent, u, w.theta, 1.0, flags, what=f"cfg3 B=12 flags={flags}")
+
+
+def test_chain_form_equals_the_tree_oracle_on_linear_parents():
+    w = synth.cfg2(DEV, B=16)
+    u = synth.make_uniforms(w.B, w.N, 2)
+    got = mars.to_host(mars.verify_chain_stochastic(w.logits, w.draft, u, w.theta, 1.0, debug=True))
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, w.theta, 1.0)
+    got["path_nodes"] = ref["path_nodes"]       # the chain call has no path output
+    compare(got, ref, w.tok, w.parent, host_f64(w.logits), u, 1.0, "chain")
+    assert (got["out_len"] == got["accept_len"] + 1).all()
+
+
+def test_cfg0_chain_fp32():
+    w = synth.cfg0(DEV, B=64, seed=9)
+    u = synth.make_uniforms(w.B, w.N, 9)
+    got = mars.to_host(mars.verify_chain_stochastic(w.logits, w.draft, u, w.theta, 1.0, debug=True))
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, w.theta, 1.0)
+    got["path_nodes"] = ref["path_nodes"]
+    compare(got, ref, w.tok, w.parent, host_f64(w.logits), u, 1.0, "cfg0")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_unaligned_rows_and_odd_sizes(dtype):
+    """Row stride and vocabulary that keep no row 16-byte aligned: scalar head / tail in the
+    streaming pass, element-wise tiles in the draw."""
+    V, ld = 4099, 4103
+    w = synth.tree_workload("t", 24, 9, 3, 3, V, dtype, DEV, 33, 0.9, 1.0, 5.0, 8.0, 0.4, ld=ld, pad_value=50.0)
+    u = synth.make_uniforms(w.B, w.N, 33)
+    base = w.logits.reshape(-1)[1:1 + (w.R - 1) * ld + V]     # shift by one element
+    shifted = torch.as_strided(base, (w.R, V), (ld, 1))
+    src = w.logits[:, :V].clone()
+    shifted.copy_(src)
+    got = mars.to_host(mars.verify_tree_stochastic(shifted, w.tok, w.parent, u, 0.9, 1.0, V=V, debug=True))
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(src), w.tok, w.parent, u, 0.9, 1.0)
+    compare(got, ref, w.tok, w.parent, host_f64(src), u, 1.0, "unaligned")
+
+
+@pytest.mark.parametrize("split", [2, 3, 7])
+def test_forced_row_splits(split, monkeypatch):
+    monkeypatch.setenv("MARS_FORCE_SPLIT", str(split))
+    w = synth.tree_workload("t", 10, 12, 3, 3, 20011, torch.bfloat16, DEV, 44, 0.9, 1.0, 6.0, 9.0, 0.4)
+    u = synth.make_uniforms(w.B, w.N, 44)
+    run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.3, what=f"split {split}")
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+def test_every_instantiation_of_the_streaming_kernel(variant, monkeypatch):
+    monkeypatch.setenv("MARS_STOCH_VARIANT", str(variant))
+    for dtype in (torch.float32, torch.bfloat16):
+        w = synth.tree_workload("t", 8, 10, 3, 3, 40000, dtype, DEV, 55, 0.9, 1.0, 6.0, 9.0, 0.4)
+        u = synth.make_uniforms(w.B, w.N, 55)
+        run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.0, what=f"variant {variant} {dtype}")
+
+
+def test_tiny_vocabularies_one_tile():
+    for V in (2, 3, 9, 200, 257):
+        w = synth.tree_workload("t", 40, 6, 2, 3, V, torch.float32, DEV, 60 + V, 0.9, 1.0, 2.0, 3.0, 0.4)
+        u = synth.make_uniforms(w.B, w.N, V)
+        run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.0, mars.STOCH_PLAIN, what=f"V={V}", max_close_frac=0.05)
+
+
+def test_special_nodes_duplicates_padding_and_out_of_range_ids():
+    w = synth.tree_workload("t", 64, 16, 4, 4, 3000, torch.float32, DEV, 70, 0.9, 1.0, 4.0, 6.0, 0.4)
+    tok = w.tok.copy()
+    tok[:, 5] = tok[:, 4]            # a repeated token (siblings in many of the trees)
+    tok[:, 7] = -1                   # padding node
+    tok[:, 9] = w.V + 5              # id outside the vocabulary
+    parent = w.parent.copy()
+    parent[:, 11] = -1               # absent node
+    u = synth.make_uniforms(w.B, w.N, 70)
+    for flags in (0, mars.STOCH_PLAIN):
+        got, ref = run_and_compare(w.logits, tok, parent, u, 0.9, 1.0, flags, what="special nodes")
+        assert (got["node_how"][:, 7] == 0).all() and (got["node_prob"][:, 9] == 0).all()
+
+
+def test_degenerate_rows_bad_trees_and_depth_cap():
+    V = 5000
+    w = synth.tree_workload("t", 6, 8, 3, 2, V, torch.float32, DEV, 80, 0.9, 1.0, 5.0, 8.0, 0.4)
+    lg = w.logits.clone()
+    lg[0 * 8 + 0, :] = float("-inf")                 # sequence 0: root row without a distribution
+    lg[1 * 8 + 0, 17] = float("inf")                 # sequence 1: +inf logit
+    lg[2 * 8 + 0, 100:200] = float("nan")            # sequence 2: NaNs count as -inf, still fine
+    parent = w.parent.copy()
+    parent[3, 4] = 6                                 # sequence 3: malformed tree
+    u = synth.make_uniforms(w.B, w.N, 80)
+    got, ref = run_and_compare(lg, w.tok, parent, u, 0.9, 1.0, what="degenerate")
+    assert ref["seq_status"].tolist()[:4] == [4, 4, 0, 1]
+    assert got["out_tokens"][1, 0] == 17 and got["out_tokens"][0, 0] == 0
+    # depth cap: uniforms of zero accept every first child; outputs hold one level only
+    u0 = np.zeros_like(u)
+    got, ref = run_and_compare(w.logits, w.tok, w.parent, u0, 0.9, 1.0, Dcap=1, what="Dcap")
+    assert (ref["seq_status"] == 2).any()
+
+
+def test_rule_variants_and_sign_flag_pass_through():
+    w = synth.tree_workload("t", 32, 12, 3, 3, 9000, torch.bfloat16, DEV, 90, 0.9, 1.0, 6.0, 9.0, 0.5)
+    u = synth.make_uniforms(w.B, w.N, 90)
+    for flags, theta in ((mars.RULE_MARGIN, 0.75), (mars.RULE_PROB_RATIO, 0.4), (mars.SIGN_LITERAL, 0.9)):
+        run_and_compare(w.logits, w.tok, w.parent, u, theta, 1.0, flags, what=f"flags {flags}")
+
+
+def test_plain_mode_preserves_the_target_distribution_on_the_gpu():
+    """A property that needs no oracle: with Eq. 1 alone the first emitted token follows the
+    root row's softmax, whatever the candidates are (20 000 sequences over one fixed tree)."""
+    rng = np.random.default_rng(5)
+    V, N, B, T = 48, 5, 20000, 0.9
+    rows = torch.tensor((rng.normal(size=(N, V)) * 1.2).astype(np.float32))
+    logits = rows.repeat(B, 1).to(DEV)
+    parent = np.array([-1, 0, 0, 0, 1], np.int32)
+    lead = torch.topk(rows[0], 3).indices.numpy()
+    tok = np.tile(np.array([-1, lead[1], lead[0], lead[2], 7], np.int32), (B, 1))
+    u = synth.make_uniforms(B, N, 5)
+    got = mars.to_host(mars.verify_tree_stochastic(logits, tok, parent, u, 0.9, T, mars.STOCH_PLAIN))
+    P = torch.softmax(rows[0].double() / T, 0).numpy()
+    f = np.bincount(got["out_tokens"][:, 0], minlength=V) / B
+    sd = np.sqrt(P * (1 - P) / B)
+    assert np.all(np.abs(f - P) <= 4.5 * sd + 1e-9)
+
+
+def test_host_errors():
+    w = synth.tree_workload("t", 2, 4, 2, 2, 100, torch.float32, DEV, 1, 0.9, 1.0, 5.0, 6.0, 0.3)
+    u = synth.make_uniforms(w.B, w.N, 1)
+    for T in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(mars.MarsError, match="invalid argument"):
+            mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, T)
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, mars.STOCH_PLAIN | mars.STOCH_RELAX_ONLY)
+    with pytest.raises(mars.MarsError, match="unsupported"):
+        mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, mars.COUNTERS_ZERO)
+    small = torch.empty(256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(mars.MarsError, match="workspace"):
+        mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, workspace=small[:16])
+
+
+def test_full_size_batch_sampled_sequences():
+    """The serving-scale batch in the launch configuration the benchmark times (256 x 60 rows of
+    151 936 bf16 logits); the oracle checks a sample of whole sequences."""
+    w = synth.cfg3(DEV)
+    u = synth.make_uniforms(w.B, w.N, 3)
+    got = mars.to_host(mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, w.theta, 1.0, debug=True))
+    assert (got["seq_status"] == 0).all()
+    pick = np.random.default_rng(0).choice(w.B, 10, replace=False)
+    for b in pick:
+        rows = synth.to_numpy_bits(w.logits[b * w.N:(b + 1) * w.N])
+        ref = orc.verify_tree_stochastic(rows, w.tok[b:b + 1], w.parent[b:b + 1], u[b:b + 1], w.theta, 1.0)
+        one = {k: got[k][b:b + 1] for k in got}
+        compare(one, ref, w.tok[b:b + 1], w.parent[b:b + 1], host_f64(w.logits[b * w.N:(b + 1) * w.N]),
+                u[b:b + 1], 1.0, f"sequence {b}", max_close_frac=1.0)
+    for b in range(w.B):
+        check_walk_is_valid(got, w.tok, w.parent, b)
+
+
+def test_zz_report_tolerated_cases():
+    """Not a check of the library: prints how many decisions of this module fell inside the
+    tolerances (run with -s to see it) and keeps the share small."""
+    print("stochastic parity:", STATS)
+    if STATS["sequences"]:
+        assert STATS["close"] <= 0.01 * STATS["sequences"] + 2
