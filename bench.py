@@ -148,6 +148,16 @@ def reduce_max_time_sum_units(elapsed_ms: float, units: float, world: int):
     return float(t.item()), float(u.item())
 
 
+def exp_unit_roofline(w, ms_per_step: float, clocks: dict):
+    """Second ceiling of the stochastic path: one 2^x per logit on the SMs' exponential units
+    (16 results per clock per SM, 148 SMs) at the SM clock sampled during the timed region."""
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965
+    peak = 148 * 16 * mhz * 1e6 / 1e9
+    achieved = w.R * w.V / (ms_per_step * 1e-3) / 1e9
+    return {"bound": "alu", "unit": "G exp/s", "achieved": achieved, "peak": peak, "frac": achieved / peak,
+            "peak_source": f"148 SMs x 16 per clock x {mhz:g} MHz (median sampled SM clock)"}
+
+
 def barrier(world: int):
     if world > 1:
         import torch.distributed as dist
@@ -156,12 +166,20 @@ def barrier(world: int):
 
 # ------------------------------------------------------------------------------ arms
 
-def run_oracle_sample(w, host_logits, seqs: int):
+def run_oracle_sample(w, host_logits, seqs: int, temperature=None, uniform=None):
     from oracle import mars_oracle as orc
     n = seqs * w.N
     t0 = time.perf_counter()
-    orc.verify_tree(host_logits[:n], w.tok[:seqs], w.parent[:seqs], w.theta)
+    if temperature is None:
+        orc.verify_tree(host_logits[:n], w.tok[:seqs], w.parent[:seqs], w.theta)
+    else:
+        orc.verify_tree_stochastic(host_logits[:n], w.tok[:seqs], w.parent[:seqs], uniform[:seqs], w.theta,
+                                   temperature)
     return time.perf_counter() - t0, n, orc.threads()
+
+
+def stochastic_tag(args) -> str:
+    return f"_stochastic_T{args.stochastic:g}" if args.stochastic else ""
 
 
 def reference_arm(args, rank: int):
@@ -178,12 +196,13 @@ def reference_arm(args, rank: int):
         w = maker("cpu", seed=seed, B=16, **kw)
     seqs = w.B
     host = synth.to_numpy_bits(w.logits)
+    uni = synth.make_uniforms(w.B, w.N, seed) if args.stochastic else None
     for _ in range(args.warmup):
-        run_oracle_sample(w, host, seqs)
+        run_oracle_sample(w, host, seqs, args.stochastic, uni)
     t = 0.0
     cores = 1
     for _ in range(args.steps):
-        dt, n, cores = run_oracle_sample(w, host, seqs)
+        dt, n, cores = run_oracle_sample(w, host, seqs, args.stochastic, uni)
         t += dt
     value = seqs * w.N * args.steps / t
     line = {
@@ -191,7 +210,7 @@ def reference_arm(args, rank: int):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": FULL_NAME[args.workload],
+        "config": {"workload": FULL_NAME[args.workload] + stochastic_tag(args),
                    "logits_dtype": "bf16" if w.logits.dtype == torch.bfloat16 else "f32", "B": w.B, "N": w.N, "V": w.V, "theta": w.theta,
                    "note": "CPU oracle; each step is a bounded sample (B sequences) of the workload"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -369,6 +388,9 @@ def main():
                     help="cudaProfilerStart/Stop around the timed region (for ncu --profile-from-start off)")
     ap.add_argument("--graph", action="store_true",
                     help="replay the steps from a CUDA graph (device time of launch-bound workloads)")
+    ap.add_argument("--stochastic", type=float, default=None, metavar="T",
+                    help="time stochastic verification at temperature T (Eq. 1 on the running residual + "
+                         "draw) instead of the deterministic rule")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the number of sequences (smaller cases for profiler captures)")
     args = ap.parse_args()
@@ -418,10 +440,21 @@ def main():
 
     ws.zero_()
     fl = mars.COUNTERS_ZERO     # the workspace starts zeroed and every call leaves its counters at zero
+    T = args.stochastic
+    if T:
+        uni_h = synth.make_uniforms(w.B, w.N, BASE_SEED[args.workload] + 1000 * rank)
+        uni = torch.as_tensor(uni_h, device=dev)
+        ws_s = torch.zeros(int(mars.lib().mars_stochastic_workspace_bytes(w.B, w.N, w.V, dt_code)),
+                           dtype=torch.uint8, device=dev)
+        out = mars.alloc_stochastic_outputs(w.B, w.N, w.N - 1, dev)
 
     def step(i, lg=None):
         lg = logits[i % copies] if lg is None else lg
-        if w.kind == "chain":
+        if T and w.kind == "chain":
+            mars.verify_chain_stochastic(lg, draft, uni, w.theta, T, workspace=ws_s, out=out)
+        elif T:
+            mars.verify_tree_stochastic(lg, tok, parent, uni, w.theta, T, workspace=ws_s, out=out)
+        elif w.kind == "chain":
             mars.verify_chain(lg, draft, w.theta, flags=fl, workspace=ws, out=out)
         else:
             mars.verify_tree(lg, tok, parent, w.theta, flags=fl, workspace=ws, out=out)
@@ -476,6 +509,7 @@ def main():
         h_logits.copy_(w.logits)
         h_tok = torch.as_tensor(w.tok).pin_memory()
         h_par = torch.as_tensor(w.parent).pin_memory()
+        h_uni = torch.as_tensor(uni_h).pin_memory() if T else None
         h_out = {k: torch.empty(out[k].shape, dtype=out[k].dtype, pin_memory=True)
                  for k in ("accept_len", "out_tokens", "out_len")}
         d_logits = torch.empty_like(w.logits)
@@ -484,6 +518,8 @@ def main():
             d_logits.copy_(h_logits, non_blocking=True)
             tok.copy_(h_tok, non_blocking=True)
             parent.copy_(h_par, non_blocking=True)
+            if T:
+                uni.copy_(h_uni, non_blocking=True)
             if w.kind == "chain":
                 draft.copy_(tok[:, 1:])
             step(0, d_logits)
@@ -500,7 +536,7 @@ def main():
         f1.record()
         torch.cuda.synchronize()
         e2e_ms, e2e_units = reduce_max_time_sum_units(f0.elapsed_time(f1), float(w.R * args.e2e_steps), world)
-        h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4
+        h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4 + (h_uni.numel() * 4 if T else 0)
         d2h = sum(h.numel() * h.element_size() for h in h_out.values())
         e2e = {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
@@ -514,14 +550,14 @@ def main():
     # ---- roofline of the one kernel on the path (algorithmic bytes: every logit once) ----
     peak, peak_src = measured_hbm_peak()
     achieved = w.logits_bytes / (elapsed_ms / args.steps * 1e-3) / 1e9
-    traffic = ncu_traffic(args.workload) if not args.batch else None
+    traffic = ncu_traffic(args.workload + ("_stochastic" if T else "")) if not args.batch else None
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         host = synth.to_numpy_bits(h_logits if h_logits is not None else w.logits)
         seqs = w.B          # the oracle finishes the whole batch in well under a minute
-        run_oracle_sample(w, host, min(seqs, 2))
-        dt, n, cores = run_oracle_sample(w, host, seqs)
+        run_oracle_sample(w, host, min(seqs, 2), T, uni_h if T else None)
+        dt, n, cores = run_oracle_sample(w, host, seqs, T, uni_h if T else None)
         cpu = {"value": n / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"all {seqs} sequences ({n} rows) of the same workload, one pass, {dt:.2f} s"}
 
@@ -530,23 +566,31 @@ def main():
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "kind": w.kind,
+        "config": {"workload": w.name + stochastic_tag(args), "kind": w.kind,
                    "logits_dtype": "bf16" if w.logits.dtype == torch.bfloat16 else "f32",
-                   "arithmetic": "fp32 comparisons and one fp32 division per row (bf16 widens exactly)", "B": w.B, "N": w.N, "V": w.V,
+                   "arithmetic": ("fp32 softmax weights 2^(z*log2(e)/T - ref) summed online, Eq. 1 on the running "
+                                  "residual, fp64 partial sums in the draw" if T else
+                                  "fp32 comparisons and one fp32 division per row (bf16 widens exactly)"),
+                   "B": w.B, "N": w.N, "V": w.V,
                    "theta": w.theta, "rows_per_step": w.R, "logits_bytes_per_step": w.logits_bytes,
                    "l2": ("inputs larger than L2" if copies == 1 else
                           f"rotating over {copies} input copies, {copies * w.logits_bytes} B > L2"),
                    "launch": "cuda graph replay" if graph is not None else "direct launches",
-                   "workspace": "zeroed once; MARS_COUNTERS_ZERO (counters reset by the kernel itself)",
+                   "workspace": ("uninitialised (records only)" if T else
+                                 "zeroed once; MARS_COUNTERS_ZERO (counters reset by the kernel itself)"),
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "us_per_step": 1e3 * ms_per_step,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,
         "clocks": clocks.summary(),
         "e2e": e2e,
-        "gpu_launches": args.steps,
+        "gpu_launches": args.steps * (2 if T else 1),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
-                     "kernel": "mars::verify_kernel", "algorithmic_bytes_per_launch": w.logits_bytes},
+                     "kernel": "mars::stoch_stream_kernel" if T else "mars::verify_kernel",
+                     "algorithmic_bytes_per_launch": w.logits_bytes,
+                     **({"note": "duration = the whole step (streaming kernel + per-sequence tail kernel); the "
+                                 "streaming kernel's own share is in profiles/",
+                         "exp_unit": exp_unit_roofline(w, elapsed_ms / args.steps, clocks.summary())} if T else {})},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)

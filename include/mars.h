@@ -327,7 +327,8 @@ mars_status_t mars_verify_records(const void *records, int G, const int32_t *tok
  *   node_how   uint8 [B, N] or NULL: 0 not visited, 1 exact match, 2 relaxed runner-up,
  *              3 accepted by Eq. 1, 4 rejected.
  *   workspace  mars_stochastic_workspace_bytes(B, N, V, dt) bytes, 256-byte aligned; contents
- *              need not be initialised.  Two kernels are enqueued; nothing is allocated.
+ *              need not be initialised (one 32-byte record per row slice).  Two kernels are
+ *              enqueued; nothing is allocated.
  *
  * mars_verify_chain_stochastic is the chain form (K rows, K-1 drafts, uniform [B, K] with
  * [b, i] judging draft i-1 and [b, 0] drawing the correction or bonus token).

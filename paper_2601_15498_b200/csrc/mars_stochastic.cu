@@ -66,163 +66,108 @@ __device__ __forceinline__ void soft_add_scalar(float &ref, float &sum, float x,
     }
 }
 
-// NaN -> -inf on the packed representation (one instruction per 16-byte word pair for bf16).
-template <int DT> __device__ __forceinline__ uint4 nan_to_neg_inf(const uint4 &v);
-template <> __device__ __forceinline__ uint4 nan_to_neg_inf<MARS_BF16>(const uint4 &v)
+// ---- packed fp32 pairs (one instruction for two lanes of work) ----------------------------
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
 {
-    return make_uint4(bmax2(v.x, 0xff80ff80u), bmax2(v.y, 0xff80ff80u), bmax2(v.z, 0xff80ff80u),
-                      bmax2(v.w, 0xff80ff80u));
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rc, rd; mov.b64 ra, {%2,%3}; mov.b64 rb, {%4,%5}; mov.b64 rc, {%6,%7};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc; mov.b64 {%0,%1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
 }
-template <> __device__ __forceinline__ uint4 nan_to_neg_inf<MARS_FP32>(const uint4 &v)
+__device__ __forceinline__ float2 add2(float2 a, float2 b)
 {
-    return make_uint4(__float_as_uint(fmaxf(__uint_as_float(v.x), -INFINITY)),
-                      __float_as_uint(fmaxf(__uint_as_float(v.y), -INFINITY)),
-                      __float_as_uint(fmaxf(__uint_as_float(v.z), -INFINITY)),
-                      __float_as_uint(fmaxf(__uint_as_float(v.w), -INFINITY)));
+    float2 d;
+    asm("{ .reg .b64 ra, rb, rd; mov.b64 ra, {%2,%3}; mov.b64 rb, {%4,%5};\n"
+        "add.rn.f32x2 rd, ra, rb; mov.b64 {%0,%1}, rd; }"
+        : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+
+// Rare path of soft_batch: the batch's sum of weights came out NaN, i.e. the batch holds a NaN
+// logit (which counts as -inf: weight 0) or a +inf logit against an infinite reference (the
+// row has no softmax; the sum is made infinite so that the tail reports it).  Re-reads the
+// thread's elements one by one; kept out of line so that the fast path carries none of it.
+template <int DT>
+__device__ __noinline__ float soft_batch_slow(const uint4 *vbase, int v0, int nvec, int U, float c, float nref)
+{
+    typedef Elem<DT> E;
+    float bs = 0.0f;
+    for (int u = 0; u < U; ++u) {
+        const int vi = v0 + u * kThreads;
+        if (vi >= nvec) continue;
+        for (int k = 0; k < E::kVec; ++k) {
+            const float x = E::scalar(vbase, vi * E::kVec + k);
+            if (x == x) {
+                const float t = fmaf(x, c, nref);
+                bs += (t == t) ? ex2f(t) : INFINITY;
+            }
+        }
+    }
+    return bs;
 }
 
 // A batch joins (ref, sum).  bm is the batch maximum (NaN operands ignored by the packed max).
-// NaN logits are mapped to -inf (weight 0) before the exponential; a +inf logit makes the
-// reference infinite and the sum NaN or infinite, which the tail reports as a row without a
-// distribution.
+// Elements are handled in pairs with packed fp32 instructions (one FMA and one add per pair);
+// the 2^t themselves come from the exponential unit, 16 results per clock and SM, which is the
+// tightest limit for bf16 rows at HBM speed.  (Moving a share of them to a polynomial on the
+// FMA pipe was measured and lost: the extra issue slots cost more than the unit gained.)  The
+// fast loop carries no per-element NaN test: a NaN shows in the batch's sum and sends the
+// batch to the slow path.
 template <int DT, int U>
-__device__ __forceinline__ void soft_batch(const uint4 (&v)[U], float bm, float c, float &ref, float &sum)
+__device__ __forceinline__ void soft_batch(const uint4 (&v)[U], float bm, float c, float &ref, float &sum,
+                                           const uint4 *vbase, int v0, int nvec)
 {
     typedef Elem<DT> E;
     const float bmc = bm * c;
     if (bmc > ref) { sum *= ex2f(ref - bmc); ref = bmc; }
     if (!(ref > -INFINITY)) return;          // nothing above -inf seen so far: all weights are 0
-    const float nref = -ref;
-    float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+    const float2 nref2 = make_float2(-ref, -ref), c2 = make_float2(c, c);
+    float2 a0 = make_float2(0.0f, 0.0f), a1 = a0;
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-        const uint4 w = nan_to_neg_inf<DT>(v[u]);
 #pragma unroll
-        for (int k = 0; k < E::kVec; k += 4) {
-            a0 += ex2f(fmaf(E::elem(w, k + 0), c, nref));
-            a1 += ex2f(fmaf(E::elem(w, k + 1), c, nref));
-            a2 += ex2f(fmaf(E::elem(w, k + 2), c, nref));
-            a3 += ex2f(fmaf(E::elem(w, k + 3), c, nref));
+        for (int k = 0; k < E::kVec; k += 2) {
+            const int pair = u * (E::kVec / 2) + k / 2;
+            const float2 t = fma2(make_float2(E::elem(v[u], k), E::elem(v[u], k + 1)), c2, nref2);
+            float2 e;
+            e.x = ex2f(t.x);
+            e.y = ex2f(t.y);
+            if (pair & 1) a1 = add2(a1, e); else a0 = add2(a0, e);
         }
     }
-    sum += (a0 + a1) + (a2 + a3);
+    a0 = add2(a0, a1);
+    float bs = a0.x + a0.y;
+    if (!(bs == bs)) bs = soft_batch_slow<DT>(vbase, v0, nvec, U, c, -ref);
+    sum += bs;
 }
 
-struct StreamParams {
-    const void *logits;
-    long long ld;
-    int V;
-    int S;       // slices per row
-    int L;       // elements per slice (multiple of 16)
-    float c;     // log2(e) / T
-    SRec *partial;   // [R*S]
-};
+// Batch load split in two, so that the next batch's loads can be in flight while the current
+// batch is worked on: issue the 16-byte loads, and later reduce the vectors to their maxima.
+template <int U>
+__device__ __forceinline__ void issue_batch(const uint4 *vbase, int v0, uint4 (&v)[U])
+{
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = ld_stream(vbase + v0 + u * kThreads);
+}
 
-template <int DT, int U, int MINB>
-__global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const StreamParams p)
+template <int DT, int U>
+__device__ __forceinline__ float reduce_batch(const uint4 (&v)[U], typename Elem<DT>::packed_t (&q)[U])
 {
     typedef Elem<DT> E;
-    __shared__ unsigned sT[2];
-    __shared__ Rec s_warp[kThreads / 32];
-    __shared__ float2 s_soft[kThreads / 32];
-
-    const int tid = threadIdx.x;
-    const long long blk = blockIdx.x;
-    const long long row = blk / p.S;
-    const int slice = (int)(blk - row * p.S);
-    const float c = p.c;
-
-    const int lo = slice * p.L;
-    const int hi = min(p.V, lo + p.L);
-    const char *rowp = (const char *)p.logits + (size_t)row * (size_t)p.ld * E::kBytes;
-
-    // [lo, hi) = head scalars | 16-byte vectors | tail scalars
-    const uintptr_t a0 = (uintptr_t)(rowp + (size_t)lo * E::kBytes);
-    int nhead = (int)(((16 - (a0 & 15)) & 15) / E::kBytes);
-    nhead = min(nhead, max(hi - lo, 0));
-    const int vlo = lo + nhead;
-    const int nvec = max(hi - vlo, 0) / E::kVec;
-    const int tlo = vlo + nvec * E::kVec;
-    const int ntail = max(hi - tlo, 0);
-    const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
-
-    constexpr int kBatchVecs = kThreads * U;
-    const int nfull = nvec / kBatchVecs;
-    uint4 v[U];
-    typename E::packed_t q[U];
-
-    float bm = (nfull > 0) ? load_batch<DT, U, false>(vbase, tid, nvec, v, q)
-                           : load_batch<DT, U, true>(vbase, tid, nvec, v, q);
-    if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
-    __syncthreads();
-
-    Rec s = empty_rec();
-    float ref = -INFINITY, sum = 0.0f;
-    if (tid < nhead) {
-        const float x = E::scalar(rowp, lo + tid);
-        insert<false>(s, x, lo + tid, sT);
-        soft_add_scalar(ref, sum, x, c);
-    }
-    {   // bootstrap of the shared runner-up bound from the first batch's maxima
-        float a1 = (bm == bm) ? bm : -INFINITY, a2 = -INFINITY;
 #pragma unroll
-        for (int m = 16; m > 0; m >>= 1) {
-            float b1 = __shfl_xor_sync(0xffffffffu, a1, m), b2 = __shfl_xor_sync(0xffffffffu, a2, m);
-            a2 = fmaxf(fminf(a1, b1), fmaxf(a2, b2));
-            a1 = fmaxf(a1, b1);
-        }
-        if ((tid & 31) == 0) { publish(sT, a1); publish(sT, a2); }
-        __syncwarp();
-    }
-    float T2 = dec(*(volatile unsigned *)&sT[1]);
-    soft_batch<DT, U>(v, bm, c, ref, sum);
-    process_batch<DT, U, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
-
-    for (int bi = 1; bi < nfull; ++bi) {
-        bm = load_batch<DT, U, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
-        T2 = dec(*(volatile unsigned *)&sT[1]);
-        soft_batch<DT, U>(v, bm, c, ref, sum);
-        process_batch<DT, U, true>(v, q, bm, T2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
-    }
-    if (nfull > 0 && nfull * kBatchVecs < nvec) {
-        bm = load_batch<DT, U, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
-        T2 = dec(*(volatile unsigned *)&sT[1]);
-        soft_batch<DT, U>(v, bm, c, ref, sum);
-        process_batch<DT, U, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
-    }
-    if (tid < ntail) {
-        const float x = E::scalar(rowp, tlo + tid);
-        insert<false>(s, x, tlo + tid, sT);
-        soft_add_scalar(ref, sum, x, c);
-    }
-
-    // ---- block merge: top-2 under the total order, (ref, sum) by rescaling ----
+    for (int u = 0; u < U; ++u) q[u] = E::vred(v[u]);
+    typename E::packed_t m[U / 2];
 #pragma unroll
-    for (int m = 16; m > 0; m >>= 1) {
-        s = merge(s, shfl_xor_rec(s, m));
-        const float rb = __shfl_xor_sync(0xffffffffu, ref, m), sb = __shfl_xor_sync(0xffffffffu, sum, m);
-        soft_merge(ref, sum, rb, sb);
-    }
-    if ((tid & 31) == 0) { s_warp[tid >> 5] = s; s_soft[tid >> 5] = make_float2(ref, sum); }
-    __syncthreads();
-    if (tid == 0) {
-        Rec r = s_warp[0];
-        float rr = s_soft[0].x, ss = s_soft[0].y;
+    for (int u = 0; u < U / 2; ++u) m[u] = E::pmax(q[2 * u], q[2 * u + 1]);
 #pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) {
-            r = merge(r, s_warp[w]);
-            soft_merge(rr, ss, s_soft[w].x, s_soft[w].y);
-        }
-        SRec o;
-        o.z1 = r.z1; o.id1 = r.id1; o.z2 = r.z2; o.id2 = r.id2; o.ref = rr; o.sum = ss; o.pad0 = 0; o.pad1 = 0;
-        p.partial[blk] = o;
-    }
+    for (int w = U / 4; w > 0; w >>= 1)
+#pragma unroll
+        for (int u = 0; u < w; ++u) m[u] = E::pmax(m[u], m[u + w]);
+    return E::to_float(m[0]);
 }
 
-// ------------------------------------------------------------------------------- tail
-
-constexpr int kTailThreads = 512;
-constexpr int kTailWarps = kTailThreads / 32;
+// ------------------------------------------------------------------- per-sequence tail
 
 struct StochTailParams {
     const void *logits;
@@ -246,26 +191,42 @@ __host__ __device__ inline size_t stoch_tail_smem_bytes(int N)
     return (size_t)N * (9 * 4 + 2) + 64;
 }
 
-// Weights 2^(z*c - ref) of the kVec elements that `lane` owns in 32-lane tile `tile` of a row
-// (element j0 = (tile*32 + lane)*kVec onwards), zero beyond V and for removed tokens.
+// The kVec logits that `lane` owns in 32-lane tile `tile` of a row (element j0 = (tile*32 +
+// lane)*kVec onwards) as one 16-byte vector; elements beyond V read as -inf.  Rows that are not
+// 16-byte aligned, and the last partial vector, are gathered element by element.
 template <int DT>
-__device__ __forceinline__ void tile_weights(const char *rowp, bool aligned, int V, long long tile, int lane,
-                                             float c, float nref, const int32_t *removed, int nrem,
-                                             float (&w)[Elem<DT>::kVec])
+__device__ __forceinline__ uint4 tile_load(const char *rowp, bool aligned, int V, long long tile, int lane)
 {
     typedef Elem<DT> E;
     const long long j0 = (tile * 32 + lane) * E::kVec;
-    if (aligned && j0 + E::kVec <= V) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)j0 * E::kBytes));
+    if (aligned && j0 + E::kVec <= V) return __ldg(reinterpret_cast<const uint4 *>(rowp + (size_t)j0 * E::kBytes));
+    uint32_t wds[4];
+    if (DT == MARS_BF16) {
+        const unsigned short *r = reinterpret_cast<const unsigned short *>(rowp);
 #pragma unroll
-        for (int k = 0; k < E::kVec; ++k) w[k] = E::elem(v, k);
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t lo = (j0 + 2 * k < V) ? r[j0 + 2 * k] : 0xff80u;
+            const uint32_t hi = (j0 + 2 * k + 1 < V) ? r[j0 + 2 * k + 1] : 0xff80u;
+            wds[k] = lo | (hi << 16);
+        }
     } else {
+        const uint32_t *r = reinterpret_cast<const uint32_t *>(rowp);
 #pragma unroll
-        for (int k = 0; k < E::kVec; ++k) w[k] = (j0 + k < V) ? E::scalar(rowp, (int)(j0 + k)) : -INFINITY;
+        for (int k = 0; k < 4; ++k) wds[k] = (j0 + k < V) ? r[j0 + k] : 0xff800000u;
     }
+    return make_uint4(wds[0], wds[1], wds[2], wds[3]);
+}
+
+// Weights 2^(z*c - ref) of those elements, zero for NaN / -inf logits and for removed tokens.
+template <int DT>
+__device__ __forceinline__ void tile_weights(const uint4 &raw, long long tile, int lane, float c, float nref,
+                                             const int32_t *removed, int nrem, float (&w)[Elem<DT>::kVec])
+{
+    typedef Elem<DT> E;
+    const long long j0 = (tile * 32 + lane) * E::kVec;
 #pragma unroll
     for (int k = 0; k < E::kVec; ++k) {
-        const float x = w[k];
+        const float x = E::elem(raw, k);
         const float t = fmaf(x, c, nref);
         w[k] = (x == x && t == t) ? ex2f(t) : 0.0f;
     }
@@ -278,14 +239,28 @@ __device__ __forceinline__ void tile_weights(const char *rowp, bool aligned, int
     }
 }
 
+// Sum of one lane's weights in a tile.
 template <int DT>
-__global__ void __launch_bounds__(kTailThreads, 1) stoch_tail_kernel(const StochTailParams p)
+__device__ __forceinline__ float tile_lane_sum(const uint4 &raw, long long tile, int lane, float c, float nref,
+                                               const int32_t *removed, int nrem)
+{
+    float w[Elem<DT>::kVec];
+    tile_weights<DT>(raw, tile, lane, c, nref, removed, nrem, w);
+    float ls = 0.0f;
+#pragma unroll
+    for (int k = 0; k < Elem<DT>::kVec; ++k) ls += w[k];
+    return ls;
+}
+
+// The per-sequence tail, run by all NT threads of one block once every record of sequence b is
+// in global memory.  smem_dyn must provide stoch_tail_smem_bytes(N) bytes, 16-byte aligned.
+template <int DT, int NT>
+__device__ void stoch_tail(const StochTailParams &p, int b, unsigned char *smem_dyn)
 {
     typedef Elem<DT> E;
-    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    constexpr int kTailThreads = NT, kTailWarps = NT / 32;
     const int N = p.N, V = p.V, S = p.S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.x;
 
     int32_t *s_id1 = reinterpret_cast<int32_t *>(smem_dyn);
     int32_t *s_id2 = s_id1 + N;
@@ -421,13 +396,18 @@ __global__ void __launch_bounds__(kTailThreads, 1) stoch_tail_kernel(const Stoch
             const long long len = (t1 - t0 + kTailWarps - 1) / kTailWarps;
             const long long w0 = min(t1, t0 + warp * len), w1 = min(t1, w0 + len);
             double acc = 0.0;
-            for (long long t = w0; t < w1; ++t) {
-                float w[E::kVec];
-                tile_weights<DT>(rowp, aligned, V, t, lane, p.c, nref, s_removed, nrem, w);
-                float ls = 0.0f;
+            long long t = w0;
+            for (; t + 8 <= w1; t += 8) {   // eight independent 16-byte loads in flight per lane
+                uint4 raw[8];
 #pragma unroll
-                for (int k = 0; k < E::kVec; ++k) ls += w[k];
-                acc += (double)ls;
+                for (int i = 0; i < 8; ++i) raw[i] = tile_load<DT>(rowp, aligned, V, t + i, lane);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    acc += (double)tile_lane_sum<DT>(raw[i], t + i, lane, p.c, nref, s_removed, nrem);
+            }
+            for (; t < w1; ++t) {
+                const uint4 raw = tile_load<DT>(rowp, aligned, V, t, lane);
+                acc += (double)tile_lane_sum<DT>(raw, t, lane, p.c, nref, s_removed, nrem);
             }
 #pragma unroll
             for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
@@ -470,7 +450,7 @@ __global__ void __launch_bounds__(kTailThreads, 1) stoch_tail_kernel(const Stoch
         if (ok && warp == 0) {
             // one tile left: lane prefix, then the element inside the lane
             float w[E::kVec];
-            tile_weights<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem, w);
+            tile_weights<DT>(tile_load<DT>(rowp, aligned, V, t0, lane), t0, lane, p.c, nref, s_removed, nrem, w);
             double ls = 0.0;
 #pragma unroll
             for (int k = 0; k < E::kVec; ++k) ls += (double)w[k];
@@ -517,6 +497,148 @@ __global__ void __launch_bounds__(kTailThreads, 1) stoch_tail_kernel(const Stoch
     }
     if (p.node_how)
         for (int i = tid; i < N; i += kTailThreads) p.node_how[(size_t)b * N + i] = s_how[i];
+}
+
+// ------------------------------------------------------------------------ streaming kernel
+
+struct StreamParams {
+    const void *logits;
+    long long ld;
+    int V;
+    int S;       // slices per row
+    int L;       // elements per slice (multiple of 16)
+    float c;     // log2(e) / T
+    SRec *partial;   // [R*S]
+};
+
+template <int DT, int U, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const StreamParams p)
+{
+    typedef Elem<DT> E;
+    __shared__ unsigned sT[2];
+    __shared__ Rec s_warp[kThreads / 32];
+    __shared__ float2 s_soft[kThreads / 32];
+
+    const int tid = threadIdx.x;
+    const long long blk = blockIdx.x;
+    const long long row = blk / p.S;
+    const int slice = (int)(blk - row * p.S);
+    const float c = p.c;
+
+    const int lo = slice * p.L;
+    const int hi = min(p.V, lo + p.L);
+    const char *rowp = (const char *)p.logits + (size_t)row * (size_t)p.ld * E::kBytes;
+
+    // [lo, hi) = head scalars | 16-byte vectors | tail scalars
+    const uintptr_t a0 = (uintptr_t)(rowp + (size_t)lo * E::kBytes);
+    int nhead = (int)(((16 - (a0 & 15)) & 15) / E::kBytes);
+    nhead = min(nhead, max(hi - lo, 0));
+    const int vlo = lo + nhead;
+    const int nvec = max(hi - vlo, 0) / E::kVec;
+    const int tlo = vlo + nvec * E::kVec;
+    const int ntail = max(hi - tlo, 0);
+    const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
+
+    constexpr int kBatchVecs = kThreads * U;
+    const int nfull = nvec / kBatchVecs;
+    uint4 v[U];
+    typename E::packed_t q[U];
+
+    float bm = (nfull > 0) ? load_batch<DT, U, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, U, true>(vbase, tid, nvec, v, q);
+    if (tid == 0) { sT[0] = enc(-INFINITY); sT[1] = enc(-INFINITY); }
+    __syncthreads();
+
+    Rec s = empty_rec();
+    float ref = -INFINITY, sum = 0.0f;
+    if (tid < nhead) {
+        const float x = E::scalar(rowp, lo + tid);
+        insert<false>(s, x, lo + tid, sT);
+        soft_add_scalar(ref, sum, x, c);
+    }
+    {   // bootstrap of the shared runner-up bound from the first batch's maxima
+        float a1 = (bm == bm) ? bm : -INFINITY, a2 = -INFINITY;
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) {
+            float b1 = __shfl_xor_sync(0xffffffffu, a1, m), b2 = __shfl_xor_sync(0xffffffffu, a2, m);
+            a2 = fmaxf(fminf(a1, b1), fmaxf(a2, b2));
+            a1 = fmaxf(a1, b1);
+        }
+        if ((tid & 31) == 0) { publish(sT, a1); publish(sT, a2); }
+        __syncwarp();
+    }
+    float T2 = dec(*(volatile unsigned *)&sT[1]);
+    soft_batch<DT, U>(v, bm, c, ref, sum, vbase, tid, nvec);
+    process_batch<DT, U, false>(v, q, bm, T2, vlo + tid * E::kVec, s, sT);
+
+    // ---- steady state: two register buffers; the loads of batch bi+1 are issued before batch
+    // bi is worked on, so memory latency overlaps the exponentials ----
+    {
+        uint4 vb[U];
+        auto consume = [&](const uint4 (&x)[U], int bi) {
+            const float m = reduce_batch<DT, U>(x, q);
+            const float t2 = dec(*(volatile unsigned *)&sT[1]);
+            soft_batch<DT, U>(x, m, c, ref, sum, vbase, bi * kBatchVecs + tid, nvec);
+            process_batch<DT, U, true>(x, q, m, t2, vlo + (bi * kBatchVecs + tid) * E::kVec, s, sT);
+        };
+        int bi = 1;
+        if (bi < nfull) issue_batch<U>(vbase, bi * kBatchVecs + tid, vb);
+        while (bi < nfull) {
+            if (bi + 1 < nfull) issue_batch<U>(vbase, (bi + 1) * kBatchVecs + tid, v);
+            consume(vb, bi);
+            if (++bi >= nfull) break;
+            if (bi + 1 < nfull) issue_batch<U>(vbase, (bi + 1) * kBatchVecs + tid, vb);
+            consume(v, bi);
+            ++bi;
+        }
+    }
+    if (nfull > 0 && nfull * kBatchVecs < nvec) {
+        bm = load_batch<DT, U, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        T2 = dec(*(volatile unsigned *)&sT[1]);
+        soft_batch<DT, U>(v, bm, c, ref, sum, vbase, nfull * kBatchVecs + tid, nvec);
+        process_batch<DT, U, true>(v, q, bm, T2, vlo + (nfull * kBatchVecs + tid) * E::kVec, s, sT);
+    }
+    if (tid < ntail) {
+        const float x = E::scalar(rowp, tlo + tid);
+        insert<false>(s, x, tlo + tid, sT);
+        soft_add_scalar(ref, sum, x, c);
+    }
+
+    // ---- block merge: top-2 under the total order, (ref, sum) by rescaling ----
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        s = merge(s, shfl_xor_rec(s, m));
+        const float rb = __shfl_xor_sync(0xffffffffu, ref, m), sb = __shfl_xor_sync(0xffffffffu, sum, m);
+        soft_merge(ref, sum, rb, sb);
+    }
+    if ((tid & 31) == 0) { s_warp[tid >> 5] = s; s_soft[tid >> 5] = make_float2(ref, sum); }
+    __syncthreads();
+    if (tid == 0) {
+        Rec r = s_warp[0];
+        float rr = s_soft[0].x, ss = s_soft[0].y;
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) {
+            r = merge(r, s_warp[w]);
+            soft_merge(rr, ss, s_soft[w].x, s_soft[w].y);
+        }
+        SRec o;
+        o.z1 = r.z1; o.id1 = r.id1; o.z2 = r.z2; o.id2 = r.id2; o.ref = rr; o.sum = ss; o.pad0 = 0; o.pad1 = 0;
+        p.partial[blk] = o;
+    }
+}
+
+// One block per sequence, launched behind the streaming kernel on the same stream.  (Running
+// the tail inside the streaming kernel, by the block that delivers a sequence's last record as
+// the deterministic path does, was measured and lost 20 %: the tail's registers and its
+// 30 us of latency-bound work do not fit a kernel tuned to keep 64 registers and four blocks
+// per SM streaming.)
+constexpr int kTailThreads = 512;
+
+template <int DT>
+__global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const StochTailParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    stoch_tail<DT, kTailThreads>(p, (int)blockIdx.x, smem_dyn);
 }
 
 // ------------------------------------------------------------------------------- host
@@ -568,26 +690,15 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     sp1.logits = logits; sp1.ld = ld; sp1.V = V; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
     sp1.partial = (SRec *)workspace;
     const unsigned grid = (unsigned)(R * sp.S);
-    // Launch shape: bf16 is bound by the exponential unit and runs best with short batches and
-    // many resident warps (4 vectors per batch, 6 blocks per SM); fp32 has half the elements
-    // per byte and keeps the deterministic path's shape (8 vectors, 4 blocks per SM).
-    // MARS_STOCH_VARIANT (test / tuning hook) forces one of the four instantiations.
-    const char *var = getenv("MARS_STOCH_VARIANT");
-    const int variant = var ? atoi(var) : (dt == MARS_BF16 ? 3 : 1);
-#define MARS_STOCH_LAUNCH(DT)                                                                    \
-    switch (variant) {                                                                           \
-    case 0: stoch_stream_kernel<DT, 8, 3><<<grid, kThreads, 0, st>>>(sp1); break;                \
-    case 1: stoch_stream_kernel<DT, 8, 4><<<grid, kThreads, 0, st>>>(sp1); break;                \
-    case 2: stoch_stream_kernel<DT, 4, 4><<<grid, kThreads, 0, st>>>(sp1); break;                \
-    default: stoch_stream_kernel<DT, 4, 6><<<grid, kThreads, 0, st>>>(sp1); break;               \
-    }
-    if (dt == MARS_BF16) { MARS_STOCH_LAUNCH(MARS_BF16) } else { MARS_STOCH_LAUNCH(MARS_FP32) }
-#undef MARS_STOCH_LAUNCH
+    // 4 vectors per batch in two register buffers, 4 blocks per SM (64 registers): measured
+    // best for both dtypes; 5 or 6 blocks per SM spill the second buffer and run at half speed.
+    if (dt == MARS_BF16) stoch_stream_kernel<MARS_BF16, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
+    else stoch_stream_kernel<MARS_FP32, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
     if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
 
     StochTailParams tp;
     tp.logits = logits; tp.ld = ld; tp.V = V; tp.N = N; tp.S = sp.S; tp.c = (float)cd; tp.theta = theta;
-    tp.flags = flags; tp.chain = chain; tp.Dcap = Dcap; tp.partial = (const SRec *)workspace;
+    tp.flags = flags; tp.chain = chain; tp.Dcap = Dcap; tp.partial = sp1.partial;
     tp.tok = tok; tp.parent = parent; tp.uniform = uniform;
     tp.accept_len = accept_len; tp.out_tokens = out_tokens; tp.path_nodes = path_nodes;
     tp.out_len = out_len; tp.seq_status = seq_status; tp.node_prob = node_prob; tp.node_how = node_how;

@@ -38,7 +38,6 @@ STATS = {"close": 0, "draw_neighbour": 0, "sequences": 0, "max_draw_dist": 0.0}
 @pytest.fixture(autouse=True)
 def _no_hooks(monkeypatch):
     monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
-    monkeypatch.delenv("MARS_STOCH_VARIANT", raising=False)
 
 
 def check_walk_is_valid(got, tok, parent, b):
@@ -214,15 +213,6 @@ def test_forced_row_splits(split, monkeypatch):
     run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.3, what=f"split {split}")
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3])
-def test_every_instantiation_of_the_streaming_kernel(variant, monkeypatch):
-    monkeypatch.setenv("MARS_STOCH_VARIANT", str(variant))
-    for dtype in (torch.float32, torch.bfloat16):
-        w = synth.tree_workload("t", 8, 10, 3, 3, 40000, dtype, DEV, 55, 0.9, 1.0, 6.0, 9.0, 0.4)
-        u = synth.make_uniforms(w.B, w.N, 55)
-        run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.0, what=f"variant {variant} {dtype}")
-
-
 def test_tiny_vocabularies_one_tile():
     for V in (2, 3, 9, 200, 257):
         w = synth.tree_workload("t", 40, 6, 2, 3, V, torch.float32, DEV, 60 + V, 0.9, 1.0, 2.0, 3.0, 0.4)
@@ -244,13 +234,16 @@ def test_special_nodes_duplicates_padding_and_out_of_range_ids():
         assert (got["node_how"][:, 7] == 0).all() and (got["node_prob"][:, 9] == 0).all()
 
 
-def test_degenerate_rows_bad_trees_and_depth_cap():
-    V = 5000
-    w = synth.tree_workload("t", 6, 8, 3, 2, V, torch.float32, DEV, 80, 0.9, 1.0, 5.0, 8.0, 0.4)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_degenerate_rows_bad_trees_and_depth_cap(dtype):
+    V = 50000
+    w = synth.tree_workload("t", 6, 8, 3, 2, V, dtype, DEV, 80, 0.9, 1.0, 5.0, 8.0, 0.4)
     lg = w.logits.clone()
     lg[0 * 8 + 0, :] = float("-inf")                 # sequence 0: root row without a distribution
     lg[1 * 8 + 0, 17] = float("inf")                 # sequence 1: +inf logit
     lg[2 * 8 + 0, 100:200] = float("nan")            # sequence 2: NaNs count as -inf, still fine
+    lg[2 * 8 + 0, 30000::997] = float("nan")
+    lg[4 * 8 + 1, 7::3] = float("-inf")              # sequence 4: a third of a row at -inf
     parent = w.parent.copy()
     parent[3, 4] = 6                                 # sequence 3: malformed tree
     u = synth.make_uniforms(w.B, w.N, 80)
@@ -268,6 +261,20 @@ def test_rule_variants_and_sign_flag_pass_through():
     u = synth.make_uniforms(w.B, w.N, 90)
     for flags, theta in ((mars.RULE_MARGIN, 0.75), (mars.RULE_PROB_RATIO, 0.4), (mars.SIGN_LITERAL, 0.9)):
         run_and_compare(w.logits, w.tok, w.parent, u, theta, 1.0, flags, what=f"flags {flags}")
+
+
+def test_repeated_calls_on_one_workspace():
+    """The workspace needs no initialisation and may be reused by later calls."""
+    w = synth.cfg3(DEV, B=6)
+    u = synth.make_uniforms(w.B, w.N, 8)
+    ws = torch.full((int(mars.lib().mars_stochastic_workspace_bytes(w.B, w.N, w.V, mars.BF16)),), 0xAB,
+                    dtype=torch.uint8, device=DEV)
+    first = mars.to_host(mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, debug=True))
+    for _ in range(3):
+        again = mars.to_host(mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, debug=True,
+                                                         workspace=ws))
+        for k in first:
+            assert np.array_equal(first[k], again[k]), k
 
 
 def test_plain_mode_preserves_the_target_distribution_on_the_gpu():
