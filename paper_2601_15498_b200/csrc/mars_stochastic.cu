@@ -25,6 +25,8 @@
 //       and the running target in fp64, so that the pick depends on the weights alone).
 #include "mars_top2_stream.cuh"
 
+#include <cooperative_groups.h>
+
 #include <cmath>
 
 #include "mars.h"
@@ -252,13 +254,92 @@ __device__ __forceinline__ float tile_lane_sum(const uint4 &raw, long long tile,
     return ls;
 }
 
-// The per-sequence tail, run by all NT threads of one block once every record of sequence b is
-// in global memory.  smem_dyn must provide stoch_tail_smem_bytes(N) bytes, 16-byte aligned.
-template <int DT, int NT>
-__device__ void stoch_tail(const StochTailParams &p, int b, unsigned char *smem_dyn)
+// ---- the per-sequence tail kernel ---------------------------------------------------------
+//
+// One thread-block cluster per sequence: a single block when the batch alone fills the GPU, up to
+// eight blocks when it does not, so that a lone sequence's draw still reads its row with eight
+// SMs.  Every block of a cluster prepares and walks the tree redundantly (the walk is
+// deterministic and cheap); the draw's pass over the row is shared: block r sums tiles
+// [r*tpc, (r+1)*tpc) into per-tile sums in ITS shared memory, and after a cluster barrier the
+// leader scans all of them through distributed shared memory, finds the tile that holds u*W
+// and resolves the element.  Rows with more tiles than the per-block table holds (|V| above
+// 262 144 bf16 / 131 072 fp32 logits) take the table-free multi-level search in one block.
+constexpr int kTailThreads = 512;
+constexpr int kTailWarps = kTailThreads / 32;
+constexpr int kMaxTilesPerBlock = 1024;   // per-tile sums kept in shared memory (8 KB)
+constexpr int kTailCluster = 8;
+
+struct TailShared {
+    double tile[kMaxTilesPerBlock];
+    double part[kTailWarps];
+    double wtot[kTailWarps];
+    int whit[kTailWarps];
+    double target;
+    long long range[2];
+    int ctl[8];       // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token, 6 last tile with mass
+    int pick_tile;
+};
+
+// Element inside one tile (warp-wide): lane prefix, then the element inside the lane.  `target` is
+// the mass that lies before the wanted element within the tile, or, with whole_row, the tile is the
+// whole row and the target is u * (its total).  Returns false if the tile holds no mass.
+template <int DT>
+__device__ __forceinline__ bool draw_in_tile(const char *rowp, bool aligned, int V, long long t0, int lane,
+                                             float c, float nref, const int32_t *removed, int nrem,
+                                             double target, bool whole_row, float u, int *picked)
 {
     typedef Elem<DT> E;
-    constexpr int kTailThreads = NT, kTailWarps = NT / 32;
+    float w[E::kVec];
+    tile_weights<DT>(tile_load<DT>(rowp, aligned, V, t0, lane), t0, lane, c, nref, removed, nrem, w);
+    double ls = 0.0;
+#pragma unroll
+    for (int k = 0; k < E::kVec; ++k) ls += (double)w[k];
+    double inc = ls;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const double o = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m) inc += o;
+    }
+    const double total = __shfl_sync(0xffffffffu, inc, 31);
+    bool good = true;
+    if (whole_row) {
+        good = (total > 0.0 && total < (double)INFINITY);
+        target = (double)u * total;
+    }
+    // the first lane WITH mass whose inclusive prefix passes the target (a warp scan of floating-
+    // point numbers need not be monotone to the last bit, hence the explicit conditions)
+    const unsigned hit = __ballot_sync(0xffffffffu, inc > target && ls > 0.0);
+    const unsigned pos = __ballot_sync(0xffffffffu, ls > 0.0);
+    const int src = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
+    if (!good || src < 0) return false;
+    if (lane == src) {
+        const double tl = fmax(target - (inc - ls), 0.0);
+        int pick = -1, lastpos = -1;
+        double cum = 0.0;
+#pragma unroll
+        for (int k = 0; k < E::kVec; ++k) {
+            if (w[k] > 0.0f) lastpos = k;
+            cum += (double)w[k];
+            if (pick < 0 && cum > tl) pick = k;
+        }
+        if (pick < 0) pick = lastpos;
+        *picked = (int)((t0 * 32 + lane) * E::kVec) + pick;
+    }
+    return true;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const StochTailParams p)
+{
+    typedef Elem<DT> E;
+    namespace cg = cooperative_groups;
+    extern __shared__ __align__(16) unsigned char smem_dyn[];
+    __shared__ TailShared sh;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int G = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const bool leader = rank == 0;
+    const int b = (int)(blockIdx.x / G);
     const int N = p.N, V = p.V, S = p.S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -274,25 +355,26 @@ __device__ void stoch_tail(const StochTailParams &p, int b, unsigned char *smem_
     unsigned char *s_relax = reinterpret_cast<unsigned char *>(s_u + N);
     unsigned char *s_how = s_relax + N;
 
-    __shared__ double s_part[kTailWarps];
-    __shared__ int s_ctl[8];     // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token
-    __shared__ double s_target;
-    __shared__ long long s_range[2];
-
+    // ---- rows: merge the slice records (four records' loads in flight at a time) ----
     const int32_t *par_g = p.chain ? nullptr : ((p.flags & MARS_SHARED_PARENT) ? p.parent : p.parent + (size_t)b * N);
     int bad = 0;
     for (int i = tid; i < N; i += kTailThreads) {
-        // merge the row's slice records
-        const SRec *src = p.partial + ((size_t)b * N + i) * S;
+        const int4 *src = reinterpret_cast<const int4 *>(p.partial + ((size_t)b * N + i) * S);
         Rec acc = empty_rec();
         float ref = -INFINITY, sum = 0.0f;
-        for (int k = 0; k < S; ++k) {
-            const int4 a = __ldcg(reinterpret_cast<const int4 *>(src + k));
-            const int4 bq = __ldcg(reinterpret_cast<const int4 *>(src + k) + 1);
-            Rec r;
-            r.z1 = __int_as_float(a.x); r.id1 = a.y; r.z2 = __int_as_float(a.z); r.id2 = a.w;
-            acc = merge(acc, r);
-            soft_merge(ref, sum, __int_as_float(bq.x), __int_as_float(bq.y));
+        for (int k0 = 0; k0 < S; k0 += 4) {
+            int4 a[4], q[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k0 + j < S) { a[j] = __ldcg(src + 2 * (k0 + j)); q[j] = __ldcg(src + 2 * (k0 + j) + 1); }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k0 + j < S) {
+                    Rec r;
+                    r.z1 = __int_as_float(a[j].x); r.id1 = a[j].y; r.z2 = __int_as_float(a[j].z); r.id2 = a[j].w;
+                    acc = merge(acc, r);
+                    soft_merge(ref, sum, __int_as_float(q[j].x), __int_as_float(q[j].y));
+                }
         }
         acc = finish_record(acc);
         s_id1[i] = acc.id1;
@@ -331,65 +413,171 @@ __device__ void stoch_tail(const StochTailParams &p, int b, unsigned char *smem_
             }
         }
         s_e[i] = e;
-        if (p.node_prob) p.node_prob[(size_t)b * N + i] = prob;
+        if (leader && p.node_prob) p.node_prob[(size_t)b * N + i] = prob;
     }
     __syncthreads();
 
-    // ---- the walk (one thread; at most N node visits) ----
-    if (tid == 0) {
+    // ---- the walk: warp 0; the children of the current node are found 32 nodes at a time with a
+    // ballot and judged in node order; every lane carries the same state ----
+    const int Wd = p.Dcap + 1;
+    int32_t *o_tok = p.out_tokens + (size_t)b * Wd;
+    int32_t *o_path = p.path_nodes ? p.path_nodes + (size_t)b * Wd : nullptr;
+    if (warp == 0) {
         int cur = 0, a = 0, status = bad ? 1 : 0, nrem = 0, draw = 0;
-        const int W = p.Dcap + 1;
-        int32_t *o_tok = p.out_tokens + (size_t)b * W;
-        int32_t *o_path = p.path_nodes ? p.path_nodes + (size_t)b * W : nullptr;
-        for (int k = 0; k < W; ++k) { o_tok[k] = -1; if (o_path) o_path[k] = -1; }
-        if (o_path) o_path[0] = 0;
+        if (leader) {
+            for (int k = lane; k < Wd; k += 32) { o_tok[k] = -1; if (o_path) o_path[k] = (k == 0) ? 0 : -1; }
+        }
         while (status == 0) {
             const float ref = s_ref[cur], sum = s_sum[cur];
             nrem = 0;
             if (!(ref > -INFINITY && ref < INFINITY && sum > 0.0f && sum < INFINITY)) { status = 4; break; }
             float rem = sum;
             int next = -1;
-            for (int i = cur + 1; i < N && next < 0; ++i) {
-                if (s_par[i] != cur || s_tok[i] < 0) continue;
-                const int x = s_tok[i];
-                bool gone = false;
-                for (int k = 0; k < nrem; ++k) gone |= (s_removed[k] == x);
-                const float ex = gone ? 0.0f : s_e[i];
-                int how = 0;
-                if (!(p.flags & MARS_STOCH_PLAIN)) {
-                    if (x == s_id1[cur]) how = (p.flags & MARS_STOCH_RELAX_ONLY) ? 0 : 1;
-                    else if (x == s_id2[cur] && s_relax[cur]) how = 2;
+            const int id1 = s_id1[cur], id2 = s_id2[cur], rlx = s_relax[cur];
+            for (int base = cur + 1; base < N && next < 0; base += 32) {
+                const int i = base + lane;
+                unsigned kids = __ballot_sync(0xffffffffu, i < N && s_par[i] == cur && s_tok[i] >= 0);
+                while (kids && next < 0) {
+                    const int j = base + __ffs(kids) - 1;
+                    kids &= kids - 1;
+                    const int x = s_tok[j];
+                    bool gone = false;
+                    for (int k = 0; k < nrem; ++k) gone |= (s_removed[k] == x);
+                    const float ex = gone ? 0.0f : s_e[j];
+                    int how = 0;
+                    if (!(p.flags & MARS_STOCH_PLAIN)) {
+                        if (x == id1) how = (p.flags & MARS_STOCH_RELAX_ONLY) ? 0 : 1;
+                        else if (x == id2 && rlx) how = 2;
+                    }
+                    if (how == 0) how = (__fmul_rn(s_u[j], rem) < ex) ? 3 : 4;   // Eq. 1 on the running residual
+                    if (lane == 0) s_how[j] = (unsigned char)how;
+                    if (how == 4) {
+                        if (ex > 0.0f) {
+                            rem = fmaxf(__fsub_rn(rem, ex), 0.0f);
+                            if (lane == 0) s_removed[nrem] = x;
+                            ++nrem;
+                            __syncwarp();
+                        }
+                    } else next = j;
                 }
-                if (how == 0) how = (__fmul_rn(s_u[i], rem) < ex) ? 3 : 4;   // Eq. 1 on the running residual
-                s_how[i] = (unsigned char)how;
-                if (how == 4) {
-                    if (ex > 0.0f) { rem = fmaxf(__fsub_rn(rem, ex), 0.0f); s_removed[nrem++] = x; }
-                } else next = i;
             }
             if (next < 0) { draw = 1; break; }
             cur = next; ++a;
-            if (a <= p.Dcap) { o_tok[a - 1] = s_tok[cur]; if (o_path) o_path[a] = cur; }
+            if (leader && lane == 0 && a <= p.Dcap) { o_tok[a - 1] = s_tok[cur]; if (o_path) o_path[a] = cur; }
         }
         if ((status == 0 || status == 4) && a > p.Dcap) status = 2;
         if (status == 1 || status == 2) {
-            for (int k = 0; k < W; ++k) { o_tok[k] = -1; if (o_path) o_path[k] = -1; }
-            if (o_path) o_path[0] = 0;
-            for (int i = 0; i < N; ++i) s_how[i] = 0;
+            __syncwarp();
+            if (leader)
+                for (int k = lane; k < Wd; k += 32) { o_tok[k] = -1; if (o_path) o_path[k] = (k == 0) ? 0 : -1; }
+            for (int i = lane; i < N; i += 32) s_how[i] = 0;
             cur = 0; a = 0; draw = 0; nrem = 0;
         }
-        s_ctl[0] = cur; s_ctl[1] = a; s_ctl[2] = status; s_ctl[3] = nrem; s_ctl[4] = draw;
-        s_ctl[5] = s_id1[cur];
+        if (lane == 0) {
+            sh.ctl[0] = cur; sh.ctl[1] = a; sh.ctl[2] = status; sh.ctl[3] = nrem; sh.ctl[4] = draw;
+            sh.ctl[5] = s_id1[cur]; sh.ctl[6] = -1;
+        }
     }
     __syncthreads();
 
     // ---- the next token: CDF inversion over the residual of row `cur` ----
-    const int cur = s_ctl[0];
-    if (s_ctl[4]) {
-        const int nrem = s_ctl[3];
-        const char *rowp = (const char *)p.logits + ((size_t)b * N + cur) * (size_t)p.ld * E::kBytes;
-        const bool aligned = (((uintptr_t)rowp) & 15) == 0;
-        const float nref = -s_ref[cur];
-        const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
+    const int cur = sh.ctl[0];
+    const int nrem = sh.ctl[3];
+    const char *rowp = (const char *)p.logits + ((size_t)b * N + cur) * (size_t)p.ld * E::kBytes;
+    const bool aligned = (((uintptr_t)rowp) & 15) == 0;
+    const float nref = -s_ref[cur];
+    const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
+    const long long tpc = (ntiles + G - 1) / G;          // tiles per block of the cluster
+    const bool table = tpc <= kMaxTilesPerBlock;          // the host launches clusters only if this holds
+
+    if (sh.ctl[4] && table) {
+        // (1) every block: per-tile sums of its share of the row, eight tiles per warp at a time
+        const long long t_lo = min(ntiles, (long long)rank * tpc), t_hi = min(ntiles, t_lo + tpc);
+        for (long long t = t_lo + warp * 8; t < t_hi; t += kTailWarps * 8) {
+            uint4 raw[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (t + i < t_hi) raw[i] = tile_load<DT>(rowp, aligned, V, t + i, lane);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (t + i < t_hi) {
+                    float ls = tile_lane_sum<DT>(raw[i], t + i, lane, p.c, nref, s_removed, nrem);
+#pragma unroll
+                    for (int m = 16; m > 0; m >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, m);
+                    if (lane == 0) sh.tile[t + i - t_lo] = (double)ls;
+                }
+            }
+        }
+        cluster.sync();
+        // (2) the leader: prefix over all tile sums (its own and, through distributed shared
+        // memory, the other blocks'), a contiguous chunk of tiles per thread
+        if (leader) {
+            const int chunk = (int)((ntiles + kTailThreads - 1) / kTailThreads);
+            const long long c_lo = min(ntiles, (long long)tid * chunk), c_hi = min(ntiles, c_lo + chunk);
+            auto tile_sum = [&](long long t) -> double {
+                const int owner = (int)(t / tpc);
+                const double *base = (owner == 0) ? sh.tile : cluster.map_shared_rank(sh.tile, owner);
+                return base[t - owner * tpc];
+            };
+            double mine = 0.0;
+            int lastpos = -1;
+            for (long long t = c_lo; t < c_hi; ++t) {
+                const double v = tile_sum(t);
+                if (v > 0.0) lastpos = (int)t;
+                mine += v;
+            }
+            double inc = mine;
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const double o = __shfl_up_sync(0xffffffffu, inc, m);
+                if (lane >= m) inc += o;
+            }
+            if (lane == 31) sh.wtot[warp] = inc;
+            if (lastpos >= 0) atomicMax(&sh.ctl[6], lastpos);
+            __syncthreads();
+            double before = 0.0, Wt = 0.0;
+            for (int k = 0; k < kTailWarps; ++k) { if (k < warp) before += sh.wtot[k]; Wt += sh.wtot[k]; }
+            inc += before;
+            const double target = (double)s_u[0] * Wt;
+            const bool good = (Wt > 0.0 && Wt < (double)INFINITY);
+            // the first thread WITH mass whose inclusive prefix passes the target
+            const unsigned hits = __ballot_sync(0xffffffffu, good && inc > target && mine > 0.0);
+            const double prev = __shfl_up_sync(0xffffffffu, inc, 1);
+            if (lane == 0) sh.whit[warp] = hits ? (__ffs(hits) - 1) : -1;
+            if (tid == 0) { sh.pick_tile = -1; sh.target = 0.0; if (!good) sh.ctl[2] = 4; }
+            __syncthreads();
+            int wsel = -1;
+            for (int k = kTailWarps - 1; k >= 0; --k) if (sh.whit[k] >= 0) wsel = k;
+            if (warp == wsel && lane == sh.whit[wsel]) {
+                double cum = (lane == 0) ? before : prev;
+                int last_in_chunk = -1;
+                for (long long t = c_lo; t < c_hi; ++t) {
+                    const double v = tile_sum(t);
+                    if (v > 0.0) last_in_chunk = (int)t;
+                    if (v > 0.0 && cum + v > target) { sh.pick_tile = (int)t; sh.target = fmax(target - cum, 0.0); break; }
+                    cum += v;
+                }
+                if (sh.pick_tile < 0) { sh.pick_tile = last_in_chunk; sh.target = (double)INFINITY; }
+            }
+            __syncthreads();
+            if (good && warp == 0) {
+                long long t0 = sh.pick_tile;
+                double target_in = sh.target;
+                if (t0 < 0) { t0 = sh.ctl[6]; target_in = (double)INFINITY; }   // rounding: the last tile with mass
+                int picked = -1;
+                bool ok = t0 >= 0;
+                if (ok) ok = draw_in_tile<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem, target_in,
+                                              false, 0.0f, &picked);
+                ok = __all_sync(0xffffffffu, ok);
+                const int all = __reduce_max_sync(0xffffffffu, picked);   // the resolving lane's element
+                if (lane == 0) { if (!ok || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
+            }
+            __syncthreads();
+        }
+        cluster.sync();     // the other blocks' tables stay alive until the leader has read them
+    } else if (sh.ctl[4]) {
+        // table-free search (one block): sum contiguous warp segments, descend into the segment that
+        // holds the target, repeat down to one tile
         long long t0 = 0, t1 = ntiles;
         bool first = true, ok = true;
         while (t1 - t0 > 1) {
@@ -411,91 +599,61 @@ __device__ void stoch_tail(const StochTailParams &p, int b, unsigned char *smem_
             }
 #pragma unroll
             for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
-            if (lane == 0) s_part[warp] = acc;
+            if (lane == 0) sh.part[warp] = acc;
             __syncthreads();
             if (tid == 0) {
                 double target;
                 bool good = true;
                 if (first) {
                     double Wt = 0.0;
-                    for (int k = 0; k < kTailWarps; ++k) Wt += s_part[k];
+                    for (int k = 0; k < kTailWarps; ++k) Wt += sh.part[k];
                     good = (Wt > 0.0 && Wt < (double)INFINITY);
                     target = (double)s_u[0] * Wt;
-                } else target = s_target;
+                } else target = sh.target;
                 int pick = -1, lastpos = -1;
                 double cum = 0.0, before = 0.0;
                 for (int k = 0; k < kTailWarps && pick < 0; ++k) {
-                    if (s_part[k] > 0.0) lastpos = k;
+                    if (sh.part[k] > 0.0) lastpos = k;
                     before = cum;
-                    cum += s_part[k];
+                    cum += sh.part[k];
                     if (cum > target) pick = k;
                 }
                 if (pick < 0) {   // rounding pushed the target past the total: the last part with mass
                     pick = lastpos;
                     before = 0.0;
-                    for (int k = 0; k < pick; ++k) before += s_part[k];
+                    for (int k = 0; k < pick; ++k) before += sh.part[k];
                 }
-                if (!good || pick < 0) { s_ctl[2] = 4; s_range[0] = 0; s_range[1] = 0; }
+                if (!good || pick < 0) { sh.ctl[2] = 4; sh.range[0] = 0; sh.range[1] = 0; }
                 else {
-                    s_target = fmax(target - before, 0.0);
-                    s_range[0] = min(t1, t0 + pick * len);
-                    s_range[1] = min(t1, s_range[0] + len);
+                    sh.target = fmax(target - before, 0.0);
+                    sh.range[0] = min(t1, t0 + pick * len);
+                    sh.range[1] = min(t1, sh.range[0] + len);
                 }
             }
             __syncthreads();
-            t0 = s_range[0]; t1 = s_range[1];
+            t0 = sh.range[0]; t1 = sh.range[1];
             first = false;
             if (t1 <= t0) { ok = false; break; }
         }
         if (ok && warp == 0) {
-            // one tile left: lane prefix, then the element inside the lane
-            float w[E::kVec];
-            tile_weights<DT>(tile_load<DT>(rowp, aligned, V, t0, lane), t0, lane, p.c, nref, s_removed, nrem, w);
-            double ls = 0.0;
-#pragma unroll
-            for (int k = 0; k < E::kVec; ++k) ls += (double)w[k];
-            double inc = ls;
-#pragma unroll
-            for (int m = 1; m < 32; m <<= 1) {
-                const double o = __shfl_up_sync(0xffffffffu, inc, m);
-                if (lane >= m) inc += o;
-            }
-            const double total = __shfl_sync(0xffffffffu, inc, 31);
-            double target;
-            bool good = true;
-            if (first) {   // the whole row is one tile
-                good = (total > 0.0 && total < (double)INFINITY);
-                target = (double)s_u[0] * total;
-            } else target = s_target;
-            const unsigned hit = __ballot_sync(0xffffffffu, inc > target);
-            const unsigned pos = __ballot_sync(0xffffffffu, ls > 0.0);
-            int src = hit ? (__ffs(hit) - 1) : (pos ? 31 - __clz(pos) : -1);
-            if (!good || src < 0) { if (lane == 0) s_ctl[2] = 4; }
-            else if (lane == src) {
-                const double tl = fmax(target - (inc - ls), 0.0);
-                int pick = -1, lastpos = -1;
-                double cum = 0.0;
-#pragma unroll
-                for (int k = 0; k < E::kVec; ++k) {
-                    if (w[k] > 0.0f) lastpos = k;
-                    cum += (double)w[k];
-                    if (pick < 0 && cum > tl) pick = k;
-                }
-                if (pick < 0) pick = lastpos;
-                s_ctl[5] = (int)((t0 * 32 + lane) * E::kVec) + pick;
-            }
+            int picked = -1;
+            bool fine = draw_in_tile<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem,
+                                         first ? 0.0 : sh.target, first, s_u[0], &picked);
+            fine = __all_sync(0xffffffffu, fine);
+            const int all = __reduce_max_sync(0xffffffffu, picked);
+            if (lane == 0) { if (!fine || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
         }
         __syncthreads();
     }
 
-    if (tid == 0) {
-        const int a = s_ctl[1], status = s_ctl[2];
-        p.out_tokens[(size_t)b * (p.Dcap + 1) + a] = (status == 4) ? s_id1[cur] : s_ctl[5];
+    if (leader && tid == 0) {
+        const int a = sh.ctl[1], status = sh.ctl[2];
+        p.out_tokens[(size_t)b * (p.Dcap + 1) + a] = (status == 4) ? s_id1[cur] : sh.ctl[5];
         p.accept_len[b] = a;
         p.out_len[b] = a + 1;
         if (p.seq_status) p.seq_status[b] = status;
     }
-    if (p.node_how)
+    if (leader && p.node_how)
         for (int i = tid; i < N; i += kTailThreads) p.node_how[(size_t)b * N + i] = s_how[i];
 }
 
@@ -627,19 +785,10 @@ __global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const Stre
     }
 }
 
-// One block per sequence, launched behind the streaming kernel on the same stream.  (Running
-// the tail inside the streaming kernel, by the block that delivers a sequence's last record as
-// the deterministic path does, was measured and lost 20 %: the tail's registers and its
-// 30 us of latency-bound work do not fit a kernel tuned to keep 64 registers and four blocks
-// per SM streaming.)
-constexpr int kTailThreads = 512;
-
-template <int DT>
-__global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const StochTailParams p)
-{
-    extern __shared__ __align__(16) unsigned char smem_dyn[];
-    stoch_tail<DT, kTailThreads>(p, (int)blockIdx.x, smem_dyn);
-}
+// (Running the tail inside the streaming kernel, by the block that delivers a sequence's last
+// record as the deterministic path does, was measured and lost 20 %: the tail's registers and its
+// latency-bound work do not fit a kernel tuned to keep 64 registers and four blocks per SM
+// streaming.  It is a kernel of its own, launched behind the streaming kernel on the same stream.)
 
 // ------------------------------------------------------------------------------- host
 
@@ -703,9 +852,35 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     tp.accept_len = accept_len; tp.out_tokens = out_tokens; tp.path_nodes = path_nodes;
     tp.out_len = out_len; tp.seq_status = seq_status; tp.node_prob = node_prob; tp.node_how = node_how;
     const size_t smem = stoch_tail_smem_bytes(N);
-    if (dt == MARS_BF16) stoch_tail_kernel<MARS_BF16><<<(unsigned)B, kTailThreads, smem, st>>>(tp);
-    else stoch_tail_kernel<MARS_FP32><<<(unsigned)B, kTailThreads, smem, st>>>(tp);
-    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+    // The largest cluster (8, 4, 2 blocks per sequence) that still fits the GPU in one wave (two
+    // blocks of 512 threads per SM) and leaves each block a share of the row that fits its tile
+    // table; rows too long for the table of a single block take the table-free search (G = 1).
+    const int kv = dt == MARS_BF16 ? 8 : 4;
+    const long long ntiles = ((long long)V + 32 * kv - 1) / (32 * kv);
+    int G = 1;
+    for (int g = kTailCluster; g > 1; g >>= 1)
+        if ((long long)B * g <= 2 * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
+    const char *force = getenv("MARS_STOCH_TAIL_CLUSTER");   // test hook: 1, 2, 4 or 8
+    if (force) {
+        const int g = atoi(force);
+        if ((g == 1 || g == 2 || g == 4 || g == 8) && (g == 1 || (ntiles + g - 1) / g <= kMaxTilesPerBlock)) G = g;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((long long)B * G));
+    cfg.blockDim = dim3(kTailThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)G;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16>, tp)
+                                              : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32>, tp);
+    if (err != cudaSuccess) { cudaGetLastError(); return MARS_ERR_CUDA; }
+    return MARS_OK;
 }
 
 }  // namespace mars

@@ -38,6 +38,7 @@ STATS = {"close": 0, "draw_neighbour": 0, "sequences": 0, "max_draw_dist": 0.0}
 @pytest.fixture(autouse=True)
 def _no_hooks(monkeypatch):
     monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
 
 
 def check_walk_is_valid(got, tok, parent, b):
@@ -211,6 +212,31 @@ def test_forced_row_splits(split, monkeypatch):
     w = synth.tree_workload("t", 10, 12, 3, 3, 20011, torch.bfloat16, DEV, 44, 0.9, 1.0, 6.0, 9.0, 0.4)
     u = synth.make_uniforms(w.B, w.N, 44)
     run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.3, what=f"split {split}")
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_draw_with_one_block_and_with_clusters(cluster, dtype, monkeypatch):
+    """The draw's pass over the row runs in one block or is shared by a cluster of 2, 4 or 8 blocks
+    (distributed shared memory); every shape must resolve the same element.  Many sequences stop at the
+    root (uniforms next to one), so every part of the row gets drawn from."""
+    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    w = synth.tree_workload("t", 96, 6, 2, 2, 70001, dtype, DEV, 66, 0.9, 1.0, 3.0, 6.0, 0.4)
+    u = synth.make_uniforms(w.B, w.N, 66)
+    u[::2, 1:] = np.float32(0.99999)
+    got, ref = run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.0, mars.STOCH_PLAIN, what=f"cluster {cluster}")
+    drawn = got["out_tokens"][np.arange(w.B), got["accept_len"]]
+    assert drawn.min() < w.V // 8 and drawn.max() > 7 * w.V // 8
+
+
+@pytest.mark.parametrize("dtype,V", [(torch.bfloat16, 270001), (torch.float32, 140003)])
+def test_rows_longer_than_the_tile_table(dtype, V):
+    """More 32-lane tiles than a block's table of tile sums holds: the table-free search."""
+    w = synth.tree_workload("t", 6, 4, 2, 2, V, dtype, DEV, 67, 0.9, 1.0, 3.0, 6.0, 0.4)
+    u = synth.make_uniforms(w.B, w.N, 67)
+    u[::2, 1:] = np.float32(0.99999)
+    run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.0, mars.STOCH_PLAIN, what=f"long rows {dtype}",
+                    max_close_frac=0.4)
 
 
 def test_tiny_vocabularies_one_tile():
