@@ -1,0 +1,125 @@
+"""Seeded differential fuzzing of the CUDA library against the CPU oracle: random batch shapes,
+vocabularies, row strides and alignments, thresholds, flags, padding nodes and special values
+(NaN, +-inf, equal logits), for the deterministic calls (bit-exact) and the stochastic calls
+(the tolerance policy of test_gpu_stochastic.py)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mars_oracle as orc
+from paper_2601_15498_b200 import mars, synth
+
+import stochastic_checks as ts
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def random_case(rng, stochastic: bool):
+    B = int(rng.integers(1, 24))
+    N = int(rng.choice([1, 2, 3, 5, 8, 17, 33, 64, 65, 70]))
+    V = int(rng.choice([2, 3, 7, 64, 255, 256, 257, 1000, 4096, 5001, 20000]))
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    pad = int(rng.choice([0, 0, 1, 3, 8]))
+    shift = int(rng.choice([0, 0, 1, 2, 5]))
+    ld = V + pad
+    R = B * N
+    sigma = float(rng.choice([0.5, 1.0, 3.0]))
+    z = torch.tensor(rng.normal(size=(R, V)) * sigma, dtype=torch.float32)
+    top = rng.uniform(2.0, 12.0, R)
+    ids = rng.integers(0, V, (R, 2))
+    z[torch.arange(R), torch.as_tensor(ids[:, 0])] = torch.tensor(top, dtype=torch.float32)
+    low = rng.random(R) < 0.4
+    rho = rng.uniform(0.8, 1.0, R)
+    for r in np.flatnonzero(low):
+        if ids[r, 1] != ids[r, 0]:
+            z[r, ids[r, 1]] = float(rho[r] * top[r])
+    if rng.random() < 0.5:      # coarse values: plenty of exact ties
+        z = torch.round(z * 2) / 2
+    if rng.random() < 0.4:      # special values
+        k = max(1, R * V // 50)
+        rr, cc = rng.integers(0, R, k), rng.integers(0, V, k)
+        vals = rng.choice([np.nan, -np.inf, 0.0, -0.0], k)
+        z[torch.as_tensor(rr), torch.as_tensor(cc)] = torch.tensor(vals, dtype=torch.float32)
+        if not stochastic and rng.random() < 0.3:
+            z[int(rng.integers(0, R)), int(rng.integers(0, V))] = float("inf")
+    z = z.to(dtype)
+    # device layout: [R, ld] with an element shift of the base pointer
+    flat = torch.full((R * ld + shift + 8,), 77.0, dtype=dtype, device=DEV)
+    view = torch.as_strided(flat[shift:], (R, V), (ld, 1))
+    view.copy_(z.to(DEV))
+    # tree
+    depth = int(rng.integers(1, 8))
+    parent = synth.make_parents(B, N, min(depth, max(N - 1, 0)), int(rng.integers(1, 5)), int(rng.integers(1 << 30)))
+    lead = torch.topk(z.float().nan_to_num(nan=-np.inf), min(2, V), dim=1).indices.numpy()
+    tok = synth.make_tokens(parent, lead, V, int(rng.integers(1 << 30)), p_top1=0.5, p_top2=0.3)
+    if N > 3 and rng.random() < 0.5:
+        tok[:, int(rng.integers(1, N))] = -1
+        parent[:, N - 1] = -1
+    if N > 2 and rng.random() < 0.15:
+        parent[int(rng.integers(0, B)), N - 1] = N - 1     # malformed
+    shared = rng.random() < 0.2
+    if shared:
+        parent = np.ascontiguousarray(parent[0])
+    theta = float(rng.choice([0.5, 0.8, 0.9, 0.95, 1.0, 1.5, -0.5]))
+    flags = 0
+    r = rng.random()
+    if r < 0.15:
+        flags |= mars.SIGN_LITERAL
+    elif r < 0.3:
+        flags |= mars.RULE_MARGIN
+        theta = float(rng.choice([0.25, 1.0, 3.0]))
+    elif r < 0.45:
+        flags |= mars.RULE_PROB_RATIO
+        theta = float(rng.choice([0.1, 0.5, 0.9]))
+    Dcap = N - 1 if rng.random() < 0.8 else int(rng.integers(0, max(N - 1, 1)))
+    host = synth.to_numpy_bits(z)
+    return dict(B=B, N=N, V=V, view=view, host=host, z=z, tok=tok, parent=parent, theta=theta, flags=flags,
+                Dcap=Dcap, keep=flat)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_deterministic_tree_and_chain(seed, monkeypatch):
+    rng = np.random.default_rng(1000 + seed)
+    if rng.random() < 0.3:
+        monkeypatch.setenv("MARS_FORCE_SPLIT", str(int(rng.integers(2, 6))))
+    else:
+        monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    for _ in range(4):
+        c = random_case(rng, stochastic=False)
+        got = mars.to_host(mars.verify_tree(c["view"], c["tok"], c["parent"], c["theta"], c["flags"], c["Dcap"],
+                                            debug=True))
+        ref = orc.verify_tree(c["host"], c["tok"], c["parent"], c["theta"], c["flags"], c["Dcap"])
+        for k in ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "top2_id", "node_flags"):
+            assert np.array_equal(got[k], ref[k]), (seed, k, c["B"], c["N"], c["V"])
+        assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32)), seed
+        if c["parent"].ndim == 2 and c["N"] > 1:
+            draft = np.ascontiguousarray(c["tok"][:, 1:])
+            gc = mars.to_host(mars.verify_chain(c["view"], draft, c["theta"], c["flags"], debug=True))
+            rc = orc.verify_chain(c["host"], draft, c["theta"], c["flags"])
+            for k in ("accept_len", "out_tokens", "out_len", "top2_id"):
+                assert np.array_equal(gc[k], rc[k]), (seed, "chain", k)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_stochastic_tree(seed, monkeypatch):
+    rng = np.random.default_rng(5000 + seed)
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    if rng.random() < 0.3:
+        monkeypatch.setenv("MARS_FORCE_SPLIT", str(int(rng.integers(2, 6))))
+    if rng.random() < 0.5:
+        monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(int(rng.choice([1, 2, 4, 8]))))
+    else:
+        monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+    for _ in range(3):
+        c = random_case(rng, stochastic=True)
+        T = float(rng.choice([0.3, 0.7, 1.0, 1.7]))
+        flags = c["flags"] | int(rng.choice([0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY]))
+        u = synth.make_uniforms(c["B"], c["N"], int(rng.integers(1 << 30)))
+        if rng.random() < 0.3:
+            u[:, 1:] = np.float32(0.9999)
+        got = mars.to_host(mars.verify_tree_stochastic(c["view"], c["tok"], c["parent"], u, c["theta"], T, flags,
+                                                       c["Dcap"], debug=True))
+        ref = orc.verify_tree_stochastic(c["host"], c["tok"], c["parent"], u, c["theta"], T, flags, c["Dcap"])
+        ts.compare(got, ref, c["tok"], c["parent"], c["z"].double().numpy(), u, T, f"fuzz {seed}",
+                   max_close_frac=0.25)
