@@ -623,3 +623,117 @@ void mars_oracle_verify_tree_stochastic(const void *logits, int dtype, int64_t l
         if (margin) { margin[2 * b] = mg_test; margin[2 * b + 1] = mg_draw; }
     }
 }
+
+/* ======================================================================================
+ * Stochastic verification of chains whose drafts were SAMPLED from a drafter's distribution:
+ * Eq. 1 in its general form (Sec. 2.2).  Draft i was drawn from Q_i = softmax(zq_i / Tq) with
+ * probability qx_i = Q_i(draft_i), supplied by the caller.  It is accepted with probability
+ * min(1, P_i(x) / Q_i(x)), i.e. iff u_i * Q_i(x) < P_i(x) for the position's uniform u_i (for a
+ * ratio of one or more this always holds since u_i < 1).  The first rejected position emits a
+ * token drawn from the residual distribution, which "compensates for the draft's approximation
+ * error": norm(max(0, P_i - Q_i)), by CDF inversion in token-id order with uniform[b, 0].  If
+ * every draft is accepted the bonus token is drawn from P of the last row.  The composition with
+ * the relaxation follows the same three modes as the tree form above (a reading of this
+ * repository; PARITY UNPINNED by the paper).  With STOCH_PLAIN this is standard speculative
+ * sampling, which leaves the target distribution unchanged -- the pin for this function.
+ *   logits  [B*K, ld]   target rows;  qlogits [B*(K-1), ldq] drafter rows (dtype_q);
+ *   draft   [B, K-1];   qx [B, K-1] float: probability with which the drafter drew the token;
+ *   uniform [B, K]:     [b, i+1] judges draft i, [b, 0] draws the emitted token;
+ *   node_how [B, K] as in the tree form (index i+1 for draft i); margin [B, 2] as there, with the
+ *   draw margin in units of total probability (not of the residual's mass).
+ *   Status 4: a row on the way has no softmax (target or drafter), or the residual has no mass.
+ * ==================================================================================== */
+void mars_oracle_verify_chain_sampled(const void *logits, int dtype, int64_t ld, const void *qlogits,
+                                      int dtype_q, int64_t ldq, const int32_t *draft, const float *qx,
+                                      const float *uniform, int B, int K, int64_t V, double theta,
+                                      double temperature, double draft_temperature, uint32_t flags,
+                                      int32_t *accept_len, int32_t *out_tokens, int32_t *out_len,
+                                      int32_t *status, double *node_prob, uint8_t *node_how, double *margin)
+{
+    size_t e = dtype == ORACLE_BF16 ? 2 : dtype == ORACLE_FP32 ? 4 : 8;
+    size_t eq = dtype_q == ORACLE_BF16 ? 2 : dtype_q == ORACLE_FP32 ? 4 : 8;
+    const double T = temperature, Tq = draft_temperature;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        const float *u = uniform + (size_t)b * K;
+        int32_t *otok = out_tokens + (size_t)b * K;
+        uint8_t *nhow = node_how ? node_how + (size_t)b * K : NULL;
+        double *nprob = node_prob ? node_prob + (size_t)b * K : NULL;
+        double mg_test = INFINITY, mg_draw = INFINITY;
+        fill(otok, K, -1);
+        for (int i = 0; i < K; ++i) { if (nhow) nhow[i] = 0; if (nprob) nprob[i] = 0.0; }
+        int a = 0, st = 0, rejected_at = -1;
+        float v2[2];
+        int32_t id2[2] = {0, 1};
+        double m = 0, S = 0;
+        const char *row = NULL;
+        /* plain softmax probability of every draft under its row (reported, not part of the walk) */
+        for (int i = 0; nprob && i < K - 1; ++i) {
+            int32_t x = draft[(size_t)b * (K - 1) + i];
+            row = (const char *)logits + ((size_t)b * K + i) * (size_t)ld * e;
+            row_softmax_stats(row, dtype, V, T, &m, &S);
+            if (x >= 0 && x < V && isfinite(m) && S > 0.0) nprob[i + 1] = exp((row_get(row, dtype, x) - m) / T) / S;
+        }
+        for (int i = 0; i < K; ++i) {       /* row i judges draft i; row K-1 only supplies the bonus */
+            row = (const char *)logits + ((size_t)b * K + i) * (size_t)ld * e;
+            top2_row_f32(row, dtype, V, v2, id2);
+            row_softmax_stats(row, dtype, V, T, &m, &S);
+            if (!isfinite(m) || !(S > 0.0)) { st = 4; break; }
+            if (i == K - 1) break;
+            int32_t x = draft[(size_t)b * (K - 1) + i];
+            double px = (x >= 0 && x < V) ? exp((row_get(row, dtype, x) - m) / T) / S : 0.0;
+            int relax = mars_oracle_relax_f32(v2[0], v2[1], (float)theta, flags);
+            int how = (flags & MARS_ORACLE_STOCH_PLAIN) ? 0 : rule(x, id2, relax);
+            if ((flags & MARS_ORACLE_STOCH_RELAX_ONLY) && how == 1) how = 0;
+            if (how == 0) {
+                double lhs = (double)u[i + 1] * (double)qx[(size_t)b * (K - 1) + i];   /* Eq. 1 */
+                double d = fabs(px - lhs);
+                if (d < mg_test) mg_test = d;
+                how = (x >= 0 && lhs < px) ? 3 : 4;
+            }
+            if (nhow) nhow[i + 1] = (uint8_t)how;
+            if (how == 4) { rejected_at = i; break; }
+            otok[a++] = x;
+        }
+        int32_t drawn = id2[0];
+        if (st == 0) {
+            /* weights of the distribution to draw from, in token-id order */
+            const char *qrow = NULL;
+            double mq = 0, Sq = 0;
+            if (rejected_at >= 0) {
+                qrow = (const char *)qlogits + ((size_t)b * (K - 1) + rejected_at) * (size_t)ldq * eq;
+                row_softmax_stats(qrow, dtype_q, V, Tq, &mq, &Sq);
+                if (!isfinite(mq) || !(Sq > 0.0)) st = 4;
+            }
+            if (st == 0) {
+                double W = 0.0;
+                for (int64_t j = 0; j < V; ++j) {
+                    double w = exp((row_get(row, dtype, j) - m) / T) / S;
+                    if (qrow) { w -= exp((row_get(qrow, dtype_q, j) - mq) / Tq) / Sq; if (w < 0.0) w = 0.0; }
+                    W += w;
+                }
+                if (!(W > 0.0)) st = 4;
+                else {
+                    double target = (double)u[0] * W, c = 0.0, lo = 0.0;
+                    int64_t pick = -1, last = -1;
+                    for (int64_t j = 0; j < V && pick < 0; ++j) {
+                        double w = exp((row_get(row, dtype, j) - m) / T) / S;
+                        if (qrow) { w -= exp((row_get(qrow, dtype_q, j) - mq) / Tq) / Sq; if (w < 0.0) w = 0.0; }
+                        if (w > 0.0) last = j;
+                        lo = c;
+                        c += w;
+                        if (c > target) pick = j;
+                    }
+                    if (pick < 0) pick = last;
+                    drawn = (int32_t)pick;
+                    double d0 = target - lo, d1 = c - target;
+                    mg_draw = d0 < d1 ? d0 : d1;
+                }
+            }
+        }
+        otok[a] = drawn;
+        accept_len[b] = a; out_len[b] = a + 1;
+        if (status) status[b] = st;
+        if (margin) { margin[2 * b] = mg_test; margin[2 * b + 1] = mg_draw; }
+    }
+}

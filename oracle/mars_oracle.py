@@ -74,6 +74,9 @@ def lib() -> ctypes.CDLL:
             L.mars_oracle_verify_tree_stochastic.argtypes = [vp, i32, i64, vp, vp, vp, i32, i32, i64, f64,
                                                              f64, u32, i32] + [vp] * 8
             L.mars_oracle_verify_tree_stochastic.restype = None
+            L.mars_oracle_verify_chain_sampled.argtypes = [vp, i32, i64, vp, i32, i64, vp, vp, vp, i32, i32, i64,
+                                                           f64, f64, f64, u32] + [vp] * 7
+            L.mars_oracle_verify_chain_sampled.restype = None
             _lib = L
     return _lib
 
@@ -285,4 +288,37 @@ def verify_tree_stochastic(logits, tok, parent, uniform, theta, temperature, fla
         float(temperature), flags, Dcap, _p(out["accept_len"]), _p(out["out_tokens"]),
         _p(out["path_nodes"]), _p(out["out_len"]), _p(out["seq_status"]), _p(out["node_prob"]),
         _p(out["node_how"]), _p(out["margin"]))
+    return out
+
+
+def verify_chain_sampled(logits, qlogits, draft, qx, uniform, theta, temperature, draft_temperature,
+                         flags: int = 0, V: int | None = None) -> dict:
+    """Stochastic verification of chains with sampled drafts (general Eq. 1); see mars_oracle.c.
+    logits [B*K, ld], qlogits [B*(K-1), ldq], draft / qx [B, K-1], uniform [B, K]."""
+    dt, V = _check_logits(logits, V)
+    draft = np.ascontiguousarray(draft, np.int32)
+    qx = np.ascontiguousarray(qx, np.float32)
+    uniform = np.ascontiguousarray(uniform, np.float32)
+    B, Km1 = draft.shape
+    K = Km1 + 1
+    if qlogits.ndim != 2 or not qlogits.flags.c_contiguous or qlogits.dtype not in _DT or qlogits.shape[1] < V:
+        raise ValueError("qlogits must be a C-contiguous [B*(K-1), >=V] array")
+    if logits.shape[0] != B * K or qlogits.shape[0] != B * Km1 or qx.shape != (B, Km1) or uniform.shape != (B, K):
+        raise ValueError("shape mismatch")
+    if not (temperature > 0 and draft_temperature > 0):
+        raise ValueError("temperatures must be positive")
+    out = {
+        "accept_len": np.empty(B, np.int32),
+        "out_tokens": np.empty((B, K), np.int32),
+        "out_len": np.empty(B, np.int32),
+        "seq_status": np.empty(B, np.int32),
+        "node_prob": np.empty((B, K), np.float64),
+        "node_how": np.empty((B, K), np.uint8),
+        "margin": np.empty((B, 2), np.float64),
+    }
+    lib().mars_oracle_verify_chain_sampled(
+        _p(logits), dt, logits.shape[1], _p(qlogits), _DT[qlogits.dtype], qlogits.shape[1], _p(draft), _p(qx),
+        _p(uniform), B, K, V, float(theta), float(temperature), float(draft_temperature), flags,
+        _p(out["accept_len"]), _p(out["out_tokens"]), _p(out["out_len"]), _p(out["seq_status"]),
+        _p(out["node_prob"]), _p(out["node_how"]), _p(out["margin"]))
     return out

@@ -289,3 +289,103 @@ def test_margins_report_how_close_each_decision_was():
     # the draw at node 1 (a leaf, nothing removed): u = 0.6 falls in token 2's interval [0.5, 0.75)
     assert out["out_tokens"][0, 1] == 2
     assert out["margin"][0, 1] == pytest.approx(min(float(np.float32(0.6)) - 0.5, 0.75 - float(np.float32(0.6))), abs=1e-12)
+
+
+# ---------------------------------------------------------------- sampled drafts (general Eq. 1)
+
+def _sampled_case(seed, B, K, V, sigma_p=1.0, sigma_q=1.0, T=1.0, Tq=1.0, same_rows=True):
+    """Target and drafter rows, drafts actually sampled from the drafter's softmax (numpy), and the
+    probability with which each was drawn."""
+    rng = np.random.default_rng(seed)
+    if same_rows:
+        rows_p = (rng.normal(size=(K, V)) * sigma_p).astype(np.float32)
+        rows_q = (rows_p[:K - 1] + rng.normal(size=(K - 1, V)) * sigma_q).astype(np.float32)
+        logits = np.ascontiguousarray(np.tile(rows_p, (B, 1)))
+        qlogits = np.ascontiguousarray(np.tile(rows_q, (B, 1)))
+    else:
+        logits = (rng.normal(size=(B * K, V)) * sigma_p).astype(np.float32)
+        qlogits = (logits.reshape(B, K, V)[:, :K - 1].reshape(-1, V)
+                   + rng.normal(size=(B * (K - 1), V)) * sigma_q).astype(np.float32)
+    Q = softmax(qlogits.astype(np.float64) / Tq, axis=1)
+    cdf = np.cumsum(Q, axis=1)
+    r = rng.random(B * (K - 1))
+    draft = np.minimum((cdf < r[:, None]).sum(axis=1), V - 1).astype(np.int32)
+    qx = Q[np.arange(B * (K - 1)), draft].astype(np.float32)
+    u = rng.random((B, K)).astype(np.float32)
+    return logits, qlogits, draft.reshape(B, K - 1), qx.reshape(B, K - 1), u
+
+
+def test_sampled_drafts_plain_mode_preserves_the_target_distribution():
+    """Speculative sampling (Eq. 1 + residual) with drafts really drawn from the drafter: the
+    first emitted token follows the target's row 0 and, where draft 0 was accepted, the second
+    follows row 1 -- whatever the drafter's distribution is."""
+    V, K, B, T, Tq = 7, 3, 200_000, 0.9, 1.2
+    logits, qlogits, draft, qx, u = _sampled_case(11, B, K, V, 0.8, 0.9, T, Tq)
+    out = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, T, Tq, orc.STOCH_PLAIN)
+    assert (out["seq_status"] == 0).all()
+    P = softmax(logits[:K].astype(np.float64) / T, axis=1)
+    _freq_close(out["out_tokens"][:, 0], P[0])
+    acc0 = out["accept_len"] >= 1
+    assert 0.2 < acc0.mean() < 0.95
+    _freq_close(out["out_tokens"][acc0, 1], P[1])
+    # acceptance rate of the first draft = sum_v min(P, Q)
+    Q0 = softmax(qlogits[0].astype(np.float64) / Tq)
+    want = np.minimum(P[0], Q0).sum()
+    assert abs(acc0.mean() - want) < 4.5 * np.sqrt(want * (1 - want) / B)
+
+
+def test_sampled_drafts_with_a_point_mass_drafter_equal_the_tree_form():
+    """A drafter that puts all its mass on the draft (Q = one-hot, qx = 1) turns the general rule
+    into the point-mass form: same decisions, same drawn tokens as the tree oracle on a chain."""
+    rng = np.random.default_rng(12)
+    B, K, V = 300, 5, 40
+    logits = (rng.normal(size=(B * K, V)) * 1.5).astype(np.float32)
+    draft = rng.integers(0, V, (B, K - 1)).astype(np.int32)
+    best = logits.reshape(B, K, V)[:, :K - 1].argmax(axis=2).astype(np.int32)
+    draft = np.where(rng.random((B, K - 1)) < 0.6, best, draft)     # most drafts aim at the target's top token
+    qlogits = np.full((B * (K - 1), V), -1e4, np.float32)
+    qlogits[np.arange(B * (K - 1)), draft.reshape(-1)] = 0.0
+    qx = np.ones((B, K - 1), np.float32)
+    u = rng.random((B, K)).astype(np.float32)
+    tok = np.concatenate([np.full((B, 1), -1, np.int32), draft], axis=1)
+    parent = synth.chain_parents(B, K)
+    for flags in (0, orc.STOCH_PLAIN, orc.STOCH_RELAX_ONLY):
+        a = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, flags)
+        t = orc.verify_tree_stochastic(logits, tok, parent, u, 0.9, 1.0, flags)
+        for k in ("accept_len", "out_tokens", "out_len", "node_how"):
+            assert np.array_equal(a[k], t[k]), (flags, k)
+        assert np.allclose(a["node_prob"], t["node_prob"], rtol=1e-12)
+    assert a["accept_len"].min() == 0 and a["accept_len"].max() >= 2
+
+
+def test_a_perfect_drafter_is_always_accepted():
+    logits, qlogits, draft, qx, u = _sampled_case(13, 400, 4, 30, 1.5, 0.0, same_rows=False)
+    out = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, orc.STOCH_PLAIN)
+    assert (out["accept_len"] == 3).all() and (out["node_how"][:, 1:] == 3).all()
+
+
+def test_residual_draw_of_the_general_form_against_numpy():
+    V, K, B = 19, 2, 600
+    logits, qlogits, draft, qx, u = _sampled_case(14, B, K, V, 1.2, 1.0, 1.1, 0.8, same_rows=False)
+    u[:, 1] = np.float32(0.999999)          # reject (almost) every draft
+    out = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.1, 0.8, orc.STOCH_PLAIN)
+    P = softmax(logits.astype(np.float64) / 1.1, axis=1)
+    Q = softmax(qlogits.astype(np.float64) / 0.8, axis=1)
+    n = 0
+    for b in range(B):
+        if out["accept_len"][b] != 0:
+            continue
+        w = np.maximum(P[b * K] - Q[b], 0.0)
+        c = np.cumsum(w)
+        want = int(np.searchsorted(c, float(u[b, 0]) * c[-1], side="right"))
+        assert out["out_tokens"][b, 0] == want
+        n += 1
+    assert n > B // 2
+
+
+def test_sampled_modes_are_nested():
+    logits, qlogits, draft, qx, u = _sampled_case(15, 500, 6, 50, 2.0, 1.0, same_rows=False)
+    a = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, orc.STOCH_PLAIN)["accept_len"]
+    r = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, orc.STOCH_RELAX_ONLY)["accept_len"]
+    d = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, 0)["accept_len"]
+    assert (a <= r).all() and (r <= d).all() and a.sum() < d.sum()
