@@ -350,6 +350,35 @@ mars_status_t mars_verify_chain_stochastic(const void *logits, int64_t ld, mars_
                                            void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Stochastic verification of chains whose drafts were SAMPLED from a drafter's distribution: the
+ * acceptance test of Eq. 1 (Sec. 2.2) in its general form.  Draft i was drawn from
+ * Q_i = softmax(draft_logits_i / draft_temperature) with probability draft_prob[b, i] = Q_i(draft_i).
+ * It is accepted iff the composition mode accepts it outright (as in mars_verify_tree_stochastic)
+ * or uniform[b, i+1] * Q_i(x) < P_i(x), which is acceptance with probability min(1, P/Q).  The
+ * first rejected position emits a token drawn from the residual distribution
+ * norm(max(0, P_i - Q_i)) by CDF inversion in token-id order with uniform[b, 0]; if every draft
+ * is accepted, or a negative draft id ends the chain, the token is drawn from P of that row.
+ * With MARS_STOCH_PLAIN this is standard speculative sampling.
+ *
+ *   draft_logits  [B*(K-1), ld_draft], same dtype as `logits`; only the row of the rejected
+ *                 position of each sequence is read (twice).
+ *   draft_prob    float [B, K-1], the probability with which the drafter drew each draft (the
+ *                 drafter knows it; it is not recomputed from draft_logits).
+ *   uniform       float [B, K]; other arguments, outputs and statuses as
+ *                 mars_verify_chain_stochastic (MARS_SEQ_BAD_DISTRIBUTION also covers a drafter
+ *                 row without a softmax and a residual without mass).
+ *   workspace     mars_stochastic_workspace_bytes(B, K, V, dt).
+ */
+mars_status_t mars_verify_chain_sampled(const void *logits, int64_t ld, mars_dtype_t dt,
+                                        const void *draft_logits, int64_t ld_draft, const int32_t *draft,
+                                        const float *draft_prob, const float *uniform, int B, int K,
+                                        int V, float theta, float temperature, float draft_temperature,
+                                        uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
+                                        int32_t *out_len, int32_t *seq_status, float *node_prob,
+                                        uint8_t *node_how, void *workspace, size_t workspace_bytes,
+                                        void *cuda_stream);
+
+/*
  * mars_verify_tree for callers that must not allocate device memory.  (The paper has no
  * counterpart; this is a deployment convenience of the library.)
  *

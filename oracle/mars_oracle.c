@@ -637,7 +637,8 @@ void mars_oracle_verify_tree_stochastic(const void *logits, int dtype, int64_t l
  * repository; PARITY UNPINNED by the paper).  With STOCH_PLAIN this is standard speculative
  * sampling, which leaves the target distribution unchanged -- the pin for this function.
  *   logits  [B*K, ld]   target rows;  qlogits [B*(K-1), ldq] drafter rows (dtype_q);
- *   draft   [B, K-1];   qx [B, K-1] float: probability with which the drafter drew the token;
+ *   draft   [B, K-1] (a negative id ends the chain: no draft there, the token is drawn from P);
+ *   qx      [B, K-1] float: probability with which the drafter drew the token;
  *   uniform [B, K]:     [b, i+1] judges draft i, [b, 0] draws the emitted token;
  *   node_how [B, K] as in the tree form (index i+1 for draft i); margin [B, 2] as there, with the
  *   draw margin in units of total probability (not of the residual's mass).
@@ -681,7 +682,8 @@ void mars_oracle_verify_chain_sampled(const void *logits, int dtype, int64_t ld,
             if (!isfinite(m) || !(S > 0.0)) { st = 4; break; }
             if (i == K - 1) break;
             int32_t x = draft[(size_t)b * (K - 1) + i];
-            double px = (x >= 0 && x < V) ? exp((row_get(row, dtype, x) - m) / T) / S : 0.0;
+            if (x < 0) break;                /* no draft here (padding): the chain ends, draw from P_i */
+            double px = (x < V) ? exp((row_get(row, dtype, x) - m) / T) / S : 0.0;
             int relax = mars_oracle_relax_f32(v2[0], v2[1], (float)theta, flags);
             int how = (flags & MARS_ORACLE_STOCH_PLAIN) ? 0 : rule(x, id2, relax);
             if ((flags & MARS_ORACLE_STOCH_RELAX_ONLY) && how == 1) how = 0;
@@ -689,7 +691,7 @@ void mars_oracle_verify_chain_sampled(const void *logits, int dtype, int64_t ld,
                 double lhs = (double)u[i + 1] * (double)qx[(size_t)b * (K - 1) + i];   /* Eq. 1 */
                 double d = fabs(px - lhs);
                 if (d < mg_test) mg_test = d;
-                how = (x >= 0 && lhs < px) ? 3 : 4;
+                how = (lhs < px) ? 3 : 4;
             }
             if (nhow) nhow[i + 1] = (uint8_t)how;
             if (how == 4) { rejected_at = i; break; }

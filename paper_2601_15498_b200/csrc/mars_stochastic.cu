@@ -183,6 +183,10 @@ struct StochTailParams {
     const int32_t *tok;      // tree [B,N]; chain: draft [B,N-1]
     const int32_t *parent;   // tree [B,N] or [N]
     const float *uniform;    // [B,N]
+    const float *qx;         // sampled chains: [B,N-1] probability with which each draft was drawn
+    const void *qlogits;     // sampled chains: drafter rows [B*(N-1), ldq], same dtype as logits
+    long long ldq;
+    float cq;                // log2(e) / T_draft
     int32_t *accept_len, *out_tokens, *path_nodes, *out_len, *seq_status;
     float *node_prob;        // [B,N] or null
     uint8_t *node_how;       // [B,N] or null
@@ -274,23 +278,82 @@ struct TailShared {
     double part[kTailWarps];
     double wtot[kTailWarps];
     int whit[kTailWarps];
+    float2 qwarp[kTailWarps];
+    float2 qstat;
     double target;
     long long range[2];
-    int ctl[8];       // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token, 6 last tile with mass
+    int ctl[8];       // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token, 6 last tile with mass,
+                      // 7 node of the rejected draft (sampled chains) or -1
     int pick_tile;
 };
+
+// ---- what a lane's elements of a tile weigh in the draw ----
+// One row: 2^(z*c - ref), removed tokens at zero (the residual of point-mass drafts).
+template <int DT>
+struct ResidualOfRow {
+    const char *rowp; bool aligned; int V; float c, nref; const int32_t *removed; int nrem;
+    struct Raw { uint4 a; };
+    __device__ __forceinline__ Raw load(long long tile, int lane) const
+    {
+        Raw r;
+        r.a = tile_load<DT>(rowp, aligned, V, tile, lane);
+        return r;
+    }
+    __device__ __forceinline__ void weights(const Raw &r, long long tile, int lane, float (&w)[Elem<DT>::kVec]) const
+    {
+        tile_weights<DT>(r.a, tile, lane, c, nref, removed, nrem, w);
+    }
+};
+
+// A target row and the drafter's row: max(0, P - Q) on normalised probabilities (the residual of
+// Eq. 1 for sampled drafts).
+template <int DT>
+struct ResidualOfPair {
+    const char *rowp, *rowq; bool aligned_p, aligned_q; int V;
+    float c, nref, inv_s, cq, nrefq, inv_sq;
+    struct Raw { uint4 a, b; };
+    __device__ __forceinline__ Raw load(long long tile, int lane) const
+    {
+        Raw r;
+        r.a = tile_load<DT>(rowp, aligned_p, V, tile, lane);
+        r.b = tile_load<DT>(rowq, aligned_q, V, tile, lane);
+        return r;
+    }
+    __device__ __forceinline__ void weights(const Raw &r, long long, int, float (&w)[Elem<DT>::kVec]) const
+    {
+        typedef Elem<DT> E;
+#pragma unroll
+        for (int k = 0; k < E::kVec; ++k) {
+            const float x = E::elem(r.a, k), y = E::elem(r.b, k);
+            const float tp = fmaf(x, c, nref), tq = fmaf(y, cq, nrefq);
+            const float pp = (x == x && tp == tp) ? ex2f(tp) * inv_s : 0.0f;
+            const float qq = (y == y && tq == tq) ? ex2f(tq) * inv_sq : 0.0f;
+            w[k] = fmaxf(pp - qq, 0.0f);
+        }
+    }
+};
+
+template <int DT, class WF>
+__device__ __forceinline__ float lane_sum(const WF &wf, const typename WF::Raw &raw, long long tile, int lane)
+{
+    float w[Elem<DT>::kVec];
+    wf.weights(raw, tile, lane, w);
+    float ls = 0.0f;
+#pragma unroll
+    for (int k = 0; k < Elem<DT>::kVec; ++k) ls += w[k];
+    return ls;
+}
 
 // Element inside one tile (warp-wide): lane prefix, then the element inside the lane.  `target` is
 // the mass that lies before the wanted element within the tile, or, with whole_row, the tile is the
 // whole row and the target is u * (its total).  Returns false if the tile holds no mass.
-template <int DT>
-__device__ __forceinline__ bool draw_in_tile(const char *rowp, bool aligned, int V, long long t0, int lane,
-                                             float c, float nref, const int32_t *removed, int nrem,
-                                             double target, bool whole_row, float u, int *picked)
+template <int DT, class WF>
+__device__ __forceinline__ bool draw_in_tile(const WF &wf, long long t0, int lane, double target, bool whole_row,
+                                             float u, int *picked)
 {
     typedef Elem<DT> E;
     float w[E::kVec];
-    tile_weights<DT>(tile_load<DT>(rowp, aligned, V, t0, lane), t0, lane, c, nref, removed, nrem, w);
+    wf.weights(wf.load(t0, lane), t0, lane, w);
     double ls = 0.0;
 #pragma unroll
     for (int k = 0; k < E::kVec; ++k) ls += (double)w[k];
@@ -328,8 +391,221 @@ __device__ __forceinline__ bool draw_in_tile(const char *rowp, bool aligned, int
     return true;
 }
 
+// CDF inversion over the weights `wf` of one row of V elements with the uniform u0, by every thread
+// of every block of the cluster (the condition to call it is the same in all of them).  On return
+// the leader's sh.ctl[5] holds the drawn token, or sh.ctl[2] == 4 if the weights have no mass.
+template <int DT, class WF>
+__device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShared &sh, const WF &wf, int V, float u0)
+{
+    typedef Elem<DT> E;
+    const int G = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const bool leader = rank == 0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
+    const long long tpc = (ntiles + G - 1) / G;          // tiles per block of the cluster
+    if (tpc <= kMaxTilesPerBlock) {                       // the host launches clusters only if this holds
+        // (1) every block: per-tile sums of its share of the row, eight tiles per warp at a time
+        const long long t_lo = min(ntiles, (long long)rank * tpc), t_hi = min(ntiles, t_lo + tpc);
+        for (long long t = t_lo + warp * 8; t < t_hi; t += kTailWarps * 8) {
+            typename WF::Raw raw[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (t + i < t_hi) raw[i] = wf.load(t + i, lane);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (t + i < t_hi) {
+                    float ls = lane_sum<DT>(wf, raw[i], t + i, lane);
+#pragma unroll
+                    for (int m = 16; m > 0; m >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, m);
+                    if (lane == 0) sh.tile[t + i - t_lo] = (double)ls;
+                }
+            }
+        }
+        cluster.sync();
+        // (2) the leader: prefix over all tile sums (its own and, through distributed shared
+        // memory, the other blocks'), a contiguous chunk of tiles per thread
+        if (leader) {
+            const int chunk = (int)((ntiles + kTailThreads - 1) / kTailThreads);
+            const long long c_lo = min(ntiles, (long long)tid * chunk), c_hi = min(ntiles, c_lo + chunk);
+            auto tile_sum = [&](long long t) -> double {
+                const int owner = (int)(t / tpc);
+                const double *base = (owner == 0) ? sh.tile : cluster.map_shared_rank(sh.tile, owner);
+                return base[t - owner * tpc];
+            };
+            double mine = 0.0;
+            int lastpos = -1;
+            for (long long t = c_lo; t < c_hi; ++t) {
+                const double v = tile_sum(t);
+                if (v > 0.0) lastpos = (int)t;
+                mine += v;
+            }
+            double inc = mine;
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const double o = __shfl_up_sync(0xffffffffu, inc, m);
+                if (lane >= m) inc += o;
+            }
+            if (lane == 31) sh.wtot[warp] = inc;
+            if (lastpos >= 0) atomicMax(&sh.ctl[6], lastpos);
+            __syncthreads();
+            double before = 0.0, Wt = 0.0;
+            for (int k = 0; k < kTailWarps; ++k) { if (k < warp) before += sh.wtot[k]; Wt += sh.wtot[k]; }
+            inc += before;
+            const double target = (double)u0 * Wt;
+            const bool good = (Wt > 0.0 && Wt < (double)INFINITY);
+            // the first thread WITH mass whose inclusive prefix passes the target
+            const unsigned hits = __ballot_sync(0xffffffffu, good && inc > target && mine > 0.0);
+            const double prev = __shfl_up_sync(0xffffffffu, inc, 1);
+            if (lane == 0) sh.whit[warp] = hits ? (__ffs(hits) - 1) : -1;
+            if (tid == 0) { sh.pick_tile = -1; sh.target = 0.0; if (!good) sh.ctl[2] = 4; }
+            __syncthreads();
+            int wsel = -1;
+            for (int k = kTailWarps - 1; k >= 0; --k) if (sh.whit[k] >= 0) wsel = k;
+            if (warp == wsel && lane == sh.whit[wsel]) {
+                double cum = (lane == 0) ? before : prev;
+                int last_in_chunk = -1;
+                for (long long t = c_lo; t < c_hi; ++t) {
+                    const double v = tile_sum(t);
+                    if (v > 0.0) last_in_chunk = (int)t;
+                    if (v > 0.0 && cum + v > target) { sh.pick_tile = (int)t; sh.target = fmax(target - cum, 0.0); break; }
+                    cum += v;
+                }
+                if (sh.pick_tile < 0) { sh.pick_tile = last_in_chunk; sh.target = (double)INFINITY; }
+            }
+            __syncthreads();
+            if (good && warp == 0) {
+                long long t0 = sh.pick_tile;
+                double target_in = sh.target;
+                if (t0 < 0) { t0 = sh.ctl[6]; target_in = (double)INFINITY; }   // rounding: the last tile with mass
+                int picked = -1;
+                bool ok = t0 >= 0;
+                if (ok) ok = draw_in_tile<DT>(wf, t0, lane, target_in, false, 0.0f, &picked);
+                ok = __all_sync(0xffffffffu, ok);
+                const int all = __reduce_max_sync(0xffffffffu, picked);   // the resolving lane's element
+                if (lane == 0) { if (!ok || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
+            }
+            __syncthreads();
+        }
+        cluster.sync();     // the other blocks' tables stay alive until the leader has read them
+    } else {
+        // table-free search (one block): sum contiguous warp segments, descend into the segment that
+        // holds the target, repeat down to one tile
+        long long t0 = 0, t1 = ntiles;
+        bool first = true, ok = true;
+        while (t1 - t0 > 1) {
+            const long long len = (t1 - t0 + kTailWarps - 1) / kTailWarps;
+            const long long w0 = min(t1, t0 + warp * len), w1 = min(t1, w0 + len);
+            double acc = 0.0;
+            long long t = w0;
+            for (; t + 8 <= w1; t += 8) {   // eight independent loads in flight per lane
+                typename WF::Raw raw[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) raw[i] = wf.load(t + i, lane);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc += (double)lane_sum<DT>(wf, raw[i], t + i, lane);
+            }
+            for (; t < w1; ++t) acc += (double)lane_sum<DT>(wf, wf.load(t, lane), t, lane);
+#pragma unroll
+            for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+            if (lane == 0) sh.part[warp] = acc;
+            __syncthreads();
+            if (tid == 0) {
+                double target;
+                bool good = true;
+                if (first) {
+                    double Wt = 0.0;
+                    for (int k = 0; k < kTailWarps; ++k) Wt += sh.part[k];
+                    good = (Wt > 0.0 && Wt < (double)INFINITY);
+                    target = (double)u0 * Wt;
+                } else target = sh.target;
+                int pick = -1, lastpos = -1;
+                double cum = 0.0, before = 0.0;
+                for (int k = 0; k < kTailWarps && pick < 0; ++k) {
+                    if (sh.part[k] > 0.0) lastpos = k;
+                    before = cum;
+                    cum += sh.part[k];
+                    if (cum > target) pick = k;
+                }
+                if (pick < 0) {   // rounding pushed the target past the total: the last part with mass
+                    pick = lastpos;
+                    before = 0.0;
+                    for (int k = 0; k < pick; ++k) before += sh.part[k];
+                }
+                if (!good || pick < 0) { sh.ctl[2] = 4; sh.range[0] = 0; sh.range[1] = 0; }
+                else {
+                    sh.target = fmax(target - before, 0.0);
+                    sh.range[0] = min(t1, t0 + pick * len);
+                    sh.range[1] = min(t1, sh.range[0] + len);
+                }
+            }
+            __syncthreads();
+            t0 = sh.range[0]; t1 = sh.range[1];
+            first = false;
+            if (t1 <= t0) { ok = false; break; }
+        }
+        if (ok && warp == 0) {
+            int picked = -1;
+            bool fine = draw_in_tile<DT>(wf, t0, lane, first ? 0.0 : sh.target, first, u0, &picked);
+            fine = __all_sync(0xffffffffu, fine);
+            const int all = __reduce_max_sync(0xffffffffu, picked);
+            if (lane == 0) { if (!fine || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
+        }
+        __syncthreads();
+    }
+}
+
+// (ref, sum) of 2^(z*c - ref) over one row, by the whole cluster: every block covers its share of
+// the tiles, the per-block results meet through distributed shared memory and every block ends up
+// with the row's total (merged in rank order, so all blocks hold the same bits).
 template <int DT>
-__global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const StochTailParams p)
+__device__ void row_softmax_cluster(cooperative_groups::cluster_group &cluster, TailShared &sh, const char *rowp,
+                                    bool aligned, int V, float c, float *ref_out, float *sum_out)
+{
+    typedef Elem<DT> E;
+    const int G = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
+    const long long tpc = (ntiles + G - 1) / G;
+    const long long t_lo = min(ntiles, (long long)rank * tpc), t_hi = min(ntiles, t_lo + tpc);
+    float ref = -INFINITY, sum = 0.0f;
+    for (long long t = t_lo + warp * 4; t < t_hi; t += kTailWarps * 4) {
+        uint4 raw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (t + i < t_hi) raw[i] = tile_load<DT>(rowp, aligned, V, t + i, lane);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (t + i < t_hi) {
+#pragma unroll
+                for (int k = 0; k < E::kVec; ++k) soft_add_scalar(ref, sum, E::elem(raw[i], k), c);
+            }
+    }
+#pragma unroll
+    for (int m = 16; m > 0; m >>= 1) {
+        const float rb = __shfl_xor_sync(0xffffffffu, ref, m), sb = __shfl_xor_sync(0xffffffffu, sum, m);
+        soft_merge(ref, sum, rb, sb);
+    }
+    if (lane == 0) sh.qwarp[warp] = make_float2(ref, sum);
+    __syncthreads();
+    if (tid == 0) {
+        float r = sh.qwarp[0].x, q = sh.qwarp[0].y;
+        for (int k = 1; k < kTailWarps; ++k) soft_merge(r, q, sh.qwarp[k].x, sh.qwarp[k].y);
+        sh.qstat = make_float2(r, q);
+    }
+    cluster.sync();
+    float r = -INFINITY, q = 0.0f;
+    for (int g = 0; g < G; ++g) {
+        const float2 v = (g == rank) ? sh.qstat : *cluster.map_shared_rank(&sh.qstat, g);
+        soft_merge(r, q, v.x, v.y);
+    }
+    *ref_out = r;
+    *sum_out = q;
+}
+
+// SAMPLED: chains whose drafts were sampled from a drafter's distribution (general Eq. 1): the
+// acceptance test carries the draft's own probability and the residual is max(0, P - Q).
+template <int DT, bool SAMPLED>
+__global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kernel(const StochTailParams p)
 {
     typedef Elem<DT> E;
     namespace cg = cooperative_groups;
@@ -339,6 +615,7 @@ __global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const Stoch
     const int G = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
     const bool leader = rank == 0;
+    (void)rank;
     const int b = (int)(blockIdx.x / G);
     const int N = p.N, V = p.V, S = p.S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -423,7 +700,7 @@ __global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const Stoch
     int32_t *o_tok = p.out_tokens + (size_t)b * Wd;
     int32_t *o_path = p.path_nodes ? p.path_nodes + (size_t)b * Wd : nullptr;
     if (warp == 0) {
-        int cur = 0, a = 0, status = bad ? 1 : 0, nrem = 0, draw = 0;
+        int cur = 0, a = 0, status = bad ? 1 : 0, nrem = 0, draw = 0, rejected = -1;
         if (leader) {
             for (int k = lane; k < Wd; k += 32) { o_tok[k] = -1; if (o_path) o_path[k] = (k == 0) ? 0 : -1; }
         }
@@ -449,10 +726,15 @@ __global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const Stoch
                         if (x == id1) how = (p.flags & MARS_STOCH_RELAX_ONLY) ? 0 : 1;
                         else if (x == id2 && rlx) how = 2;
                     }
-                    if (how == 0) how = (__fmul_rn(s_u[j], rem) < ex) ? 3 : 4;   // Eq. 1 on the running residual
+                    if (how == 0) {
+                        float lhs = s_u[j];
+                        if (SAMPLED) lhs = __fmul_rn(lhs, p.qx[(size_t)b * (N - 1) + (j - 1)]);   // u * Q(x) < P(x)
+                        how = (__fmul_rn(lhs, rem) < ex) ? 3 : 4;    // Eq. 1 on the running residual
+                    }
                     if (lane == 0) s_how[j] = (unsigned char)how;
                     if (how == 4) {
-                        if (ex > 0.0f) {
+                        if (SAMPLED) rejected = j;     // the residual needs the drafter's row, not a removal
+                        else if (ex > 0.0f) {
                             rem = fmaxf(__fsub_rn(rem, ex), 0.0f);
                             if (lane == 0) s_removed[nrem] = x;
                             ++nrem;
@@ -471,177 +753,41 @@ __global__ void __launch_bounds__(kTailThreads, 2) stoch_tail_kernel(const Stoch
             if (leader)
                 for (int k = lane; k < Wd; k += 32) { o_tok[k] = -1; if (o_path) o_path[k] = (k == 0) ? 0 : -1; }
             for (int i = lane; i < N; i += 32) s_how[i] = 0;
-            cur = 0; a = 0; draw = 0; nrem = 0;
+            cur = 0; a = 0; draw = 0; nrem = 0; rejected = -1;
         }
         if (lane == 0) {
             sh.ctl[0] = cur; sh.ctl[1] = a; sh.ctl[2] = status; sh.ctl[3] = nrem; sh.ctl[4] = draw;
-            sh.ctl[5] = s_id1[cur]; sh.ctl[6] = -1;
+            sh.ctl[5] = s_id1[cur]; sh.ctl[6] = -1; sh.ctl[7] = rejected;
         }
     }
     __syncthreads();
 
     // ---- the next token: CDF inversion over the residual of row `cur` ----
     const int cur = sh.ctl[0];
-    const int nrem = sh.ctl[3];
-    const char *rowp = (const char *)p.logits + ((size_t)b * N + cur) * (size_t)p.ld * E::kBytes;
-    const bool aligned = (((uintptr_t)rowp) & 15) == 0;
-    const float nref = -s_ref[cur];
-    const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
-    const long long tpc = (ntiles + G - 1) / G;          // tiles per block of the cluster
-    const bool table = tpc <= kMaxTilesPerBlock;          // the host launches clusters only if this holds
-
-    if (sh.ctl[4] && table) {
-        // (1) every block: per-tile sums of its share of the row, eight tiles per warp at a time
-        const long long t_lo = min(ntiles, (long long)rank * tpc), t_hi = min(ntiles, t_lo + tpc);
-        for (long long t = t_lo + warp * 8; t < t_hi; t += kTailWarps * 8) {
-            uint4 raw[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (t + i < t_hi) raw[i] = tile_load<DT>(rowp, aligned, V, t + i, lane);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (t + i < t_hi) {
-                    float ls = tile_lane_sum<DT>(raw[i], t + i, lane, p.c, nref, s_removed, nrem);
-#pragma unroll
-                    for (int m = 16; m > 0; m >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, m);
-                    if (lane == 0) sh.tile[t + i - t_lo] = (double)ls;
-                }
+    if (sh.ctl[4]) {
+        const char *rowp = (const char *)p.logits + ((size_t)b * N + cur) * (size_t)p.ld * E::kBytes;
+        const bool aligned = (((uintptr_t)rowp) & 15) == 0;
+        const int rejected = sh.ctl[7];
+        if (SAMPLED && rejected >= 0) {
+            // draft `rejected - 1` failed Eq. 1: draw from max(0, P - Q) with Q the drafter's row
+            const char *rowq = (const char *)p.qlogits + ((size_t)b * (N - 1) + (rejected - 1)) * (size_t)p.ldq * E::kBytes;
+            const bool aligned_q = (((uintptr_t)rowq) & 15) == 0;
+            float refq, sumq;
+            row_softmax_cluster<DT>(cluster, sh, rowq, aligned_q, V, p.cq, &refq, &sumq);
+            if (!(refq > -INFINITY && refq < INFINITY && sumq > 0.0f && sumq < INFINITY)) {
+                if (tid == 0) sh.ctl[2] = 4;      // the drafter's row has no softmax (same in every block)
+            } else {
+                ResidualOfPair<DT> wf;
+                wf.rowp = rowp; wf.rowq = rowq; wf.aligned_p = aligned; wf.aligned_q = aligned_q; wf.V = V;
+                wf.c = p.c; wf.nref = -s_ref[cur]; wf.inv_s = __fdiv_rn(1.0f, s_sum[cur]);
+                wf.cq = p.cq; wf.nrefq = -refq; wf.inv_sq = __fdiv_rn(1.0f, sumq);
+                draw_token<DT>(cluster, sh, wf, V, s_u[0]);
             }
-        }
-        cluster.sync();
-        // (2) the leader: prefix over all tile sums (its own and, through distributed shared
-        // memory, the other blocks'), a contiguous chunk of tiles per thread
-        if (leader) {
-            const int chunk = (int)((ntiles + kTailThreads - 1) / kTailThreads);
-            const long long c_lo = min(ntiles, (long long)tid * chunk), c_hi = min(ntiles, c_lo + chunk);
-            auto tile_sum = [&](long long t) -> double {
-                const int owner = (int)(t / tpc);
-                const double *base = (owner == 0) ? sh.tile : cluster.map_shared_rank(sh.tile, owner);
-                return base[t - owner * tpc];
-            };
-            double mine = 0.0;
-            int lastpos = -1;
-            for (long long t = c_lo; t < c_hi; ++t) {
-                const double v = tile_sum(t);
-                if (v > 0.0) lastpos = (int)t;
-                mine += v;
-            }
-            double inc = mine;
-#pragma unroll
-            for (int m = 1; m < 32; m <<= 1) {
-                const double o = __shfl_up_sync(0xffffffffu, inc, m);
-                if (lane >= m) inc += o;
-            }
-            if (lane == 31) sh.wtot[warp] = inc;
-            if (lastpos >= 0) atomicMax(&sh.ctl[6], lastpos);
-            __syncthreads();
-            double before = 0.0, Wt = 0.0;
-            for (int k = 0; k < kTailWarps; ++k) { if (k < warp) before += sh.wtot[k]; Wt += sh.wtot[k]; }
-            inc += before;
-            const double target = (double)s_u[0] * Wt;
-            const bool good = (Wt > 0.0 && Wt < (double)INFINITY);
-            // the first thread WITH mass whose inclusive prefix passes the target
-            const unsigned hits = __ballot_sync(0xffffffffu, good && inc > target && mine > 0.0);
-            const double prev = __shfl_up_sync(0xffffffffu, inc, 1);
-            if (lane == 0) sh.whit[warp] = hits ? (__ffs(hits) - 1) : -1;
-            if (tid == 0) { sh.pick_tile = -1; sh.target = 0.0; if (!good) sh.ctl[2] = 4; }
-            __syncthreads();
-            int wsel = -1;
-            for (int k = kTailWarps - 1; k >= 0; --k) if (sh.whit[k] >= 0) wsel = k;
-            if (warp == wsel && lane == sh.whit[wsel]) {
-                double cum = (lane == 0) ? before : prev;
-                int last_in_chunk = -1;
-                for (long long t = c_lo; t < c_hi; ++t) {
-                    const double v = tile_sum(t);
-                    if (v > 0.0) last_in_chunk = (int)t;
-                    if (v > 0.0 && cum + v > target) { sh.pick_tile = (int)t; sh.target = fmax(target - cum, 0.0); break; }
-                    cum += v;
-                }
-                if (sh.pick_tile < 0) { sh.pick_tile = last_in_chunk; sh.target = (double)INFINITY; }
-            }
-            __syncthreads();
-            if (good && warp == 0) {
-                long long t0 = sh.pick_tile;
-                double target_in = sh.target;
-                if (t0 < 0) { t0 = sh.ctl[6]; target_in = (double)INFINITY; }   // rounding: the last tile with mass
-                int picked = -1;
-                bool ok = t0 >= 0;
-                if (ok) ok = draw_in_tile<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem, target_in,
-                                              false, 0.0f, &picked);
-                ok = __all_sync(0xffffffffu, ok);
-                const int all = __reduce_max_sync(0xffffffffu, picked);   // the resolving lane's element
-                if (lane == 0) { if (!ok || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
-            }
-            __syncthreads();
-        }
-        cluster.sync();     // the other blocks' tables stay alive until the leader has read them
-    } else if (sh.ctl[4]) {
-        // table-free search (one block): sum contiguous warp segments, descend into the segment that
-        // holds the target, repeat down to one tile
-        long long t0 = 0, t1 = ntiles;
-        bool first = true, ok = true;
-        while (t1 - t0 > 1) {
-            const long long len = (t1 - t0 + kTailWarps - 1) / kTailWarps;
-            const long long w0 = min(t1, t0 + warp * len), w1 = min(t1, w0 + len);
-            double acc = 0.0;
-            long long t = w0;
-            for (; t + 8 <= w1; t += 8) {   // eight independent 16-byte loads in flight per lane
-                uint4 raw[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) raw[i] = tile_load<DT>(rowp, aligned, V, t + i, lane);
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    acc += (double)tile_lane_sum<DT>(raw[i], t + i, lane, p.c, nref, s_removed, nrem);
-            }
-            for (; t < w1; ++t) {
-                const uint4 raw = tile_load<DT>(rowp, aligned, V, t, lane);
-                acc += (double)tile_lane_sum<DT>(raw, t, lane, p.c, nref, s_removed, nrem);
-            }
-#pragma unroll
-            for (int m = 16; m > 0; m >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
-            if (lane == 0) sh.part[warp] = acc;
-            __syncthreads();
-            if (tid == 0) {
-                double target;
-                bool good = true;
-                if (first) {
-                    double Wt = 0.0;
-                    for (int k = 0; k < kTailWarps; ++k) Wt += sh.part[k];
-                    good = (Wt > 0.0 && Wt < (double)INFINITY);
-                    target = (double)s_u[0] * Wt;
-                } else target = sh.target;
-                int pick = -1, lastpos = -1;
-                double cum = 0.0, before = 0.0;
-                for (int k = 0; k < kTailWarps && pick < 0; ++k) {
-                    if (sh.part[k] > 0.0) lastpos = k;
-                    before = cum;
-                    cum += sh.part[k];
-                    if (cum > target) pick = k;
-                }
-                if (pick < 0) {   // rounding pushed the target past the total: the last part with mass
-                    pick = lastpos;
-                    before = 0.0;
-                    for (int k = 0; k < pick; ++k) before += sh.part[k];
-                }
-                if (!good || pick < 0) { sh.ctl[2] = 4; sh.range[0] = 0; sh.range[1] = 0; }
-                else {
-                    sh.target = fmax(target - before, 0.0);
-                    sh.range[0] = min(t1, t0 + pick * len);
-                    sh.range[1] = min(t1, sh.range[0] + len);
-                }
-            }
-            __syncthreads();
-            t0 = sh.range[0]; t1 = sh.range[1];
-            first = false;
-            if (t1 <= t0) { ok = false; break; }
-        }
-        if (ok && warp == 0) {
-            int picked = -1;
-            bool fine = draw_in_tile<DT>(rowp, aligned, V, t0, lane, p.c, nref, s_removed, nrem,
-                                         first ? 0.0 : sh.target, first, s_u[0], &picked);
-            fine = __all_sync(0xffffffffu, fine);
-            const int all = __reduce_max_sync(0xffffffffu, picked);
-            if (lane == 0) { if (!fine || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
+        } else {
+            ResidualOfRow<DT> wf;
+            wf.rowp = rowp; wf.aligned = aligned; wf.V = V; wf.c = p.c; wf.nref = -s_ref[cur];
+            wf.removed = s_removed; wf.nrem = sh.ctl[3];
+            draw_token<DT>(cluster, sh, wf, V, s_u[0]);
         }
         __syncthreads();
     }
@@ -803,8 +949,16 @@ static bool stoch_sizes_supported(int B, int N, int V, int dt)
     return true;
 }
 
+struct SampledDrafts {        // chains whose drafts were sampled from a drafter (general Eq. 1)
+    const void *qlogits;
+    int64_t ldq;
+    const float *qx;
+    float draft_temperature;
+};
+
 static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t dt, const int32_t *tok,
-                                    const int32_t *parent, const float *uniform, int chain, int B, int N,
+                                    const int32_t *parent, const float *uniform, const SampledDrafts *sd,
+                                    int chain, int B, int N,
                                     int V, float theta, float temperature, uint32_t flags,
                                     int32_t *accept_len, int32_t *out_tokens, int32_t *path_nodes,
                                     int32_t *out_len, int Dcap, int32_t *seq_status, float *node_prob,
@@ -814,6 +968,15 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     if (B < 1 || N < 1 || V < 2 || !logits || !uniform) return MARS_ERR_INVALID_ARG;
     if (ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || !(temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
+    double cqd = 0.0;
+    if (sd) {
+        if (!chain) return MARS_ERR_INVALID_ARG;
+        if (N > 1 && (!sd->qlogits || !sd->qx || sd->ldq < V)) return MARS_ERR_INVALID_ARG;
+        if (!(sd->draft_temperature > 0.0f) || !(sd->draft_temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
+        if ((uintptr_t)sd->qlogits % (dt == MARS_BF16 ? 2 : 4)) return MARS_ERR_INVALID_ARG;
+        cqd = 1.4426950408889634074 / (double)sd->draft_temperature;
+        if (!(cqd < 3.0e38)) return MARS_ERR_INVALID_ARG;
+    }
     if (!accept_len || !out_tokens || !out_len) return MARS_ERR_INVALID_ARG;
     if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
     if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
@@ -849,17 +1012,19 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     tp.logits = logits; tp.ld = ld; tp.V = V; tp.N = N; tp.S = sp.S; tp.c = (float)cd; tp.theta = theta;
     tp.flags = flags; tp.chain = chain; tp.Dcap = Dcap; tp.partial = sp1.partial;
     tp.tok = tok; tp.parent = parent; tp.uniform = uniform;
+    tp.qx = sd ? sd->qx : nullptr; tp.qlogits = sd ? sd->qlogits : nullptr; tp.ldq = sd ? sd->ldq : 0;
+    tp.cq = (float)cqd;
     tp.accept_len = accept_len; tp.out_tokens = out_tokens; tp.path_nodes = path_nodes;
     tp.out_len = out_len; tp.seq_status = seq_status; tp.node_prob = node_prob; tp.node_how = node_how;
     const size_t smem = stoch_tail_smem_bytes(N);
     // The largest cluster (8, 4, 2 blocks per sequence) that still fits the GPU in one wave (two
-    // blocks of 512 threads per SM) and leaves each block a share of the row that fits its tile
+    // blocks of 512 threads per SM; one for sampled chains, whose draw holds two rows in registers) and leaves each block a share of the row that fits its tile
     // table; rows too long for the table of a single block take the table-free search (G = 1).
     const int kv = dt == MARS_BF16 ? 8 : 4;
     const long long ntiles = ((long long)V + 32 * kv - 1) / (32 * kv);
     int G = 1;
     for (int g = kTailCluster; g > 1; g >>= 1)
-        if ((long long)B * g <= 2 * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
+        if ((long long)B * g <= (sd ? 1 : 2) * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
     const char *force = getenv("MARS_STOCH_TAIL_CLUSTER");   // test hook: 1, 2, 4 or 8
     if (force) {
         const int g = atoi(force);
@@ -877,8 +1042,13 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16>, tp)
-                                              : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32>, tp);
+    cudaError_t err;
+    if (sd)
+        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, true>, tp)
+                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, true>, tp);
+    else
+        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, false>, tp)
+                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, false>, tp);
     if (err != cudaSuccess) { cudaGetLastError(); return MARS_ERR_CUDA; }
     return MARS_OK;
 }
@@ -902,7 +1072,7 @@ mars_status_t mars_verify_tree_stochastic(const void *logits, int64_t ld, mars_d
                                           uint8_t *node_how, void *workspace, size_t workspace_bytes,
                                           void *cuda_stream)
 {
-    return mars::run_stochastic(logits, ld, dt, tok, parent, uniform, 0, B, N, V, theta, temperature, flags,
+    return mars::run_stochastic(logits, ld, dt, tok, parent, uniform, nullptr, 0, B, N, V, theta, temperature, flags,
                                 accept_len, out_tokens, path_nodes, out_len, Dcap, seq_status, node_prob,
                                 node_how, workspace, workspace_bytes, cuda_stream);
 }
@@ -915,9 +1085,25 @@ mars_status_t mars_verify_chain_stochastic(const void *logits, int64_t ld, mars_
                                            size_t workspace_bytes, void *cuda_stream)
 {
     if (flags & MARS_SHARED_PARENT) return MARS_ERR_INVALID_ARG;
-    return mars::run_stochastic(logits, ld, dt, draft, nullptr, uniform, 1, B, K, V, theta, temperature, flags,
-                                accept_len, out_tokens, nullptr, out_len, K - 1, seq_status, node_prob,
+    return mars::run_stochastic(logits, ld, dt, draft, nullptr, uniform, nullptr, 1, B, K, V, theta, temperature,
+                                flags, accept_len, out_tokens, nullptr, out_len, K - 1, seq_status, node_prob,
                                 node_how, workspace, workspace_bytes, cuda_stream);
+}
+
+mars_status_t mars_verify_chain_sampled(const void *logits, int64_t ld, mars_dtype_t dt, const void *draft_logits,
+                                        int64_t ld_draft, const int32_t *draft, const float *draft_prob,
+                                        const float *uniform, int B, int K, int V, float theta, float temperature,
+                                        float draft_temperature, uint32_t flags, int32_t *accept_len,
+                                        int32_t *out_tokens, int32_t *out_len, int32_t *seq_status,
+                                        float *node_prob, uint8_t *node_how, void *workspace,
+                                        size_t workspace_bytes, void *cuda_stream)
+{
+    if (flags & MARS_SHARED_PARENT) return MARS_ERR_INVALID_ARG;
+    mars::SampledDrafts sd;
+    sd.qlogits = draft_logits; sd.ldq = ld_draft; sd.qx = draft_prob; sd.draft_temperature = draft_temperature;
+    return mars::run_stochastic(logits, ld, dt, draft, nullptr, uniform, &sd, 1, B, K, V, theta, temperature, flags,
+                                accept_len, out_tokens, nullptr, out_len, K - 1, seq_status, node_prob, node_how,
+                                workspace, workspace_bytes, cuda_stream);
 }
 
 }  // extern "C"

@@ -85,6 +85,9 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_chain_stochastic.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, f32, u32,
                                                        vp, vp, vp, vp, vp, vp, vp, sz, vp]
             L.mars_verify_chain_stochastic.restype = i32
+            L.mars_verify_chain_sampled.argtypes = [vp, i64, i32, vp, i64, vp, vp, vp, i32, i32, i32, f32, f32, f32,
+                                                    u32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+            L.mars_verify_chain_sampled.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -354,6 +357,45 @@ def verify_chain_stochastic(logits: torch.Tensor, draft, uniform, theta: float, 
             workspace.data_ptr(), wbytes, _stream())
     _check(code, "mars_verify_chain_stochastic")
     out["_keepalive"] = (draft, uniform, workspace)
+    return out
+
+
+def verify_chain_sampled(logits: torch.Tensor, draft_logits: torch.Tensor, draft, draft_prob, uniform,
+                         theta: float, temperature: float, draft_temperature: float, flags: int = 0,
+                         V: int | None = None, debug: bool = False, workspace: torch.Tensor | None = None,
+                         out: dict | None = None) -> dict:
+    """mars_verify_chain_sampled on the current stream: K target rows and K-1 drafter rows per
+    sequence, drafts [B, K-1] with their drafter probabilities, uniform [B, K]."""
+    dev = logits.device
+    draft = _dev_i32(draft, dev)
+    draft_prob = _dev_f32(draft_prob, dev)
+    uniform = _dev_f32(uniform, dev)
+    B, Km1 = draft.shape
+    K = Km1 + 1
+    if tuple(uniform.shape) != (B, K) or tuple(draft_prob.shape) != (B, Km1):
+        raise MarsError("uniform must be [B, K] and draft_prob [B, K-1]")
+    dt, ld, V = _logits_args(logits, B * K, V)
+    if Km1 > 0:
+        dtq, ldq, _ = _logits_args(draft_logits, B * Km1, V)
+        if dtq != dt or draft_logits.shape[1] < V:
+            raise MarsError("draft_logits must have the dtype of logits and at least V columns")
+    else:
+        ldq = V
+    workspace, wbytes = _stoch_workspace(B, K, V, dt, dev, workspace)
+    if out is None:
+        out = alloc_stochastic_outputs(B, K, K - 1, dev, debug)
+    with torch.cuda.device(dev):
+        code = lib().mars_verify_chain_sampled(
+            logits.data_ptr(), ld, dt, draft_logits.data_ptr() if Km1 > 0 else None, ldq,
+            draft.data_ptr() if Km1 > 0 else None, draft_prob.data_ptr() if Km1 > 0 else None,
+            uniform.data_ptr(), B, K, V, float(theta), float(temperature), float(draft_temperature), flags,
+            out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(), out["out_len"].data_ptr(),
+            out["seq_status"].data_ptr(),
+            out["node_prob"].data_ptr() if "node_prob" in out else None,
+            out["node_how"].data_ptr() if "node_how" in out else None,
+            workspace.data_ptr(), wbytes, _stream())
+    _check(code, "mars_verify_chain_sampled")
+    out["_keepalive"] = (draft, draft_prob, uniform, draft_logits, workspace)
     return out
 
 

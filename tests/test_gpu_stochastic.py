@@ -9,7 +9,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
-from stochastic_checks import DEV, STATS, check_walk_is_valid, compare, host_f64
+from stochastic_checks import (DECISION_TOL, DEV, PROB_RTOL, STATS, check_walk_is_valid, compare,
+                               host_f64)
 
 pytestmark = pytest.mark.gpu
 
@@ -271,6 +272,111 @@ def test_full_size_batch_sampled_sequences():
                 u[b:b + 1], 1.0, f"sequence {b}", max_close_frac=1.0)
     for b in range(w.B):
         check_walk_is_valid(got, w.tok, w.parent, b)
+
+
+# ---------------------------------------------------------------- sampled drafts (general Eq. 1)
+
+def sampled_case(seed, B, K, V, dtype, sigma_q=1.0, T=1.0, Tq=1.0, ld_pad=0):
+    """Target rows from the chain recipe, drafter rows = target rows + noise, drafts really drawn
+    from the drafter's softmax (torch, on the host) with their probabilities."""
+    w = synth.chain_workload("t", B, K, V, dtype, DEV, seed, 0.9, 1.5, 6.0, 10.0, 0.4)
+    g = torch.Generator().manual_seed(seed)
+    z = w.logits.float().cpu().reshape(B, K, V)[:, :K - 1].reshape(-1, V)
+    zq = (z + torch.randn(z.shape, generator=g) * sigma_q).to(dtype)
+    Q = torch.softmax(zq.double() / Tq, dim=1)
+    draft = torch.multinomial(Q, 1, generator=g).reshape(-1)
+    qx = Q[torch.arange(Q.shape[0]), draft].float()
+    qdev = torch.full((B * (K - 1), V + ld_pad), 55.0, dtype=dtype, device=DEV)
+    qdev[:, :V] = zq.to(DEV)
+    u = synth.make_uniforms(B, K, seed)
+    return w, qdev, zq, draft.reshape(B, K - 1).numpy().astype(np.int32), qx.reshape(B, K - 1).numpy(), u
+
+
+def compare_sampled(got, ref, what):
+    B = ref["accept_len"].shape[0]
+    n_close = 0
+    for b in range(B):
+        a = int(ref["accept_len"][b])
+        same_walk = all(np.array_equal(got[k][b], ref[k][b]) for k in ("accept_len", "out_len", "seq_status", "node_how")) \
+            and np.array_equal(got["out_tokens"][b, :a], ref["out_tokens"][b, :a])
+        if not same_walk:
+            assert ref["margin"][b, 0] < DECISION_TOL, (what, b, ref["margin"][b])
+            n_close += 1
+            continue
+        if got["out_tokens"][b, a] != ref["out_tokens"][b, a]:
+            # the draw margin of this oracle is in units of total probability
+            assert ref["margin"][b, 1] < 2e-6, (what, b, got["out_tokens"][b], ref["out_tokens"][b], ref["margin"][b])
+            n_close += 1
+    np.testing.assert_allclose(got["node_prob"], ref["node_prob"], rtol=PROB_RTOL, atol=1e-30, err_msg=what)
+    assert n_close <= max(2, B // 50), (what, n_close)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY])
+def test_sampled_chains(dtype, flags):
+    w, qdev, zq, draft, qx, u = sampled_case(31, 64, 6, 30011, dtype, 1.0, 0.9, 1.1, ld_pad=5)
+    got = mars.to_host(mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, 0.9, 1.1, flags, V=w.V, debug=True))
+    ref = orc.verify_chain_sampled(synth.to_numpy_bits(w.logits), synth.to_numpy_bits(zq), draft, qx, u, 0.9, 0.9, 1.1,
+                                   flags)
+    compare_sampled(got, ref, f"sampled {dtype} {flags}")
+    how = ref["node_how"]
+    assert (how == 3).any() and (how == 4).any() and ref["accept_len"].max() >= 2
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4, 8])
+def test_sampled_chains_cluster_shapes(cluster, monkeypatch):
+    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    w, qdev, zq, draft, qx, u = sampled_case(32, 40, 4, 70001, torch.bfloat16, 1.5)
+    u[:, 1] = np.float32(0.99999)          # most sequences reject their first draft: residual draws
+    got = mars.to_host(mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, 1.0, 1.0, mars.STOCH_PLAIN,
+                                                 debug=True))
+    ref = orc.verify_chain_sampled(synth.to_numpy_bits(w.logits), synth.to_numpy_bits(zq), draft, qx, u, 0.9, 1.0,
+                                   1.0, orc.STOCH_PLAIN)
+    compare_sampled(got, ref, f"sampled cluster {cluster}")
+    assert (ref["accept_len"] == 0).mean() > 0.5
+
+
+def test_sampled_chains_special_cases():
+    w, qdev, zq, draft, qx, u = sampled_case(33, 12, 5, 5003, torch.float32, 1.0)
+    draft[0, 1] = -1                         # the chain of sequence 0 ends after one draft
+    qdev[1 * 4 + 0, :] = float("-inf")       # drafter row without a softmax
+    zq[1 * 4 + 0, :] = float("-inf")
+    u[1, 1] = np.float32(0.999999)           # make sure sequence 1 rejects its first draft
+    qdev[2 * 4 + 0, 100:200] = float("nan")
+    zq[2 * 4 + 0, 100:200] = float("nan")
+    lg = w.logits.clone()
+    lg[3 * 5 + 1, :] = float("-inf")         # target row without a softmax on the way
+    got = mars.to_host(mars.verify_chain_sampled(lg, qdev, draft, qx, u, 0.9, 1.0, 1.0, debug=True))
+    ref = orc.verify_chain_sampled(synth.to_numpy_bits(lg), synth.to_numpy_bits(zq), draft, qx, u, 0.9, 1.0, 1.0)
+    compare_sampled(got, ref, "sampled special")
+    assert ref["seq_status"][1] == 4 or ref["accept_len"][1] > 0
+
+
+def test_sampled_plain_mode_preserves_the_target_distribution_on_the_gpu():
+    """Speculative sampling on the GPU with drafts really drawn from the drafter: the first emitted
+    token follows the target's first row."""
+    rng = np.random.default_rng(7)
+    V, K, B, T, Tq = 40, 3, 30000, 0.9, 1.3
+    rows = torch.tensor((rng.normal(size=(K, V)) * 1.0).astype(np.float32))
+    rows_q = rows[:K - 1] + torch.tensor((rng.normal(size=(K - 1, V)) * 0.8).astype(np.float32))
+    Q = torch.softmax(rows_q.double() / Tq, dim=1)
+    g = torch.Generator().manual_seed(7)
+    draft = torch.stack([torch.multinomial(Q[i], B, replacement=True, generator=g) for i in range(K - 1)], dim=1)
+    qx = torch.stack([Q[i][draft[:, i]] for i in range(K - 1)], dim=1).float()
+    u = synth.make_uniforms(B, K, 7)
+    got = mars.to_host(mars.verify_chain_sampled(rows.repeat(B, 1).to(DEV), rows_q.repeat(B, 1).to(DEV),
+                                                 draft.int().numpy(), qx.numpy(), u, 0.9, T, Tq, mars.STOCH_PLAIN))
+    P = torch.softmax(rows[0].double() / T, 0).numpy()
+    f = np.bincount(got["out_tokens"][:, 0], minlength=V) / B
+    assert np.all(np.abs(f - P) <= 4.5 * np.sqrt(P * (1 - P) / B) + 1e-9)
+
+
+def test_sampled_host_errors():
+    w, qdev, zq, draft, qx, u = sampled_case(34, 2, 3, 200, torch.float32)
+    with pytest.raises(mars.MarsError, match="invalid argument"):
+        mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, 1.0, 0.0)
+    with pytest.raises(mars.MarsError, match="dtype"):
+        mars.verify_chain_sampled(w.logits, qdev.to(torch.bfloat16), draft, qx, u, 0.9, 1.0, 1.0)
 
 
 def test_zz_report_tolerated_cases():
