@@ -598,6 +598,7 @@ __device__ void row_softmax_cluster(cooperative_groups::cluster_group &cluster, 
         const float2 v = (g == rank) ? sh.qstat : *cluster.map_shared_rank(&sh.qstat, g);
         soft_merge(r, q, v.x, v.y);
     }
+    cluster.sync();     // no block may move on (and possibly exit) while another still reads its result
     *ref_out = r;
     *sum_out = q;
 }
@@ -1003,7 +1004,8 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     sp1.partial = (SRec *)workspace;
     const unsigned grid = (unsigned)(R * sp.S);
     // 4 vectors per batch in two register buffers, 4 blocks per SM (64 registers): measured
-    // best for both dtypes; 5 or 6 blocks per SM spill the second buffer and run at half speed.
+    // best for both dtypes; 5 or 6 blocks per SM spill the second buffer and run at half speed,
+    // and 2 vectors per batch at 5 to 8 blocks per SM lose 10 to 50 %.
     if (dt == MARS_BF16) stoch_stream_kernel<MARS_BF16, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
     else stoch_stream_kernel<MARS_FP32, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
     if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
