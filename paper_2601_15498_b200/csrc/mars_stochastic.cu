@@ -16,13 +16,16 @@
 //       times c = log2(e)/T) and sum = SUM 2^(z*c - ref); the reference only moves when a
 //       batch maximum exceeds it, which the top-2 filter computes anyway.  One 32-byte record
 //       {z1, id1, z2, id2, ref, sum} per slice.
-//   stoch_tail_kernel     one block per sequence: merges slice records, gathers the logit of
-//       every node's token from its parent's row (one scalar load per node, all in parallel),
-//       walks the tree (Eq. 1 on the running residual, or the margin rule), then draws the next
-//       token from the residual of the row where the walk stopped by inverting its CDF in
-//       token-id order: the row is summed by contiguous warp segments, the segment holding
-//       u*W is split again, and so on down to one 32-lane tile and one element (partial sums
-//       and the running target in fp64, so that the pick depends on the weights alone).
+//   stoch_tail_kernel     one thread-block cluster (1 to 8 blocks) per sequence: merges slice
+//       records, gathers the logit of every node's token from its parent's row (one scalar load
+//       per node, all in parallel), walks the tree (Eq. 1 on the running residual, or the margin
+//       rule), then draws the next token from the residual of the row where the walk stopped by
+//       inverting its CDF in token-id order: per-tile sums spread over the cluster's shared
+//       memories, an fp64 prefix over them by the leader, then one tile and one element.
+//
+// A template flag of the tail covers chains whose drafts were sampled from a drafter's
+// distribution Q (Eq. 1 in its general form): the test carries Q(x) and the residual is
+// max(0, P - Q), read from the target's and the drafter's row of the rejected position.
 #include "mars_top2_stream.cuh"
 
 #include <cooperative_groups.h>
@@ -243,19 +246,6 @@ __device__ __forceinline__ void tile_weights(const uint4 &raw, long long tile, i
             for (int k = 0; k < E::kVec; ++k) if (k == (int)d) w[k] = 0.0f;
         }
     }
-}
-
-// Sum of one lane's weights in a tile.
-template <int DT>
-__device__ __forceinline__ float tile_lane_sum(const uint4 &raw, long long tile, int lane, float c, float nref,
-                                               const int32_t *removed, int nrem)
-{
-    float w[Elem<DT>::kVec];
-    tile_weights<DT>(raw, tile, lane, c, nref, removed, nrem, w);
-    float ls = 0.0f;
-#pragma unroll
-    for (int k = 0; k < Elem<DT>::kVec; ++k) ls += w[k];
-    return ls;
 }
 
 // ---- the per-sequence tail kernel ---------------------------------------------------------
