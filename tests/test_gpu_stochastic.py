@@ -159,6 +159,27 @@ def test_largest_supported_tree():
     assert ref["accept_len"].max() >= 1
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_rising_rows_at_low_temperature(dtype):
+    """Rows sorted in ascending order at T = 0.05: every thread meets ever larger logits, far beyond
+    the slack of its softmax reference (which must then move), and the weights span hundreds of
+    binary orders of magnitude."""
+    w = third_candidates(synth.tree_workload("t", 8, 6, 2, 2, 60000, dtype, DEV, 91, 0.9, 2.0, 9.0, 12.0, 0.4), 91,
+                         delta=0.02)
+    srt, order = torch.sort(w.logits.float(), dim=1)
+    w.logits.copy_(srt.to(dtype))
+    inv = torch.argsort(order, dim=1).cpu().numpy()          # old id -> new id, per row
+    par = w.parent
+    for b in range(w.B):
+        for i in range(1, w.N):
+            if par[b, i] >= 0 and w.tok[b, i] >= 0:
+                w.tok[b, i] = inv[b * w.N + par[b, i], w.tok[b, i]]
+    u = synth.make_uniforms(w.B, w.N, 91)
+    for T in (0.05, 1.0):
+        run_and_compare(w.logits, w.tok, w.parent, u, 0.9, T, mars.STOCH_PLAIN, what=f"rising rows T={T}",
+                        max_close_frac=0.3)
+
+
 def test_tiny_vocabularies_one_tile():
     for V in (2, 3, 9, 200, 257):
         w = synth.tree_workload("t", 40, 6, 2, 3, V, torch.float32, DEV, 60 + V, 0.9, 1.0, 2.0, 3.0, 0.4)
