@@ -12,9 +12,9 @@
 //
 //   stoch_stream_kernel   one pass over every logits row, as in the deterministic path (16-byte
 //       streaming loads, filtered exact top-2 in registers), that also accumulates the softmax
-//       denominator online: every thread keeps a reference `ref` (a batch maximum times
-//       c = log2(e)/T, within a fixed slack of its largest) and sum = SUM 2^(z*c - ref); the
-//       batch maxima are those the top-2 filter computes anyway.  One 32-byte record
+//       denominator online: every thread keeps a reference `ref` (its largest batch maximum
+//       times c = log2(e)/T) and sum = SUM 2^(z*c - ref); the reference only moves when a
+//       batch maximum exceeds it, which the top-2 filter computes anyway.  One 32-byte record
 //       {z1, id1, z2, id2, ref, sum} per slice.
 //   stoch_tail_kernel     one thread-block cluster (1 to 8 blocks) per sequence: merges slice
 //       records, gathers the logit of every node's token from its parent's row (one scalar load
@@ -118,28 +118,16 @@ __device__ __noinline__ float soft_batch_slow(const uint4 *vbase, int v0, int nv
 // tightest limit for bf16 rows at HBM speed.  (Moving a share of them to a polynomial on the
 // FMA pipe was measured and lost: the extra issue slots cost more than the unit gained.)  The
 // fast loop carries no per-element NaN test: a NaN shows in the batch's sum and sends the
-// batch to the slow path.
-// A thread's reference need not be its exact running maximum: weights up to 2^64 are as accurate
-// in fp32 as weights up to 1, and sums of 2^64 * |V| stay far below the format's range.  So the
-// reference is set by the thread's first finite batch and moved only when a later batch maximum
-// exceeds it by more than this slack (in units of the scaled logits) -- which spares the
-// exponential unit one rescaling factor per batch (measured: 5 % on fp32 rows, none lost on bf16).
-constexpr float kRebaseSlack = 64.0f;
-
-// Moves a thread's reference up to `to` (out of line: rare after a thread's first batch).
-__device__ __noinline__ void soft_rebase(float &ref, float &sum, float to)
-{
-    sum *= ex2f(ref - to);
-    ref = to;
-}
-
+// batch to the slow path.  (Also measured and dropped: a reference that moves only when a batch
+// maximum exceeds it by a slack of 64, through an out-of-line call, to save the rescaling
+// exponential per batch -- 19 % more cycles on bf16 rows at full clock.)
 template <int DT, int U>
 __device__ __forceinline__ void soft_batch(const uint4 (&v)[U], float bm, float c, float &ref, float &sum,
                                            const uint4 *vbase, int v0, int nvec)
 {
     typedef Elem<DT> E;
     const float bmc = bm * c;
-    if (bmc > ref + kRebaseSlack) soft_rebase(ref, sum, bmc);
+    if (bmc > ref) { sum *= ex2f(ref - bmc); ref = bmc; }
     if (!(ref > -INFINITY)) return;          // nothing above -inf seen so far: all weights are 0
     const float2 nref2 = make_float2(-ref, -ref), c2 = make_float2(c, c);
     float2 a0 = make_float2(0.0f, 0.0f), a1 = a0;
