@@ -392,6 +392,22 @@ def test_sampled_plain_mode_preserves_the_target_distribution_on_the_gpu():
     assert np.all(np.abs(f - P) <= 4.5 * np.sqrt(P * (1 - P) / B) + 1e-9)
 
 
+def test_sampled_chain_without_drafts_and_many_short_sequences():
+    # K = 1: nothing to judge, the token is a draw from the only row
+    w = synth.chain_workload("t", 50, 1, 3001, torch.float32, DEV, 35, 0.9, 1.0, 4.0, 6.0, 0.3)
+    u = synth.make_uniforms(w.B, 1, 35)
+    draft = np.zeros((w.B, 0), np.int32)
+    qx = np.zeros((w.B, 0), np.float32)
+    got = mars.to_host(mars.verify_chain_sampled(w.logits, None, draft, qx, u, 0.9, 1.0, 1.0, debug=True))
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, 0.9, 1.0)
+    assert (got["accept_len"] == 0).all() and np.array_equal(got["out_tokens"], ref["out_tokens"])
+    # 3000 sequences of two rows: one block per sequence, many more blocks than the GPU holds at once
+    w, qdev, zq, draft, qx, u = sampled_case(36, 3000, 2, 517, torch.bfloat16, 1.0)
+    got = mars.to_host(mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, 1.0, 1.0, debug=True))
+    ref = orc.verify_chain_sampled(synth.to_numpy_bits(w.logits), synth.to_numpy_bits(zq), draft, qx, u, 0.9, 1.0, 1.0)
+    compare_sampled(got, ref, "many short sequences")
+
+
 def test_sampled_host_errors():
     w, qdev, zq, draft, qx, u = sampled_case(34, 2, 3, 200, torch.float32)
     with pytest.raises(mars.MarsError, match="invalid argument"):
