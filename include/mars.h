@@ -379,6 +379,52 @@ mars_status_t mars_verify_chain_sampled(const void *logits, int64_t ld, mars_dty
                                         void *cuda_stream);
 
 /*
+ * Vocabulary-parallel stochastic verification (a tensor-parallel LM head at T > 0, the setting of
+ * the paper's multi-GPU runs: Sec. 4.1, temperature 1, models above 32B on 8 GPUs).  Rank g holds
+ * columns [id_offset, id_offset + V_local) of every logits row.  Same reading of Sec. 2.2 / Eq. 1 /
+ * Eq. 3 as mars_verify_tree_stochastic; three calls with two exchanges between them:
+ *
+ *   1. mars_stochastic_shard_records: one streaming pass over the local shard -> per row a
+ *      32-byte record {float z1; int32 id1; float z2; int32 id2; float ref; float sum; 8 bytes pad}
+ *      (top-2 with GLOBAL token ids, and the shard's softmax mass sum * 2^ref in the scaled
+ *      domain z * log2(e) / T), and per node the logit of tok[i] in its parent's row if the shard
+ *      holds that column, NaN otherwise.
+ *      -- exchange: all-gather records (32 B x B*N per rank) and node logits (4 B x B*N) --
+ *   2. mars_stochastic_shard_verify: every rank merges the shards' records, walks the tree
+ *      identically (all outputs of mars_verify_tree_stochastic except the drawn token are final
+ *      and equal on all ranks), derives from the shards' masses which shard holds the token that
+ *      uniform[b, 0] selects from the residual, and only that rank reads its part of the row to
+ *      resolve it.  token_part[b] = that token (global id) on the owning rank, -1 on the others;
+ *      for sequences without a draw (status not MARS_SEQ_OK) every rank reports the fallback.
+ *      out_tokens[b, accept_len[b]] holds the fallback (the row's top-1) until step 3.
+ *      -- exchange: all-gather token_part (4 B x B per rank) --
+ *   3. mars_stochastic_shard_finish: writes the drawn token into out_tokens[b, accept_len[b]].
+ *
+ *   records_all [shards, B*N] records, node_logit_all [shards, B*N] floats, token_all [shards, B]:
+ *   shard g's array at offset g * (B*N) resp. g * B, in LOCAL memory; my_shard is this rank's
+ *   position in them.  shards <= 254.  workspace of step 1:
+ *   mars_stochastic_workspace_bytes(B, N, V_local, dt).  Results agree with the unsharded call up
+ *   to the rounding of fp32 sums taken in a different order (not bit for bit).
+ */
+mars_status_t mars_stochastic_shard_records(const void *logits_local, int64_t ld, mars_dtype_t dt,
+                                            const int32_t *tok, const int32_t *parent, int B, int N,
+                                            int V_local, int32_t id_offset, float temperature,
+                                            uint32_t flags, void *records, float *node_logit,
+                                            void *workspace, size_t workspace_bytes, void *cuda_stream);
+mars_status_t mars_stochastic_shard_verify(const void *logits_local, int64_t ld, mars_dtype_t dt,
+                                           const void *records_all, const float *node_logit_all,
+                                           int shards, int my_shard, const int32_t *tok,
+                                           const int32_t *parent, const float *uniform, int B, int N,
+                                           int V_local, int32_t id_offset, float theta, float temperature,
+                                           uint32_t flags, int32_t *accept_len, int32_t *out_tokens,
+                                           int32_t *path_nodes, int32_t *out_len, int Dcap,
+                                           int32_t *seq_status, float *node_prob, uint8_t *node_how,
+                                           int32_t *token_part, void *cuda_stream);
+mars_status_t mars_stochastic_shard_finish(const int32_t *token_all, int shards, int B, int Dcap,
+                                           const int32_t *accept_len, int32_t *out_tokens,
+                                           int32_t *seq_status, void *cuda_stream);
+
+/*
  * mars_verify_tree for callers that must not allocate device memory.  (The paper has no
  * counterpart; this is a deployment convenience of the library.)
  *

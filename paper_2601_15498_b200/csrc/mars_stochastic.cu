@@ -188,6 +188,11 @@ struct StochTailParams {
     const int32_t *tok;      // tree [B,N]; chain: draft [B,N-1]
     const int32_t *parent;   // tree [B,N] or [N]
     const float *uniform;    // [B,N]
+    // vocabulary-sharded form (mode 2): `logits` is this rank's column range [id_offset, id_offset+V)
+    const SRec *records_all;      // [G_shards, B*N] records of all shards, global token ids
+    const float *node_logit_all;  // [G_shards, B*N] logit of tok[i] in its parent's row where the shard holds it, else NaN
+    int shards, my_shard, id_offset;
+    int32_t *token_part;          // [B] the drawn token (global id) if this shard owns it, else -1
     const float *qx;         // sampled chains: [B,N-1] probability with which each draft was drawn
     const void *qlogits;     // sampled chains: drafter rows [B*(N-1), ldq], same dtype as logits
     long long ldq;
@@ -199,7 +204,7 @@ struct StochTailParams {
 
 __host__ __device__ inline size_t stoch_tail_smem_bytes(int N)
 {
-    return (size_t)N * (9 * 4 + 2) + 64;
+    return (size_t)N * (9 * 4 + 3) + 64;
 }
 
 // The kVec logits that `lane` owns in 32-lane tile `tile` of a row (element j0 = (tile*32 +
@@ -277,6 +282,8 @@ struct TailShared {
     int ctl[8];       // 0 cur, 1 accept_len, 2 status, 3 nrem, 4 draw?, 5 picked token, 6 last tile with mass,
                       // 7 node of the rejected draft (sampled chains) or -1
     int pick_tile;
+    int gstar;            // sharded form: the shard that owns the drawn token
+    double target_abs;    // ... and the mass that lies before it inside that shard
 };
 
 // ---- what a lane's elements of a tile weigh in the draw ----
@@ -359,7 +366,7 @@ __device__ __forceinline__ bool draw_in_tile(const WF &wf, long long t0, int lan
     bool good = true;
     if (whole_row) {
         good = (total > 0.0 && total < (double)INFINITY);
-        target = (double)u * total;
+        if (u >= 0.0f) target = (double)u * total;      // u < 0: `target` is already absolute
     }
     // the first lane WITH mass whose inclusive prefix passes the target (a warp scan of floating-
     // point numbers need not be monotone to the last bit, hence the explicit conditions)
@@ -387,7 +394,8 @@ __device__ __forceinline__ bool draw_in_tile(const WF &wf, long long t0, int lan
 // of every block of the cluster (the condition to call it is the same in all of them).  On return
 // the leader's sh.ctl[5] holds the drawn token, or sh.ctl[2] == 4 if the weights have no mass.
 template <int DT, class WF>
-__device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShared &sh, const WF &wf, int V, float u0)
+__device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShared &sh, const WF &wf, int V, float u0,
+                           const double *target_abs = nullptr)
 {
     typedef Elem<DT> E;
     const int G = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
@@ -443,7 +451,7 @@ __device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShare
             double before = 0.0, Wt = 0.0;
             for (int k = 0; k < kTailWarps; ++k) { if (k < warp) before += sh.wtot[k]; Wt += sh.wtot[k]; }
             inc += before;
-            const double target = (double)u0 * Wt;
+            const double target = target_abs ? *target_abs : (double)u0 * Wt;
             const bool good = (Wt > 0.0 && Wt < (double)INFINITY);
             // the first thread WITH mass whose inclusive prefix passes the target
             const unsigned hits = __ballot_sync(0xffffffffu, good && inc > target && mine > 0.0);
@@ -508,7 +516,7 @@ __device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShare
                     double Wt = 0.0;
                     for (int k = 0; k < kTailWarps; ++k) Wt += sh.part[k];
                     good = (Wt > 0.0 && Wt < (double)INFINITY);
-                    target = (double)u0 * Wt;
+                    target = target_abs ? *target_abs : (double)u0 * Wt;
                 } else target = sh.target;
                 int pick = -1, lastpos = -1;
                 double cum = 0.0, before = 0.0;
@@ -537,7 +545,8 @@ __device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShare
         }
         if (ok && warp == 0) {
             int picked = -1;
-            bool fine = draw_in_tile<DT>(wf, t0, lane, first ? 0.0 : sh.target, first, u0, &picked);
+            bool fine = draw_in_tile<DT>(wf, t0, lane, first ? (target_abs ? *target_abs : 0.0) : sh.target, first,
+                                         target_abs ? -1.0f : u0, &picked);
             fine = __all_sync(0xffffffffu, fine);
             const int all = __reduce_max_sync(0xffffffffu, picked);
             if (lane == 0) { if (!fine || all < 0) sh.ctl[2] = 4; else sh.ctl[5] = all; }
@@ -595,11 +604,17 @@ __device__ void row_softmax_cluster(cooperative_groups::cluster_group &cluster, 
     *sum_out = q;
 }
 
-// SAMPLED: chains whose drafts were sampled from a drafter's distribution (general Eq. 1): the
-// acceptance test carries the draft's own probability and the residual is max(0, P - Q).
-template <int DT, bool SAMPLED>
-__global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kernel(const StochTailParams p)
+// MODE 1 (sampled): chains whose drafts were sampled from a drafter's distribution (general
+// Eq. 1): the acceptance test carries the draft's own probability and the residual is max(0, P - Q).
+// MODE 2 (sharded): the vocabulary is split over ranks; the rows' records and the candidates'
+// logits of all shards have been gathered, every rank walks the tree identically, works out from
+// the shards' masses which shard holds the drawn token, and only that rank reads its part of the
+// row; the token is left in token_part for a last exchange.
+template <int DT, int MODE>
+__global__ void __launch_bounds__(kTailThreads, MODE == 1 ? 1 : 2) stoch_tail_kernel(const StochTailParams p)
 {
+    constexpr bool SAMPLED = MODE == 1;
+    constexpr bool SHARDED = MODE == 2;
     typedef Elem<DT> E;
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) unsigned char smem_dyn[];
@@ -624,19 +639,23 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
     float *s_u = s_e + N;
     unsigned char *s_relax = reinterpret_cast<unsigned char *>(s_u + N);
     unsigned char *s_how = s_relax + N;
+    unsigned char *s_own = s_how + N;      // sharded form: the shard that holds the node's token (255: none)
 
     // ---- rows: merge the slice records (four records' loads in flight at a time) ----
     const int32_t *par_g = p.chain ? nullptr : ((p.flags & MARS_SHARED_PARENT) ? p.parent : p.parent + (size_t)b * N);
     int bad = 0;
     for (int i = tid; i < N; i += kTailThreads) {
-        const int4 *src = reinterpret_cast<const int4 *>(p.partial + ((size_t)b * N + i) * S);
+        // slices of the row (contiguous records), or in the sharded form the row's record of every shard
+        const int4 *src = SHARDED ? reinterpret_cast<const int4 *>(p.records_all + ((size_t)b * N + i))
+                                  : reinterpret_cast<const int4 *>(p.partial + ((size_t)b * N + i) * S);
+        const size_t step = SHARDED ? (size_t)2 * gridDim.x / G * N : 2;      // in int4 units (a record is two)
         Rec acc = empty_rec();
         float ref = -INFINITY, sum = 0.0f;
         for (int k0 = 0; k0 < S; k0 += 4) {
             int4 a[4], q[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (k0 + j < S) { a[j] = __ldcg(src + 2 * (k0 + j)); q[j] = __ldcg(src + 2 * (k0 + j) + 1); }
+                if (k0 + j < S) { a[j] = __ldcg(src + step * (k0 + j)); q[j] = __ldcg(src + step * (k0 + j) + 1); }
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 if (k0 + j < S) {
@@ -672,11 +691,22 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
     for (int i = tid; i < N; i += kTailThreads) {
         float e = 0.0f, prob = 0.0f;
         const int pa = s_par[i], tk = s_tok[i];
-        if (!bad && i > 0 && pa >= 0 && tk >= 0 && tk < V) {
+        unsigned char own = 255;
+        float xs = __int_as_float(0x7fc00000);
+        if (SHARDED && !bad && i > 0 && pa >= 0 && tk >= 0) {
+            // the one shard whose column range holds the token reported its logit, the others NaN
+            const size_t R = (size_t)(gridDim.x / G) * N;
+            for (int g = 0; g < S; ++g) {
+                const float z = __ldcg(p.node_logit_all + (size_t)g * R + (size_t)b * N + i);
+                if (z == z && own == 255) { xs = z; own = (unsigned char)g; }
+            }
+        }
+        if (SHARDED) s_own[i] = own;
+        if (!bad && i > 0 && pa >= 0 && tk >= 0 && (SHARDED ? own != 255 : tk < V)) {
             const float ref = s_ref[pa], sum = s_sum[pa];
             if (ref > -INFINITY && ref < INFINITY && sum > 0.0f && sum < INFINITY) {
                 const char *rowp = (const char *)p.logits + ((size_t)b * N + pa) * (size_t)p.ld * E::kBytes;
-                const float x = E::scalar(rowp, tk);
+                const float x = SHARDED ? xs : E::scalar(rowp, tk);
                 const float t = fmaf(x, p.c, -ref);
                 e = (x == x && t == t) ? ex2f(t) : 0.0f;
                 prob = __fdiv_rn(e, sum);
@@ -700,6 +730,10 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
         while (status == 0) {
             const float ref = s_ref[cur], sum = s_sum[cur];
             nrem = 0;
+            if (SHARDED) {      // mass removed from each shard's part of this row (the tile table is idle here)
+                for (int g = lane; g < S; g += 32) sh.tile[g] = 0.0;
+                __syncwarp();
+            }
             if (!(ref > -INFINITY && ref < INFINITY && sum > 0.0f && sum < INFINITY)) { status = 4; break; }
             float rem = sum;
             int next = -1;
@@ -729,6 +763,7 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
                         if (SAMPLED) rejected = j;     // the residual needs the drafter's row, not a removal
                         else if (ex > 0.0f) {
                             rem = fmaxf(__fsub_rn(rem, ex), 0.0f);
+                            if (SHARDED && lane == 0) sh.tile[s_own[j]] += (double)ex;
                             if (lane == 0) s_removed[nrem] = x;
                             ++nrem;
                             __syncwarp();
@@ -776,6 +811,58 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
                 wf.cq = p.cq; wf.nrefq = -refq; wf.inv_sq = __fdiv_rn(1.0f, sumq);
                 draw_token<DT>(cluster, sh, wf, V, s_u[0]);
             }
+        } else if (SHARDED) {
+            // Which shard holds the drawn token follows from the shards' records: shard g's part of
+            // the row weighs sum_g * 2^(ref_g - ref) minus what the walk removed from it.
+            if (tid == 0) {
+                const size_t R = (size_t)(gridDim.x / G) * N;
+                const float ref = s_ref[cur];
+                double Wt = 0.0;
+                for (int g = 0; g < S; ++g) {
+                    const SRec *r = p.records_all + (size_t)g * R + (size_t)b * N + cur;
+                    const float rg = __ldcg(&r->ref), sg = __ldcg(&r->sum);
+                    double m = (rg > -INFINITY) ? (double)(sg * ex2f(rg - ref)) - sh.tile[g] : 0.0;
+                    if (!(m > 0.0)) m = 0.0;
+                    sh.tile[g] = m;
+                    Wt += m;
+                }
+                int pick = -1, lastpos = -1;
+                double cum = 0.0, before = 0.0;
+                const double target = (double)s_u[0] * Wt;
+                for (int g = 0; g < S && pick < 0; ++g) {
+                    if (sh.tile[g] > 0.0) lastpos = g;
+                    before = cum;
+                    cum += sh.tile[g];
+                    if (sh.tile[g] > 0.0 && cum > target) pick = g;
+                }
+                if (pick < 0) {
+                    pick = lastpos;
+                    before = 0.0;
+                    for (int g = 0; g < pick; ++g) before += sh.tile[g];
+                }
+                if (!(Wt > 0.0 && Wt < (double)INFINITY) || pick < 0) { sh.ctl[2] = 4; sh.gstar = -1; }
+                else { sh.gstar = pick; sh.target_abs = fmax(target - before, 0.0); }
+            }
+            __syncthreads();
+            // removed tokens as local column indices (those of other shards fall outside every tile)
+            for (int k = tid; k < sh.ctl[3]; k += kTailThreads) {
+                const int x = s_removed[k] - p.id_offset;
+                s_removed[k] = (x >= 0 && x < V) ? x : -0x40000000;
+            }
+            __syncthreads();
+            if (sh.gstar == p.my_shard) {        // the same decision in every block of the cluster
+                ResidualOfRow<DT> wf;
+                wf.rowp = rowp; wf.aligned = aligned; wf.V = V; wf.c = p.c; wf.nref = -s_ref[cur];
+                wf.removed = s_removed; wf.nrem = sh.ctl[3];
+                if (tid == 0) sh.ctl[5] = -1;
+                __syncthreads();
+                draw_token<DT>(cluster, sh, wf, V, s_u[0], &sh.target_abs);
+                __syncthreads();
+                if (tid == 0) {
+                    if (sh.ctl[2] == 4 || sh.ctl[5] < 0) { sh.ctl[2] = 0; sh.ctl[5] = -1; }   // rounding left this shard empty
+                    else sh.ctl[5] += p.id_offset;
+                }
+            } else if (tid == 0 && sh.gstar >= 0) sh.ctl[5] = -1;
         } else {
             ResidualOfRow<DT> wf;
             wf.rowp = rowp; wf.aligned = aligned; wf.V = V; wf.c = p.c; wf.nref = -s_ref[cur];
@@ -785,6 +872,13 @@ __global__ void __launch_bounds__(kTailThreads, SAMPLED ? 1 : 2) stoch_tail_kern
         __syncthreads();
     }
 
+    if (SHARDED && leader && tid == 0) {
+        // the drawn token travels separately: every rank reports the fallback (the row's top-1) for
+        // sequences without a draw, the owning rank the drawn token, the others -1
+        const int status = sh.ctl[2];
+        p.token_part[b] = (status != 0 || !sh.ctl[4]) ? s_id1[cur] : sh.ctl[5];
+        sh.ctl[5] = s_id1[cur];
+    }
     if (leader && tid == 0) {
         const int a = sh.ctl[1], status = sh.ctl[2];
         p.out_tokens[(size_t)b * (p.Dcap + 1) + a] = (status == 4) ? s_id1[cur] : sh.ctl[5];
@@ -929,6 +1023,71 @@ __global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const Stre
 // latency-bound work do not fit a kernel tuned to keep 64 registers and four blocks per SM
 // streaming.  It is a kernel of its own, launched behind the streaming kernel on the same stream.)
 
+// ---- vocabulary-sharded form: step 1 and step 3 kernels --------------------------------------
+
+struct ShardRecordsParams {
+    const void *logits;      // this rank's columns [id_offset, id_offset + V) of every row
+    long long ld;
+    int V, N, S, id_offset;
+    long long R;
+    uint32_t flags;
+    const SRec *partial;     // [R*S] from the streaming kernel
+    const int32_t *tok, *parent;
+    SRec *records;           // [R] out: the row's record over this shard, global token ids
+    float *node_logit;       // [R] out: logit of tok[i] in its parent's row if this shard holds it, else NaN
+};
+
+template <int DT>
+__global__ void stoch_shard_records_kernel(const ShardRecordsParams p)
+{
+    typedef Elem<DT> E;
+    const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= p.R) return;
+    const int4 *src = reinterpret_cast<const int4 *>(p.partial + (size_t)r * p.S);
+    Rec acc = empty_rec();
+    float ref = -INFINITY, sum = 0.0f;
+    for (int k = 0; k < p.S; ++k) {
+        const int4 a = __ldcg(src + 2 * k), q = __ldcg(src + 2 * k + 1);
+        Rec x;
+        x.z1 = __int_as_float(a.x); x.id1 = a.y; x.z2 = __int_as_float(a.z); x.id2 = a.w;
+        acc = merge(acc, x);
+        soft_merge(ref, sum, __int_as_float(q.x), __int_as_float(q.y));
+    }
+    SRec o;
+    o.z1 = acc.z1; o.id1 = acc.id1 == kNoId ? kNoId : acc.id1 + p.id_offset;
+    o.z2 = acc.z2; o.id2 = acc.id2 == kNoId ? kNoId : acc.id2 + p.id_offset;
+    o.ref = ref; o.sum = sum; o.pad0 = 0; o.pad1 = 0;
+    p.records[r] = o;
+    const long long b = r / p.N;
+    const int i = (int)(r - b * p.N);
+    float z = __int_as_float(0x7fc00000);
+    if (i > 0) {
+        const int pa = ((p.flags & MARS_SHARED_PARENT) ? p.parent : p.parent + (size_t)b * p.N)[i];
+        const int x = p.tok[r] - p.id_offset;
+        if (pa >= 0 && pa < i && p.tok[r] >= 0 && x >= 0 && x < p.V) {
+            const char *rowp = (const char *)p.logits + ((size_t)b * p.N + pa) * (size_t)p.ld * E::kBytes;
+            const float v = E::scalar(rowp, x);
+            z = (v == v) ? v : -INFINITY;       // a NaN logit counts as -inf; NaN means "not in this shard"
+        }
+    }
+    p.node_logit[r] = z;
+}
+
+// Step 3: the drawn token of every sequence is the one entry >= 0 among the ranks' reports (or
+// the fallback that all ranks report alike); a sequence nobody could draw for keeps the fallback
+// already in place and gets MARS_SEQ_BAD_DISTRIBUTION.
+__global__ void stoch_shard_finish_kernel(const int32_t *token_all, int shards, int B, int W, const int32_t *accept_len,
+                                          int32_t *out_tokens, int32_t *seq_status)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int t = -1;
+    for (int g = 0; g < shards; ++g) t = max(t, token_all[(size_t)g * B + b]);
+    const int a = accept_len[b];
+    if (t >= 0) out_tokens[(size_t)b * W + a] = t;
+    else if (seq_status) seq_status[b] = MARS_SEQ_BAD_DISTRIBUTION;
+}
+
 // ------------------------------------------------------------------------------- host
 
 static size_t stoch_ws_bytes(long long R, int S) { return ((size_t)R * S * sizeof(SRec) + 255) / 256 * 256; }
@@ -1038,11 +1197,11 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     cfg.numAttrs = 1;
     cudaError_t err;
     if (sd)
-        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, true>, tp)
-                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, true>, tp);
+        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, 1>, tp)
+                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, 1>, tp);
     else
-        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, false>, tp)
-                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, false>, tp);
+        err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, 0>, tp)
+                                : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, 0>, tp);
     if (err != cudaSuccess) { cudaGetLastError(); return MARS_ERR_CUDA; }
     return MARS_OK;
 }
@@ -1099,5 +1258,118 @@ mars_status_t mars_verify_chain_sampled(const void *logits, int64_t ld, mars_dty
                                 accept_len, out_tokens, nullptr, out_len, K - 1, seq_status, node_prob, node_how,
                                 workspace, workspace_bytes, cuda_stream);
 }
+
+// ---- vocabulary-sharded stochastic verification ----------------------------------------------
+
+mars_status_t mars_stochastic_shard_records(const void *logits_local, int64_t ld, mars_dtype_t dt,
+                                            const int32_t *tok, const int32_t *parent, int B, int N,
+                                            int V_local, int32_t id_offset, float temperature, uint32_t flags,
+                                            void *records, float *node_logit, void *workspace,
+                                            size_t workspace_bytes, void *cuda_stream)
+{
+    using namespace mars;
+    if (B < 1 || N < 1 || V_local < 2 || !logits_local || !tok || !parent || !records || !node_logit)
+        return MARS_ERR_INVALID_ARG;
+    if (ld < V_local || id_offset < 0 || ((uintptr_t)records & 15)) return MARS_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !(temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
+    if (flags & ~MARS_SHARED_PARENT) return MARS_ERR_UNSUPPORTED;
+    if (!stoch_sizes_supported(B, N, V_local, (int)dt)) return MARS_ERR_UNSUPPORTED;
+    if ((uintptr_t)logits_local % (dt == MARS_BF16 ? 2 : 4)) return MARS_ERR_INVALID_ARG;
+    const double cd = 1.4426950408889634074 / (double)temperature;
+    if (!(cd < 3.0e38)) return MARS_ERR_INVALID_ARG;
+    const long long R = (long long)B * N;
+    const Split sp = choose_split(R, V_local, (int)dt);
+    if (R * sp.S > 0x7fffffffll) return MARS_ERR_UNSUPPORTED;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < stoch_ws_bytes(R, sp.S)) return MARS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    StreamParams sp1;
+    sp1.logits = logits_local; sp1.ld = ld; sp1.V = V_local; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
+    sp1.partial = (SRec *)workspace;
+    const unsigned grid = (unsigned)(R * sp.S);
+    if (dt == MARS_BF16) stoch_stream_kernel<MARS_BF16, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
+    else stoch_stream_kernel<MARS_FP32, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
+    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    ShardRecordsParams rp;
+    rp.logits = logits_local; rp.ld = ld; rp.V = V_local; rp.N = N; rp.S = sp.S; rp.id_offset = id_offset; rp.R = R;
+    rp.flags = flags; rp.partial = sp1.partial; rp.tok = tok; rp.parent = parent;
+    rp.records = (SRec *)records; rp.node_logit = node_logit;
+    const unsigned g2 = (unsigned)((R + 255) / 256);
+    if (dt == MARS_BF16) stoch_shard_records_kernel<MARS_BF16><<<g2, 256, 0, st>>>(rp);
+    else stoch_shard_records_kernel<MARS_FP32><<<g2, 256, 0, st>>>(rp);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+}
+
+mars_status_t mars_stochastic_shard_verify(const void *logits_local, int64_t ld, mars_dtype_t dt,
+                                           const void *records_all, const float *node_logit_all, int shards,
+                                           int my_shard, const int32_t *tok, const int32_t *parent,
+                                           const float *uniform, int B, int N, int V_local, int32_t id_offset,
+                                           float theta, float temperature, uint32_t flags, int32_t *accept_len,
+                                           int32_t *out_tokens, int32_t *path_nodes, int32_t *out_len, int Dcap,
+                                           int32_t *seq_status, float *node_prob, uint8_t *node_how,
+                                           int32_t *token_part, void *cuda_stream)
+{
+    using namespace mars;
+    if (B < 1 || N < 1 || V_local < 2 || !logits_local || !records_all || !node_logit_all || !tok || !parent ||
+        !uniform || !accept_len || !out_tokens || !out_len || !token_part)
+        return MARS_ERR_INVALID_ARG;
+    if (shards < 1 || shards > 254 || my_shard < 0 || my_shard >= shards || ld < V_local || Dcap < 0 || id_offset < 0 ||
+        theta != theta || ((uintptr_t)records_all & 15))
+        return MARS_ERR_INVALID_ARG;
+    if (!(temperature > 0.0f) || !(temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO | MARS_STOCH_PLAIN |
+                  MARS_STOCH_RELAX_ONLY))
+        return MARS_ERR_UNSUPPORTED;
+    if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
+    if ((flags & MARS_STOCH_PLAIN) && (flags & MARS_STOCH_RELAX_ONLY)) return MARS_ERR_INVALID_ARG;
+    rule_threshold(&theta, &flags);
+    if (!stoch_sizes_supported(B, N, V_local, (int)dt)) return MARS_ERR_UNSUPPORTED;
+    const double cd = 1.4426950408889634074 / (double)temperature;
+    if (!(cd < 3.0e38)) return MARS_ERR_INVALID_ARG;
+    StochTailParams tp = {};
+    tp.logits = logits_local; tp.ld = ld; tp.V = V_local; tp.N = N; tp.S = shards; tp.c = (float)cd; tp.theta = theta;
+    tp.flags = flags; tp.chain = 0; tp.Dcap = Dcap; tp.partial = nullptr;
+    tp.tok = tok; tp.parent = parent; tp.uniform = uniform;
+    tp.records_all = (const SRec *)records_all; tp.node_logit_all = node_logit_all;
+    tp.shards = shards; tp.my_shard = my_shard; tp.id_offset = id_offset; tp.token_part = token_part;
+    tp.accept_len = accept_len; tp.out_tokens = out_tokens; tp.path_nodes = path_nodes;
+    tp.out_len = out_len; tp.seq_status = seq_status; tp.node_prob = node_prob; tp.node_how = node_how;
+    const int kv = dt == MARS_BF16 ? 8 : 4;
+    const long long ntiles = ((long long)V_local + 32 * kv - 1) / (32 * kv);
+    int G = 1;
+    for (int g = kTailCluster; g > 1; g >>= 1)
+        if ((long long)B * g <= 2 * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
+    const char *force = getenv("MARS_STOCH_TAIL_CLUSTER");   // test hook: 1, 2, 4 or 8
+    if (force) {
+        const int g = atoi(force);
+        if ((g == 1 || g == 2 || g == 4 || g == 8) && (g == 1 || (ntiles + g - 1) / g <= kMaxTilesPerBlock)) G = g;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((long long)B * G));
+    cfg.blockDim = dim3(kTailThreads);
+    cfg.dynamicSmemBytes = stoch_tail_smem_bytes(N);
+    cfg.stream = (cudaStream_t)cuda_stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)G;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = (dt == MARS_BF16) ? cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_BF16, 2>, tp)
+                                              : cudaLaunchKernelEx(&cfg, stoch_tail_kernel<MARS_FP32, 2>, tp);
+    if (err != cudaSuccess) { cudaGetLastError(); return MARS_ERR_CUDA; }
+    return MARS_OK;
+}
+
+mars_status_t mars_stochastic_shard_finish(const int32_t *token_all, int shards, int B, int Dcap,
+                                           const int32_t *accept_len, int32_t *out_tokens, int32_t *seq_status,
+                                           void *cuda_stream)
+{
+    if (!token_all || !accept_len || !out_tokens || shards < 1 || B < 1 || Dcap < 0) return MARS_ERR_INVALID_ARG;
+    mars::stoch_shard_finish_kernel<<<(unsigned)((B + 255) / 256), 256, 0, (cudaStream_t)cuda_stream>>>(
+        token_all, shards, B, Dcap + 1, accept_len, out_tokens, seq_status);
+    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+}
+
 
 }  // extern "C"

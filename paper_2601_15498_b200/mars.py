@@ -88,6 +88,14 @@ def lib() -> ctypes.CDLL:
             L.mars_verify_chain_sampled.argtypes = [vp, i64, i32, vp, i64, vp, vp, vp, i32, i32, i32, f32, f32, f32,
                                                     u32, vp, vp, vp, vp, vp, vp, vp, sz, vp]
             L.mars_verify_chain_sampled.restype = i32
+            L.mars_stochastic_shard_records.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, i32, f32, u32, vp, vp,
+                                                        vp, sz, vp]
+            L.mars_stochastic_shard_records.restype = i32
+            L.mars_stochastic_shard_verify.argtypes = [vp, i64, i32, vp, vp, i32, i32, vp, vp, vp, i32, i32, i32,
+                                                       i32, f32, f32, u32, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]
+            L.mars_stochastic_shard_verify.restype = i32
+            L.mars_stochastic_shard_finish.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
+            L.mars_stochastic_shard_finish.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -396,6 +404,79 @@ def verify_chain_sampled(logits: torch.Tensor, draft_logits: torch.Tensor, draft
             workspace.data_ptr(), wbytes, _stream())
     _check(code, "mars_verify_chain_sampled")
     out["_keepalive"] = (draft, draft_prob, uniform, draft_logits, workspace)
+    return out
+
+
+def stochastic_shard_records(logits_local: torch.Tensor, tok, parent, id_offset: int, temperature: float,
+                             V_local: int | None = None, flags: int = 0,
+                             workspace: torch.Tensor | None = None):
+    """mars_stochastic_shard_records on the current stream: (records int32 [B*N, 8], node_logit
+    float32 [B*N]) of one vocabulary shard."""
+    dev = logits_local.device
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    dt, ld, V_local = _logits_args(logits_local, B * N, V_local)
+    workspace, wbytes = _stoch_workspace(B, N, V_local, dt, dev, workspace)
+    records = torch.empty((B * N, 8), dtype=torch.int32, device=dev)
+    node_logit = torch.empty((B * N,), dtype=torch.float32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_stochastic_shard_records(
+            logits_local.data_ptr(), ld, dt, tok.data_ptr(), parent.data_ptr(), B, N, V_local, int(id_offset),
+            float(temperature), flags, records.data_ptr(), node_logit.data_ptr(), workspace.data_ptr(), wbytes,
+            _stream())
+    _check(code, "mars_stochastic_shard_records")
+    return records, node_logit
+
+
+def stochastic_shard_verify(logits_local: torch.Tensor, records_all: torch.Tensor, node_logit_all: torch.Tensor,
+                            my_shard: int, id_offset: int, tok, parent, uniform, theta: float,
+                            temperature: float, flags: int = 0, Dcap: int | None = None,
+                            V_local: int | None = None, debug: bool = False, out: dict | None = None):
+    """mars_stochastic_shard_verify on the current stream: records_all int32 [G, B*N, 8],
+    node_logit_all float32 [G, B*N].  Returns (outputs, token_part int32 [B])."""
+    dev = logits_local.device
+    tok = _dev_i32(tok, dev)
+    parent = _dev_i32(parent, dev)
+    uniform = _dev_f32(uniform, dev)
+    B, N = tok.shape
+    if parent.dim() == 1:
+        flags |= SHARED_PARENT
+    dt, ld, V_local = _logits_args(logits_local, B * N, V_local)
+    G = records_all.shape[0]
+    if not (records_all.is_cuda and records_all.dtype == torch.int32 and records_all.is_contiguous()
+            and tuple(records_all.shape) == (G, B * N, 8) and node_logit_all.is_contiguous()
+            and node_logit_all.dtype == torch.float32 and tuple(node_logit_all.shape) == (G, B * N)):
+        raise MarsError("records_all must be int32 [G, B*N, 8] and node_logit_all float32 [G, B*N], contiguous")
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    if out is None:
+        out = alloc_stochastic_outputs(B, N, Dcap, dev, debug)
+    token_part = torch.full((B,), -777, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        code = lib().mars_stochastic_shard_verify(
+            logits_local.data_ptr(), ld, dt, records_all.data_ptr(), node_logit_all.data_ptr(), G, int(my_shard),
+            tok.data_ptr(), parent.data_ptr(), uniform.data_ptr(), B, N, V_local, int(id_offset), float(theta),
+            float(temperature), flags, out["accept_len"].data_ptr(), out["out_tokens"].data_ptr(),
+            out["path_nodes"].data_ptr(), out["out_len"].data_ptr(), Dcap, out["seq_status"].data_ptr(),
+            out["node_prob"].data_ptr() if "node_prob" in out else None,
+            out["node_how"].data_ptr() if "node_how" in out else None, token_part.data_ptr(), _stream())
+    _check(code, "mars_stochastic_shard_verify")
+    out["_keepalive"] = (tok, parent, uniform, records_all, node_logit_all)
+    return out, token_part
+
+
+def stochastic_shard_finish(token_all: torch.Tensor, out: dict) -> dict:
+    """mars_stochastic_shard_finish on the current stream: token_all int32 [G, B]."""
+    if not (token_all.is_cuda and token_all.dtype == torch.int32 and token_all.is_contiguous() and token_all.dim() == 2):
+        raise MarsError("token_all must be a contiguous int32 [G, B] device tensor")
+    G, B = token_all.shape
+    Dcap = out["out_tokens"].shape[1] - 1
+    with torch.cuda.device(token_all.device):
+        code = lib().mars_stochastic_shard_finish(token_all.data_ptr(), G, B, Dcap, out["accept_len"].data_ptr(),
+                                                  out["out_tokens"].data_ptr(), out["seq_status"].data_ptr(), _stream())
+    _check(code, "mars_stochastic_shard_finish")
     return out
 
 

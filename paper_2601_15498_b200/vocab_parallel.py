@@ -6,6 +6,9 @@ all-gather those records into local memory (NCCL through ``torch.distributed``; 
 per rank), and every rank then merges and verifies locally (``mars_verify_records``).  The
 merge operator is associative and commutative, so all ranks obtain outputs bit-identical to a
 single-GPU ``mars_verify_tree`` on the unsharded logits.
+
+The stochastic form (``verify_tree_stochastic_vocab_parallel``) has two exchange steps: the
+records (with each shard's softmax mass) and the candidates' logits, then the drawn tokens.
 """
 from __future__ import annotations
 
@@ -47,3 +50,34 @@ def verify_tree_vocab_parallel(logits_local: torch.Tensor, id_offset: int, tok, 
     dist.all_gather_into_tensor(flat, rec, group=group)           # rank r's records at rows [r*R, (r+1)*R)
     gathered = flat.view((world,) + tuple(rec.shape))
     return verify(gathered, tok, parent, theta, flags=flags, debug=debug)
+
+
+def _all_gather(t: torch.Tensor, world: int, group) -> torch.Tensor:
+    t = t.contiguous()
+    flat = torch.empty((world * t.shape[0],) + tuple(t.shape[1:]), dtype=t.dtype, device=t.device)
+    dist.all_gather_into_tensor(flat, t, group=group)
+    return flat.view((world,) + tuple(t.shape))
+
+
+def verify_tree_stochastic_vocab_parallel(logits_local: torch.Tensor, id_offset: int, tok, parent, uniform,
+                                          theta: float, temperature: float, group=None, flags: int = 0,
+                                          debug: bool = False, records=None, verify=None, finish=None) -> dict:
+    """One vocabulary-parallel stochastic verification step on this rank: per-shard records and
+    candidate logits, an all-gather of both (36 B x rows per rank), the walk and the owning
+    shard's draw, an all-gather of the drawn tokens (4 B x sequences per rank), and the final
+    placement.  ``records`` / ``verify`` / ``finish`` default to the CUDA library's entry points;
+    they are parameters so that the collective plumbing can be exercised with CPU ranks."""
+    if records is None or verify is None or finish is None:
+        from . import mars
+        records = records or mars.stochastic_shard_records
+        verify = verify or mars.stochastic_shard_verify
+        finish = finish or mars.stochastic_shard_finish
+    world = dist.get_world_size(group)
+    rank = dist.get_rank(group)
+    rec, zl = records(logits_local, tok, parent, id_offset, temperature)
+    rec_all = _all_gather(rec, world, group)
+    zl_all = _all_gather(zl, world, group)
+    out, token_part = verify(logits_local, rec_all, zl_all, rank, id_offset, tok, parent, uniform, theta,
+                             temperature, flags=flags, debug=debug)
+    token_all = _all_gather(token_part, world, group)
+    return finish(token_all, out)

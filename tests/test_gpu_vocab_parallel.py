@@ -82,3 +82,84 @@ def test_sharded_lm_head_equals_unsharded_bit_for_bit(world):
     out = mars.to_host(mars.verify_records(torch.stack(recs), tok, w.parent, 0.9, debug=True))
     assert_same(out, ref, KEYS_TREE, f"lm head world={world}")
     assert (out["seq_status"] == 0).all() and out["accept_len"].max() >= 1
+
+
+# ---------------------------------------------------------------- stochastic form (T > 0)
+
+def sharded_stochastic(logits, tok, parent, u, theta, T, ranges, flags=0):
+    """The ranks' calls made one after the other on one GPU, stacked as the all-gathers would
+    deliver them; returns every rank's final outputs."""
+    from stochastic_checks import host_f64  # noqa: F401  (shared tolerance policy lives there)
+    G = len(ranges)
+    recs, zls = [], []
+    for lo, hi in ranges:
+        r, z = mars.stochastic_shard_records(logits[:, lo:hi], tok, parent, lo, T, V_local=hi - lo)
+        recs.append(r)
+        zls.append(z)
+    rec_all, zl_all = torch.stack(recs), torch.stack(zls)
+    outs, parts = [], []
+    for g, (lo, hi) in enumerate(ranges):
+        o, part = mars.stochastic_shard_verify(logits[:, lo:hi], rec_all, zl_all, g, lo, tok, parent, u, theta, T,
+                                               flags, V_local=hi - lo, debug=True)
+        outs.append(o)
+        parts.append(part)
+    token_all = torch.stack(parts)
+    return [mars.to_host(mars.stochastic_shard_finish(token_all, o)) for o in outs], token_all.cpu().numpy()
+
+
+@pytest.mark.parametrize("world", [1, 2, 3, 8])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_stochastic_sharded_against_the_oracle(world, dtype):
+    import stochastic_checks as sc
+    w = synth.tree_workload("vps", 12, 20, 4, 3, 40009, dtype, DEV, 120 + world, 0.9, 1.0, 9.0, 16.0, 0.4)
+    u = synth.make_uniforms(w.B, w.N, 120 + world)
+    u[::3, 1:] = np.float32(0.99999)            # a third of the sequences draw at the root
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, w.theta, 1.0)
+    ranges = vocab_parallel.shard_ranges(w.V, world)
+    for flags in (0, mars.STOCH_PLAIN):
+        ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, w.theta, 1.0, flags)
+        outs, token_all = sharded_stochastic(w.logits, w.tok, w.parent, u, w.theta, 1.0, ranges, flags)
+        for g, o in enumerate(outs):
+            sc.compare(o, ref, w.tok, w.parent, sc.host_f64(w.logits), u, 1.0, f"world={world} rank={g}",
+                       max_close_frac=0.1)
+        for k in ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "node_how"):
+            for o in outs[1:]:
+                assert np.array_equal(o[k], outs[0][k]), k      # every rank ends with the same result
+        owners = (token_all >= 0).sum(axis=0)
+        ok = outs[0]["seq_status"] == 0
+        assert (owners[ok] == 1).all()                           # exactly one shard drew each token
+
+
+def test_stochastic_sharded_degenerate_rows_and_tiny_shards():
+    import stochastic_checks as sc
+    V = 3000
+    w = synth.tree_workload("vps", 8, 10, 3, 3, V, torch.float32, DEV, 131, 0.9, 1.0, 5.0, 8.0, 0.4)
+    lg = w.logits.clone()
+    lg[0 * 10 + 0, :] = float("-inf")
+    lg[1 * 10 + 0, 17] = float("inf")
+    lg[2 * 10 + 0, 100:1200] = float("nan")
+    lg[3 * 10 + 0, 0:2000] = float("-inf")       # whole shards without mass
+    u = synth.make_uniforms(w.B, w.N, 131)
+    ranges = [(0, 2), (2, 1000), (1000, 1003), (1003, 2000), (2000, V)]
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(lg), w.tok, w.parent, u, 0.9, 1.0)
+    outs, _ = sharded_stochastic(lg, w.tok, w.parent, u, 0.9, 1.0, ranges)
+    assert ref["seq_status"].tolist()[:2] == [4, 4]
+    for o in outs:
+        sc.compare(o, ref, w.tok, w.parent, sc.host_f64(lg), u, 1.0, "degenerate sharded", max_close_frac=0.3)
+
+
+@pytest.mark.parametrize("cluster", [1, 4, 8])
+def test_stochastic_sharded_cluster_shapes(cluster, monkeypatch):
+    import stochastic_checks as sc
+    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    w = synth.tree_workload("vps", 30, 6, 2, 2, 90011, torch.bfloat16, DEV, 140, 0.9, 1.0, 3.0, 6.0, 0.4)
+    u = synth.make_uniforms(w.B, w.N, 140)
+    u[::2, 1:] = np.float32(0.99999)
+    ref = orc.verify_tree_stochastic(synth.to_numpy_bits(w.logits), w.tok, w.parent, u, 0.9, 1.0, mars.STOCH_PLAIN)
+    outs, _ = sharded_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, vocab_parallel.shard_ranges(w.V, 4),
+                                 mars.STOCH_PLAIN)
+    for g, o in enumerate(outs):
+        sc.compare(o, ref, w.tok, w.parent, sc.host_f64(w.logits), u, 1.0, f"cluster {cluster} rank {g}",
+                   max_close_frac=0.1)
+    drawn = outs[0]["out_tokens"][np.arange(w.B), outs[0]["accept_len"]]
+    assert drawn.min() < w.V // 4 and drawn.max() > 3 * w.V // 4       # tokens from the first and the last shard

@@ -79,3 +79,59 @@ def test_two_rank_all_gather_layout_and_content():
     cand = np.concatenate([g0[0][:, [1, 3]], g0[1][:, [1, 3]]], axis=1)
     for r in range(10):
         assert full_idx[r, 0] in cand[r] and full_idx[r, 1] in cand[r]
+
+
+def _rank_stochastic(rank, world, port, q):
+    """Stand-ins for the three library calls (no arithmetic of the method: they only tag what they
+    are given), to check what the orchestration gathers and in which layout."""
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    B, N = 3, 4
+    seen = {}
+
+    def records(local, tok, parent, off, T):
+        rec = torch.full((B * N, 8), rank, dtype=torch.int32)
+        rec[:, 1] = off
+        return rec, torch.full((B * N,), float(rank))
+
+    def verify(local, rec_all, zl_all, my_shard, off, tok, parent, uniform, theta, T, flags=0, debug=False):
+        seen["rec"], seen["zl"], seen["me"] = rec_all.clone(), zl_all.clone(), my_shard
+        part = torch.full((B,), -1, dtype=torch.int32)
+        part[rank::world] = 100 + rank          # this "shard" owns every world-th sequence
+        return {"accept_len": torch.zeros(B, dtype=torch.int32)}, part
+
+    def finish(token_all, out):
+        out["token_all"] = token_all.clone()
+        return out
+
+    lo, hi = vocab_parallel.shard_ranges(64, world)[rank]
+    out = vocab_parallel.verify_tree_stochastic_vocab_parallel(
+        torch.zeros((B * N, hi - lo)), lo, np.zeros((B, N), np.int32), np.zeros((B, N), np.int32),
+        np.zeros((B, N), np.float32), 0.9, 1.0, records=records, verify=verify, finish=finish)
+    q.put((rank, seen["rec"].numpy(), seen["zl"].numpy(), seen["me"], out["token_all"].numpy()))
+    dist.destroy_process_group()
+
+
+def test_two_rank_stochastic_exchanges():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_rank_stochastic, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = {}
+    for _ in procs:
+        r, rec, zl, me, tok_all = q.get(timeout=120)
+        got[r] = (rec, zl, me, tok_all)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    lo1 = vocab_parallel.shard_ranges(64, 2)[1][0]
+    for r in (0, 1):
+        rec, zl, me, tok_all = got[r]
+        assert me == r and rec.shape == (2, 12, 8) and zl.shape == (2, 12) and tok_all.shape == (2, 3)
+        assert (rec[0][:, 0] == 0).all() and (rec[1][:, 0] == 1).all()          # shard g at position g
+        assert (rec[0][:, 1] == 0).all() and (rec[1][:, 1] == lo1).all()
+        assert (zl[0] == 0).all() and (zl[1] == 1).all()
+        assert tok_all.max(axis=0).tolist() == [100, 101, 100]                  # one owner per sequence
+    assert np.array_equal(got[0][3], got[1][3])
