@@ -242,12 +242,13 @@ __device__ __forceinline__ void tile_weights(const uint4 &raw, long long tile, i
     const long long j0 = (tile * 32 + lane) * E::kVec;
 #pragma unroll
     for (int k = 0; k < E::kVec; ++k) {
-        const float x = E::elem(raw, k);
-        const float t = fmaf(x, c, nref);
-        w[k] = (x == x && t == t) ? ex2f(t) : 0.0f;
+        // NaN -> -inf with one max (weight 0); the reference of a row that is drawn from is finite
+        // and at least every z*c, so the exponent is never NaN or positive beyond rounding
+        const float x = fmaxf(E::elem(raw, k), -INFINITY);
+        w[k] = ex2f(fmaf(x, c, nref));
     }
     for (int r = 0; r < nrem; ++r) {
-        const long long d = (long long)removed[r] - j0;
+        const int d = removed[r] - (int)j0;
         if (d >= 0 && d < E::kVec) {
 #pragma unroll
             for (int k = 0; k < E::kVec; ++k) if (k == (int)d) w[k] = 0.0f;
