@@ -405,16 +405,19 @@ __device__ void draw_token(cooperative_groups::cluster_group &cluster, TailShare
     const long long ntiles = ((long long)V + 32 * E::kVec - 1) / (32 * E::kVec);
     const long long tpc = (ntiles + G - 1) / G;          // tiles per block of the cluster
     if (tpc <= kMaxTilesPerBlock) {                       // the host launches clusters only if this holds
-        // (1) every block: per-tile sums of its share of the row, eight tiles per warp at a time
+        // (1) every block: per-tile sums of its share of the row
         const long long t_lo = min(ntiles, (long long)rank * tpc), t_hi = min(ntiles, t_lo + tpc);
-        for (long long t = t_lo + warp * 8; t < t_hi; t += kTailWarps * 8) {
+        // up to eight tiles per warp at a time, fewer when the block's share is small, so that all
+        // warps take part
+        const int per = (int)min(8ll, max(1ll, (t_hi - t_lo + kTailWarps - 1) / kTailWarps));
+        for (long long t = t_lo + warp * per; t < t_hi; t += kTailWarps * per) {
             typename WF::Raw raw[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                if (t + i < t_hi) raw[i] = wf.load(t + i, lane);
+                if (i < per && t + i < t_hi) raw[i] = wf.load(t + i, lane);
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                if (t + i < t_hi) {
+                if (i < per && t + i < t_hi) {
                     float ls = lane_sum<DT>(wf, raw[i], t + i, lane);
 #pragma unroll
                     for (int m = 16; m > 0; m >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, m);
