@@ -20,11 +20,6 @@ of several times over these and flag only a few decisions in 10^5.
 import os
 
 import numpy as np
-import pytest
-import torch
-
-from oracle import mars_oracle as orc
-from paper_2601_15498_b200 import mars, synth
 
 DEV = os.environ.get("MARS_TEST_DEVICE", "cuda:0")
 PROB_RTOL = 2e-5

@@ -1,7 +1,5 @@
 """Parity of stochastic (T > 0) verification with the CPU oracle, through the C ABI.  The
 comparison policy and its tolerances are in stochastic_checks.py."""
-import os
-
 import numpy as np
 import pytest
 import torch

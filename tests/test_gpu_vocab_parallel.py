@@ -89,7 +89,6 @@ def test_sharded_lm_head_equals_unsharded_bit_for_bit(world):
 def sharded_stochastic(logits, tok, parent, u, theta, T, ranges, flags=0):
     """The ranks' calls made one after the other on one GPU, stacked as the all-gathers would
     deliver them; returns every rank's final outputs."""
-    from stochastic_checks import host_f64  # noqa: F401  (shared tolerance policy lives there)
     G = len(ranges)
     recs, zls = [], []
     for lo, hi in ranges:
