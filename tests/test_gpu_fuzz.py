@@ -113,7 +113,7 @@ def test_stochastic_tree(seed, monkeypatch):
         monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
     for _ in range(3):
         c = random_case(rng, stochastic=True)
-        T = float(rng.choice([0.3, 0.7, 1.0, 1.7]))
+        T = float(rng.choice([0.02, 0.3, 0.7, 1.0, 1.7, 50.0]))
         flags = c["flags"] | int(rng.choice([0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY]))
         u = synth.make_uniforms(c["B"], c["N"], int(rng.integers(1 << 30)))
         if rng.random() < 0.3:
