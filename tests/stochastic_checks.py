@@ -1,4 +1,5 @@
-"""Comparison policy shared by the GPU tests of stochastic verification (not a test module).
+"""Comparison policy and case builders shared by the GPU tests of stochastic verification (not a
+test module).
 
 The oracle evaluates the softmax in fp64, the library in fp32 with the hardware 2^x; the
 uniforms are inputs shared by both.  Bar:
@@ -20,6 +21,9 @@ of several times over these and flag only a few decisions in 10^5.
 import os
 
 import numpy as np
+import torch
+
+from paper_2601_15498_b200 import mars, synth
 
 DEV = os.environ.get("MARS_TEST_DEVICE", "cuda:0")
 PROB_RTOL = 2e-5
@@ -100,3 +104,60 @@ def host_f64(logits, V=None):
     return x if V is None else x[:, :V]
 
 
+
+
+# ---- sampled chains and the vocabulary-sharded form: shared case builders and checks ----
+
+def sampled_case(seed, B, K, V, dtype, sigma_q=1.0, T=1.0, Tq=1.0, ld_pad=0):
+    """Target rows from the chain recipe, drafter rows = target rows + noise, drafts really drawn
+    from the drafter's softmax (torch, on the host) with their probabilities."""
+    w = synth.chain_workload("t", B, K, V, dtype, DEV, seed, 0.9, 1.5, 6.0, 10.0, 0.4)
+    g = torch.Generator().manual_seed(seed)
+    z = w.logits.float().cpu().reshape(B, K, V)[:, :K - 1].reshape(-1, V)
+    zq = (z + torch.randn(z.shape, generator=g) * sigma_q).to(dtype)
+    Q = torch.softmax(zq.double() / Tq, dim=1)
+    draft = torch.multinomial(Q, 1, generator=g).reshape(-1)
+    qx = Q[torch.arange(Q.shape[0]), draft].float()
+    qdev = torch.full((B * (K - 1), V + ld_pad), 55.0, dtype=dtype, device=DEV)
+    qdev[:, :V] = zq.to(DEV)
+    u = synth.make_uniforms(B, K, seed)
+    return w, qdev, zq, draft.reshape(B, K - 1).numpy().astype(np.int32), qx.reshape(B, K - 1).numpy(), u
+
+
+def compare_sampled(got, ref, what):
+    B = ref["accept_len"].shape[0]
+    n_close = 0
+    for b in range(B):
+        a = int(ref["accept_len"][b])
+        same_walk = all(np.array_equal(got[k][b], ref[k][b]) for k in ("accept_len", "out_len", "seq_status", "node_how")) \
+            and np.array_equal(got["out_tokens"][b, :a], ref["out_tokens"][b, :a])
+        if not same_walk:
+            assert ref["margin"][b, 0] < DECISION_TOL, (what, b, ref["margin"][b])
+            n_close += 1
+            continue
+        if got["out_tokens"][b, a] != ref["out_tokens"][b, a]:
+            # the draw margin of this oracle is in units of total probability
+            assert ref["margin"][b, 1] < 2e-6, (what, b, got["out_tokens"][b], ref["out_tokens"][b], ref["margin"][b])
+            n_close += 1
+    np.testing.assert_allclose(got["node_prob"], ref["node_prob"], rtol=PROB_RTOL, atol=1e-30, err_msg=what)
+    assert n_close <= max(2, B // 50), (what, n_close)
+
+
+def sharded_stochastic(logits, tok, parent, u, theta, T, ranges, flags=0):
+    """The ranks' calls made one after the other on one GPU, stacked as the all-gathers would
+    deliver them; returns every rank's final outputs."""
+    G = len(ranges)
+    recs, zls = [], []
+    for lo, hi in ranges:
+        r, z = mars.stochastic_shard_records(logits[:, lo:hi], tok, parent, lo, T, V_local=hi - lo)
+        recs.append(r)
+        zls.append(z)
+    rec_all, zl_all = torch.stack(recs), torch.stack(zls)
+    outs, parts = [], []
+    for g, (lo, hi) in enumerate(ranges):
+        o, part = mars.stochastic_shard_verify(logits[:, lo:hi], rec_all, zl_all, g, lo, tok, parent, u, theta, T,
+                                               flags, V_local=hi - lo, debug=True)
+        outs.append(o)
+        parts.append(part)
+    token_all = torch.stack(parts)
+    return [mars.to_host(mars.stochastic_shard_finish(token_all, o)) for o in outs], token_all.cpu().numpy()

@@ -123,3 +123,54 @@ def test_stochastic_tree(seed, monkeypatch):
         ref = orc.verify_tree_stochastic(c["host"], c["tok"], c["parent"], u, c["theta"], T, flags, c["Dcap"])
         ts.compare(got, ref, c["tok"], c["parent"], c["z"].double().numpy(), u, T, f"fuzz {seed}",
                    max_close_frac=0.25)
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_sampled_chains(seed, monkeypatch):
+    rng = np.random.default_rng(9000 + seed)
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    if rng.random() < 0.5:
+        monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(int(rng.choice([1, 2, 4, 8]))))
+    else:
+        monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+    for _ in range(3):
+        B, K = int(rng.integers(1, 40)), int(rng.choice([2, 3, 5, 9]))
+        V = int(rng.choice([9, 257, 1000, 5001, 40000]))
+        dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+        T, Tq = float(rng.choice([0.5, 1.0, 2.0])), float(rng.choice([0.7, 1.0, 1.5]))
+        flags = int(rng.choice([0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY]))
+        w, qdev, zq, draft, qx, u = ts.sampled_case(int(rng.integers(1 << 20)), B, K, V, dtype,
+                                                    float(rng.choice([0.3, 1.0, 2.0])), T, Tq,
+                                                    ld_pad=int(rng.choice([0, 3])))
+        if rng.random() < 0.3:
+            u[:, 1:] = np.float32(0.9999)
+        got = mars.to_host(mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, T, Tq, flags, V=V, debug=True))
+        ref = orc.verify_chain_sampled(synth.to_numpy_bits(w.logits), synth.to_numpy_bits(zq), draft, qx, u, 0.9, T, Tq,
+                                       flags)
+        ts.compare_sampled(got, ref, f"fuzz sampled {seed}")
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_sharded_stochastic_tree(seed, monkeypatch):
+    rng = np.random.default_rng(7000 + seed)
+    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+    for _ in range(2):
+        c = random_case(rng, stochastic=True)
+        if c["V"] < 8:
+            continue
+        V = c["V"]
+        cuts = sorted(set(int(x) for x in rng.integers(2, V - 2, int(rng.integers(0, 4)))))
+        edges = [0] + [x for x in cuts if 2 <= x <= V - 2] + [V]
+        ranges = [(a, b) for a, b in zip(edges, edges[1:]) if b - a >= 2]
+        if not ranges or ranges[0][0] != 0 or ranges[-1][1] != V or any(a2 != b1 for (_, b1), (a2, _) in zip(ranges, ranges[1:])):
+            ranges = [(0, V)]
+        T = float(rng.choice([0.5, 1.0, 2.0]))
+        flags = c["flags"] | int(rng.choice([0, mars.STOCH_PLAIN]))
+        u = synth.make_uniforms(c["B"], c["N"], int(rng.integers(1 << 30)))
+        logits = c["view"].contiguous()
+        ref = orc.verify_tree_stochastic(c["host"], c["tok"], c["parent"], u, c["theta"], T, flags)
+        outs, _ = ts.sharded_stochastic(logits, c["tok"], c["parent"], u, c["theta"], T, ranges, flags)
+        for o in outs:
+            ts.compare(o, ref, c["tok"], c["parent"], c["z"].double().numpy(), u, T, f"fuzz sharded {seed}",
+                       max_close_frac=0.25)

@@ -7,8 +7,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
-from stochastic_checks import (DECISION_TOL, DEV, PROB_RTOL, STATS, check_walk_is_valid, compare,
-                               host_f64)
+from stochastic_checks import (DEV, STATS, check_walk_is_valid, compare, compare_sampled, host_f64,
+                               sampled_case)
 
 pytestmark = pytest.mark.gpu
 
@@ -294,41 +294,6 @@ def test_full_size_batch_sampled_sequences():
 
 
 # ---------------------------------------------------------------- sampled drafts (general Eq. 1)
-
-def sampled_case(seed, B, K, V, dtype, sigma_q=1.0, T=1.0, Tq=1.0, ld_pad=0):
-    """Target rows from the chain recipe, drafter rows = target rows + noise, drafts really drawn
-    from the drafter's softmax (torch, on the host) with their probabilities."""
-    w = synth.chain_workload("t", B, K, V, dtype, DEV, seed, 0.9, 1.5, 6.0, 10.0, 0.4)
-    g = torch.Generator().manual_seed(seed)
-    z = w.logits.float().cpu().reshape(B, K, V)[:, :K - 1].reshape(-1, V)
-    zq = (z + torch.randn(z.shape, generator=g) * sigma_q).to(dtype)
-    Q = torch.softmax(zq.double() / Tq, dim=1)
-    draft = torch.multinomial(Q, 1, generator=g).reshape(-1)
-    qx = Q[torch.arange(Q.shape[0]), draft].float()
-    qdev = torch.full((B * (K - 1), V + ld_pad), 55.0, dtype=dtype, device=DEV)
-    qdev[:, :V] = zq.to(DEV)
-    u = synth.make_uniforms(B, K, seed)
-    return w, qdev, zq, draft.reshape(B, K - 1).numpy().astype(np.int32), qx.reshape(B, K - 1).numpy(), u
-
-
-def compare_sampled(got, ref, what):
-    B = ref["accept_len"].shape[0]
-    n_close = 0
-    for b in range(B):
-        a = int(ref["accept_len"][b])
-        same_walk = all(np.array_equal(got[k][b], ref[k][b]) for k in ("accept_len", "out_len", "seq_status", "node_how")) \
-            and np.array_equal(got["out_tokens"][b, :a], ref["out_tokens"][b, :a])
-        if not same_walk:
-            assert ref["margin"][b, 0] < DECISION_TOL, (what, b, ref["margin"][b])
-            n_close += 1
-            continue
-        if got["out_tokens"][b, a] != ref["out_tokens"][b, a]:
-            # the draw margin of this oracle is in units of total probability
-            assert ref["margin"][b, 1] < 2e-6, (what, b, got["out_tokens"][b], ref["out_tokens"][b], ref["margin"][b])
-            n_close += 1
-    np.testing.assert_allclose(got["node_prob"], ref["node_prob"], rtol=PROB_RTOL, atol=1e-30, err_msg=what)
-    assert n_close <= max(2, B // 50), (what, n_close)
-
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("flags", [0, mars.STOCH_PLAIN, mars.STOCH_RELAX_ONLY])

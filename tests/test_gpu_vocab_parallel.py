@@ -9,6 +9,8 @@ from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth, vocab_parallel
 from tests.test_gpu_parity import KEYS_TREE, assert_same, special_rows
 
+from stochastic_checks import sharded_stochastic
+
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
@@ -85,26 +87,6 @@ def test_sharded_lm_head_equals_unsharded_bit_for_bit(world):
 
 
 # ---------------------------------------------------------------- stochastic form (T > 0)
-
-def sharded_stochastic(logits, tok, parent, u, theta, T, ranges, flags=0):
-    """The ranks' calls made one after the other on one GPU, stacked as the all-gathers would
-    deliver them; returns every rank's final outputs."""
-    G = len(ranges)
-    recs, zls = [], []
-    for lo, hi in ranges:
-        r, z = mars.stochastic_shard_records(logits[:, lo:hi], tok, parent, lo, T, V_local=hi - lo)
-        recs.append(r)
-        zls.append(z)
-    rec_all, zl_all = torch.stack(recs), torch.stack(zls)
-    outs, parts = [], []
-    for g, (lo, hi) in enumerate(ranges):
-        o, part = mars.stochastic_shard_verify(logits[:, lo:hi], rec_all, zl_all, g, lo, tok, parent, u, theta, T,
-                                               flags, V_local=hi - lo, debug=True)
-        outs.append(o)
-        parts.append(part)
-    token_all = torch.stack(parts)
-    return [mars.to_host(mars.stochastic_shard_finish(token_all, o)) for o in outs], token_all.cpu().numpy()
-
 
 @pytest.mark.parametrize("world", [1, 2, 3, 8])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
