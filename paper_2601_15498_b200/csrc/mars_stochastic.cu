@@ -287,6 +287,10 @@ struct TailShared {
     double target_abs;    // ... and the mass that lies before it inside that shard
 };
 
+// static + dynamic shared memory of the tail stay within the 48 KB that need no opt-in, up to the node cap
+static_assert(sizeof(TailShared) + MARS_MAX_NODES * (9 * 4 + 3) + 64 + 256 <= 48 * 1024,
+              "tail kernel: shared memory above 48 KB at MARS_MAX_NODES");
+
 // ---- what a lane's elements of a tile weigh in the draw ----
 // One row: 2^(z*c - ref), removed tokens at zero (the residual of point-mass drafts).
 template <int DT>
@@ -1327,6 +1331,7 @@ mars_status_t mars_stochastic_shard_verify(const void *logits_local, int64_t ld,
     if ((flags & MARS_STOCH_PLAIN) && (flags & MARS_STOCH_RELAX_ONLY)) return MARS_ERR_INVALID_ARG;
     rule_threshold(&theta, &flags);
     if (!stoch_sizes_supported(B, N, V_local, (int)dt)) return MARS_ERR_UNSUPPORTED;
+    if ((uintptr_t)logits_local % (dt == MARS_BF16 ? 2 : 4)) return MARS_ERR_INVALID_ARG;
     const double cd = 1.4426950408889634074 / (double)temperature;
     if (!(cd < 3.0e38)) return MARS_ERR_INVALID_ARG;
     StochTailParams tp = {};
