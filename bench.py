@@ -501,6 +501,22 @@ def main():
     value = total_units / (total_ms * 1e-3)
     ms_per_step = total_ms / args.steps
 
+    # ---- spread of single steps: an event pair around every repetition (median, p10, p90) ----
+    reps = int(min(100, max(20, 200.0 / max(ms_per_step, 1e-3))))
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for i, (a, b) in enumerate(pairs):
+        a.record()
+        if graph is not None:
+            graph.replay()
+        else:
+            step(i)
+        b.record()
+    torch.cuda.synchronize()
+    per = sorted(a.elapsed_time(b) * 1e3 / (copies if graph is not None else 1) for a, b in pairs)
+    step_us = {"median": per[len(per) // 2], "p10": per[len(per) // 10], "p90": per[(9 * len(per)) // 10],
+               "reps": reps, "note": ("per step of one graph replay" if graph is not None else
+                                      "one event pair per step, launch gaps included")}
+
     # ---- end to end: host buffers in, results out, copies inside the timed region ----
     e2e = None
     h_logits = None
@@ -579,7 +595,7 @@ def main():
                    "workspace": ("uninitialised (records only)" if T else
                                  "zeroed once; MARS_COUNTERS_ZERO (counters reset by the kernel itself)"),
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
-        "us_per_step": 1e3 * ms_per_step,
+        "us_per_step": 1e3 * ms_per_step, "step_us": step_us,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,
         "clocks": clocks.summary(),
         "e2e": e2e,
