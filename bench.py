@@ -517,6 +517,20 @@ def main():
                "reps": reps, "note": ("per step of one graph replay" if graph is not None else
                                       "one event pair per step, launch gaps included")}
 
+    # ---- this GPU's read-only ceiling on the same bytes: the library's streaming probe ----
+    read_gbs = None
+    if w.logits.is_contiguous() and w.logits_bytes >= 3 * L2_BYTES:
+        row_bytes = w.V * w.logits.element_size()
+        for _ in range(3):
+            mars.stream_read_probe(w.logits, row_bytes)
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(20):
+            mars.stream_read_probe(w.logits, row_bytes)
+        r1.record()
+        torch.cuda.synchronize()
+        read_gbs = w.logits_bytes * 20 / (r0.elapsed_time(r1) * 1e-3) / 1e9
+
     # ---- end to end: host buffers in, results out, copies inside the timed region ----
     e2e = None
     h_logits = None
@@ -597,6 +611,8 @@ def main():
                    "parallelism": f"dp{world} (independent sequences, no collective)"},
         "us_per_step": 1e3 * ms_per_step, "step_us": step_us,
         "hbm_gbs": achieved, "frac_of_8TBps_nominal": achieved / HBM_NOMINAL_GBS,
+        "read_only_ceiling_gbs": read_gbs,
+        "frac_of_read_only_ceiling": (achieved / read_gbs) if read_gbs else None,
         "clocks": clocks.summary(),
         "e2e": e2e,
         "gpu_launches": args.steps * (2 if T else 1),

@@ -233,6 +233,17 @@ mars_status_t mars_top2_histograms(const float *top2_val, int64_t rows, float z1
 mars_status_t mars_selftest_bounded_wait(int64_t budget_cycles, void *scratch32, void *cuda_stream);
 
 /*
+ * Read-only streaming probe (the paper has no counterpart; a measurement aid).  Reads `bytes`
+ * bytes of device memory once, in chunks of `chunk_bytes` per thread block, with the 16-byte
+ * streaming loads and the launch shape of the verification kernel, and keeps only the maximum
+ * of the 32-bit words read (atomicMax into *out_max, which the caller zeroes).  Its rate is the
+ * ceiling for a kernel that must read every logit; bench.py reports it beside the copy bandwidth.
+ *   buffer 16-byte aligned; bytes, chunk_bytes >= 16 (chunk_bytes = one logits row in bench.py).
+ */
+mars_status_t mars_selftest_stream_read(const void *buffer, size_t bytes, size_t chunk_bytes,
+                                        uint32_t *out_max, void *cuda_stream);
+
+/*
  * Vocabulary-parallel verification, step 1 of 2: top-2 of one vocabulary shard.
  * When the logits are sharded over the vocabulary (a tensor-parallel LM head), each rank
  * holds columns [id_offset, id_offset + V_local) of every row.  This call reduces the local

@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
             L.mars_stochastic_shard_verify.restype = i32
             L.mars_stochastic_shard_finish.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
             L.mars_stochastic_shard_finish.restype = i32
+            L.mars_selftest_stream_read.argtypes = [vp, sz, sz, vp, vp]
+            L.mars_selftest_stream_read.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
             _lib = L
@@ -477,6 +479,19 @@ def stochastic_shard_finish(token_all: torch.Tensor, out: dict) -> dict:
         code = lib().mars_stochastic_shard_finish(token_all.data_ptr(), G, B, Dcap, out["accept_len"].data_ptr(),
                                                   out["out_tokens"].data_ptr(), out["seq_status"].data_ptr(), _stream())
     _check(code, "mars_stochastic_shard_finish")
+    return out
+
+
+def stream_read_probe(buffer: torch.Tensor, chunk_bytes: int) -> torch.Tensor:
+    """mars_selftest_stream_read on the current stream over the whole (contiguous) tensor; returns
+    the one-word result tensor (the call is asynchronous)."""
+    if not (buffer.is_cuda and buffer.is_contiguous()):
+        raise MarsError("buffer must be a contiguous device tensor")
+    out = torch.zeros((1,), dtype=torch.int32, device=buffer.device)
+    with torch.cuda.device(buffer.device):
+        code = lib().mars_selftest_stream_read(buffer.data_ptr(), buffer.numel() * buffer.element_size(),
+                                               int(chunk_bytes), out.data_ptr(), _stream())
+    _check(code, "mars_selftest_stream_read")
     return out
 
 

@@ -35,3 +35,17 @@ def test_histogram_argument_checks():
     hist, outl = mars.top2_histograms(v[:0].contiguous(), 0.0, 1.0, 8)                  # no rows
     torch.cuda.synchronize()
     assert int(hist.sum()) == 0 and int(outl.sum()) == 0
+
+
+def test_stream_read_probe_reads_every_word():
+    """The read-only probe returns the maximum of the 32-bit words of the buffer, whatever the
+    chunking -- which it can only do if every word was read."""
+    g = torch.Generator().manual_seed(3)
+    buf = torch.randint(0, 2 ** 30, (1 << 20,), generator=g, dtype=torch.int32)
+    buf[777_777] = 2 ** 31 - 5
+    d = buf.to("cuda:0")
+    for chunk in (16, 4096, 303872, 1 << 22):
+        out = mars.stream_read_probe(d, chunk)
+        torch.cuda.synchronize()
+        assert int(out.item()) == 2 ** 31 - 5, chunk
+    assert int(mars.stream_read_probe(d[:777_000], 303872).item()) == int(buf[:777_000].max())
