@@ -287,9 +287,15 @@ void mars_oracle_verify_tree(const void *logits, int dtype, int64_t ld, const in
 }
 
 /*
- * Whole path, chain form: a literal walk of Algorithm 1 over K rows and K-1 drafts.
- * Row i is the target's distribution for draft i; if every draft is accepted the last
- * row supplies the bonus token (Table 1 caption), so out_len <= K.
+ * Whole path, chain form (the rule of Sec. 3.4 applied along a chain, as Algorithm 1 / Sec. 3.4
+ * define it): K rows, K-1 drafts; row i is the target's distribution that judges draft i.
+ * Stated as a definition rather than as a loop with early exit:
+ *   keep[i]    = draft i, taken alone, passes the three-way rule on row i
+ *   accept_len = a = the number of leading positions with keep[i] set (the first failure ends
+ *                the accepted prefix, whatever comes after it)
+ *   output     = draft[0..a) followed by the top-1 of row a -- the target's own choice at the
+ *                first failed position, or, when a = K-1, the extra token that the last row
+ *                supplies (Table 1 caption), so out_len = a + 1 <= K.
  *   draft [B,K-1]; out_tokens [B,K] padded with -1.
  */
 void mars_oracle_verify_chain(const void *logits, int dtype, int64_t ld, const int32_t *draft,
@@ -302,36 +308,24 @@ void mars_oracle_verify_chain(const void *logits, int dtype, int64_t ld, const i
     if (dbg_id) memcpy(dbg_id, id_buf, (size_t)R * 2 * sizeof(int32_t));
     if (dbg_val) memcpy(dbg_val, val_buf, (size_t)R * 2 * (dtype == ORACLE_FP64 ? 8 : 4));
     for (int b = 0; b < B; ++b) {
+        const int32_t *d = draft + (size_t)b * (K - 1);
+        const int32_t *ids = id_buf + 2 * (size_t)b * K;
+        uint8_t keep[K];                       /* K >= 1 */
+        for (int i = 0; i < K - 1; ++i) {
+            int64_t r = (int64_t)b * K + i;
+            int relax = dtype == ORACLE_FP64
+                ? mars_oracle_relax_f64(((const double *)val_buf)[2 * r], ((const double *)val_buf)[2 * r + 1], theta, flags)
+                : mars_oracle_relax_f32(((const float *)val_buf)[2 * r], ((const float *)val_buf)[2 * r + 1], (float)theta, flags);
+            keep[i] = (uint8_t)(rule(d[i], ids + 2 * i, relax) != 0);
+        }
+        int a = 0;
+        while (a < K - 1 && keep[a]) ++a;
         int32_t *out = out_tokens + (size_t)b * K;
         fill(out, K, -1);
-        int n = 0, stopped = 0;
-        for (int i = 0; i < K - 1 && !stopped; ++i) {
-            int64_t r = (int64_t)b * K + i;
-            int relax;
-            if (dtype == ORACLE_FP64) {
-                const double *v = (const double *)val_buf + 2 * r;
-                relax = mars_oracle_relax_f64(v[0], v[1], theta, flags);
-            } else {
-                const float *v = (const float *)val_buf + 2 * r;
-                relax = mars_oracle_relax_f32(v[0], v[1], (float)theta, flags);
-            }
-            int32_t t = draft[(size_t)b * (K - 1) + i];
-            if (t >= 0 && t == id_buf[2 * r]) {
-                out[n++] = t;                       /* exact match: keep draft */
-            } else if (t >= 0 && t == id_buf[2 * r + 1] && relax) {
-                out[n++] = t;                       /* adaptive relaxation: keep draft */
-            } else {
-                out[n++] = id_buf[2 * r];           /* correction: target top-1, stop */
-                stopped = 1;
-            }
-        }
-        if (stopped) {
-            accept_len[b] = n - 1;
-        } else {
-            accept_len[b] = n;
-            out[n++] = id_buf[2 * ((int64_t)b * K + (K - 1))]; /* bonus token */
-        }
-        out_len[b] = n;
+        memcpy(out, d, (size_t)a * sizeof(int32_t));
+        out[a] = ids[2 * a];
+        accept_len[b] = a;
+        out_len[b] = a + 1;
     }
 }
 

@@ -124,28 +124,45 @@ def test_fig2_worked_example():
             assert out["accept_len"][0] == 0 and out["out_tokens"][0].tolist() == [4, -1]
 
 
+PRECISIONS = [pytest.param(False, id="fp32"), pytest.param(True, id="fp64")]
+
+
+def _ty(fp64):
+    """Decision type of the stored-logits path (fp32) or of the projected-logits path (fp64)."""
+    return np.float64 if fp64 else F32
+
+
+@pytest.mark.parametrize("fp64", PRECISIONS)
 @pytest.mark.parametrize("theta", [0.9, 0.84, 0.95, 0.5])
 @pytest.mark.parametrize("k", [-3, 0, 4])
-def test_ratio_one_ulp_around_theta(theta, k):
-    """z1 a power of two makes z2/z1 exact, so r > theta iff z2 > theta*z1 (strict)."""
-    th = F32(theta)
-    z1 = F32(2.0 ** k)
-    on = F32(th * z1)                    # exact: scaling by a power of two
-    up = np.nextafter(on, F32(np.inf), dtype=F32)
-    dn = np.nextafter(on, F32(-np.inf), dtype=F32)
-    assert orc.relax(z1, up, th)
-    assert not orc.relax(z1, on, th)     # r == theta rejects
-    assert not orc.relax(z1, dn, th)
+def test_ratio_one_ulp_around_theta(theta, k, fp64):
+    """z1 a power of two makes z2/z1 exact, so r > theta iff z2 > theta*z1 (strict); the planted
+    values sit one ulp of the decision type around theta*z1."""
+    T = _ty(fp64)
+    th = T(F32(theta))                   # theta is handed to the library as an fp32 value
+    z1 = T(2.0 ** k)
+    on = T(th * z1)                      # exact: scaling by a power of two
+    up = np.nextafter(on, T(np.inf), dtype=T)
+    dn = np.nextafter(on, T(-np.inf), dtype=T)
+    assert up > on > dn
+    assert orc.relax(z1, up, th, fp64=fp64)
+    assert not orc.relax(z1, on, th, fp64=fp64)     # r == theta rejects
+    assert not orc.relax(z1, dn, th, fp64=fp64)
+    # operands the other way round would accept all three (z1/z2 > 1 > theta)
     # through the whole path as well
     for z2, want in ((up, 1), (on, 0), (dn, 0)):
-        z = np.full((2, 8), -1.0, F32)
+        z = np.full((2, 8), -1.0, T)
         z[:, 2] = z1
         z[:, 5] = z2
         out = orc.verify_chain(z, np.array([[5]], np.int32), float(th))
         assert out["accept_len"][0] == want
+        tok = np.array([[-1, 5]], np.int32)
+        par = np.array([[-1, 0]], np.int32)
+        assert orc.verify_tree(z, tok, par, float(th))["accept_len"][0] == want
 
 
-def test_ratio_equals_adaptive_margin_form():
+@pytest.mark.parametrize("fp64", PRECISIONS)
+def test_ratio_equals_adaptive_margin_form(fp64):
     """Eq. 6: r > theta  <=>  Delta < (1 - theta) z1, checked in fp64 away from equality."""
     rng = np.random.default_rng(5)
     n = 0
@@ -158,25 +175,31 @@ def test_ratio_equals_adaptive_margin_form():
         if abs(lhs - rhs) < 1e-4 * max(1.0, abs(float(z1))):
             continue
         n += 1
-        assert orc.relax(z1, z2, theta) == (lhs < rhs), (z1, z2, theta)
+        assert orc.relax(z1, z2, theta, fp64=fp64) == (lhs < rhs), (z1, z2, theta)
     assert n > 15000
 
 
-def test_ratio_bounded_on_positive_rows_and_sign_guard():
+@pytest.mark.parametrize("fp64", PRECISIONS)
+def test_ratio_bounded_on_positive_rows_and_sign_guard(fp64):
     rng = np.random.default_rng(6)
-    z = np.abs(rng.normal(0, 3, size=(64, 100))).astype(np.float32) + 0.01
+    z = (np.abs(rng.normal(0, 3, size=(64, 100))) + 0.01).astype(_ty(fp64))
     val, _ = orc.top2(z)
+    assert val.dtype == _ty(fp64)
     r = val[:, 1] / val[:, 0]
     assert ((r > 0) & (r <= 1)).all()           # Sec. 3.3: r in (0, 1] on positive logits
+
+    def rx(z1, z2, theta, flags=0):
+        return orc.relax(z1, z2, theta, flags, fp64=fp64)
     # non-positive top-1: the guarded rule never relaxes; the literal ratio would
-    assert not orc.relax(-2.0, -3.0, 0.9)
-    assert orc.relax(-2.0, -3.0, 0.9, orc.SIGN_LITERAL)       # (-3)/(-2) = 1.5 > 0.9
-    assert not orc.relax(0.0, -1.0, 0.9) and not orc.relax(0.0, -1.0, 0.9, orc.SIGN_LITERAL)
-    assert not orc.relax(0.0, 0.0, 0.9, orc.SIGN_LITERAL)     # 0/0 = NaN compares false
-    assert not orc.relax(np.inf, np.inf, 0.9)                 # inf/inf = NaN
-    assert not orc.relax(5.0, -1.0, 0.0)                      # r < 0
-    assert orc.relax(4.0, 4.0, 0.999)                         # exact tie: r = 1
-    assert not orc.relax(4.0, 4.0, 1.0)                       # theta >= 1 is strict greedy
+    assert not rx(-2.0, -3.0, 0.9)
+    assert rx(-2.0, -3.0, 0.9, orc.SIGN_LITERAL)       # (-3)/(-2) = 1.5 > 0.9
+    assert not rx(0.0, -1.0, 0.9) and not rx(0.0, -1.0, 0.9, orc.SIGN_LITERAL)
+    assert not rx(0.0, 0.0, 0.9, orc.SIGN_LITERAL)     # 0/0 = NaN compares false
+    assert not rx(np.inf, np.inf, 0.9)                 # inf/inf = NaN
+    assert not rx(5.0, -1.0, 0.0)                      # r < 0
+    assert rx(4.0, 4.0, 0.999)                         # exact tie: r = 1
+    assert not rx(4.0, 4.0, 1.0)                       # theta >= 1 is strict greedy
+    assert not rx(4.0, 3.999, 1.0) and not rx(4.0, 4.0, 1.5)
 
 
 def test_scale_invariance_power_of_two():
@@ -475,22 +498,70 @@ def test_lmhead_small_against_hand_fp64():
     assert (out["top2_id"] == order[:, :2]).all()
 
 
+@pytest.mark.parametrize("sign_literal", [False, True])
+def test_lmhead_planted_ratio_decides_in_fp64(sign_literal):
+    """One-hot W_o turns the projection into a gather, so every logit is known exactly and the
+    ratio of the planted pair can be put just above / exactly at / just below theta = 3/4 with
+    z1 a power of two (the division is exact).  The hidden values are bf16-representable, and one
+    bf16 step at 12 is far more than one fp64 ulp, so this pins direction and strictness of the
+    fp64 rule through the projection; the guard is pinned by the negative-logit rows."""
+    d, V = 8, 12
+    theta = 0.75
+    w = np.zeros((V, d), np.float32)
+    w[np.arange(V), np.arange(V) % d] = 1.0          # z[r, j] = h[r, j % d]
+    w[d:, :] = 0.0                                   # columns 8..11 stay at logit 0
+    cases = [                                        # (h0 = z1 at id 0, h1 = z2 at id 1, relaxes?)
+        (16.0, 12.0625, True),                       # r = 0.75390625 > theta
+        (16.0, 12.0, False),                         # r == theta rejects
+        (16.0, 11.9375, False),
+    ]
+    for h0, h1, want in cases:
+        h = np.full((2, d), -4.0, np.float32)
+        h[:, 0], h[:, 1] = h0, h1
+        hb, wb = bf16_bits(h), bf16_bits(w)
+        z = orc.lmhead_logits(hb, wb)
+        assert z[0, 0] == h0 and z[0, 1] == h1 and (z[0, 2:8] == -4.0).all() and (z[0, 8:] == 0).all()
+        tok = np.array([[-1, 1]], np.int32)
+        par = np.array([[-1, 0]], np.int32)
+        flags = orc.SIGN_LITERAL if sign_literal else 0
+        out = orc.lmhead_verify_tree(hb, wb, None, tok, par, theta, flags)
+        assert out["top2_id"][0].tolist() == [0, 1]
+        assert out["accept_len"][0] == int(want), (h0, h1)
+        assert out["out_tokens"][0].tolist() == ([1, 0] if want else [0, -1])
+    # all logits negative: top-1 = -8 at id 0, runner-up -12 at id 1, ratio 1.5 > theta.  The
+    # guarded rule must not relax, the literal one does.
+    w2 = np.eye(d, dtype=np.float32)                 # V = d: z[r, j] = h[r, j], no zero logits
+    h = np.full((2, d), -30.0, np.float32)
+    h[:, 0], h[:, 1] = -8.0, -12.0
+    hb, wb = bf16_bits(h), bf16_bits(w2)
+    out = orc.lmhead_verify_tree(hb, wb, None, np.array([[-1, 1]], np.int32), np.array([[-1, 0]], np.int32),
+                                 theta, orc.SIGN_LITERAL if sign_literal else 0)
+    assert out["top2_id"][0].tolist() == [0, 1]
+    assert out["accept_len"][0] == int(sign_literal)
+
+
 # --------------------------------------------------------------------------- rule variants
 
-def test_margin_variant_one_ulp_and_through_chain():
-    """Fixed-margin indicator: relax iff Delta = z1 - z2 < c (strict), one fp32 subtraction."""
-    c = F32(0.5)
-    z1 = F32(8.0)
-    on = F32(7.5)                                           # Delta == c exactly
-    closer = np.nextafter(on, F32(np.inf), dtype=F32)       # Delta just below c
-    farther = np.nextafter(on, F32(-np.inf), dtype=F32)
-    assert orc.relax(z1, closer, c, orc.RULE_MARGIN)
-    assert not orc.relax(z1, on, c, orc.RULE_MARGIN)
-    assert not orc.relax(z1, farther, c, orc.RULE_MARGIN)
-    assert orc.relax(-3.0, -3.25, c, orc.RULE_MARGIN)       # no sign guard for this indicator
-    assert not orc.relax(5.0, -np.inf, c, orc.RULE_MARGIN)
+@pytest.mark.parametrize("fp64", PRECISIONS)
+def test_margin_variant_one_ulp_and_through_chain(fp64):
+    """Fixed-margin indicator: relax iff Delta = z1 - z2 < c (strict), one subtraction in the
+    decision type."""
+    T = _ty(fp64)
+    c = T(0.5)
+    z1 = T(8.0)
+    on = T(7.5)                                             # Delta == c exactly
+    closer = np.nextafter(on, T(np.inf), dtype=T)           # Delta just below c
+    farther = np.nextafter(on, T(-np.inf), dtype=T)
+
+    def rx(a, b, th, flags):
+        return orc.relax(a, b, th, flags, fp64=fp64)
+    assert rx(z1, closer, c, orc.RULE_MARGIN)
+    assert not rx(z1, on, c, orc.RULE_MARGIN)
+    assert not rx(z1, farther, c, orc.RULE_MARGIN)
+    assert rx(-3.0, -3.25, c, orc.RULE_MARGIN)              # no sign guard for this indicator
+    assert not rx(5.0, -np.inf, c, orc.RULE_MARGIN)
     for z2, want in ((closer, 1), (on, 0)):
-        z = np.full((2, 8), -1.0, F32)
+        z = np.full((2, 8), -1.0, T)
         z[:, 2] = z1
         z[:, 5] = z2
         out = orc.verify_chain(z, np.array([[5]], np.int32), float(c), orc.RULE_MARGIN)
@@ -499,10 +570,14 @@ def test_margin_variant_one_ulp_and_through_chain():
         assert out["accept_len"][0] == 1                     # exact match is unaffected
 
 
-def test_prob_ratio_variant_against_softmax_definition():
+@pytest.mark.parametrize("fp64", PRECISIONS)
+def test_prob_ratio_variant_against_softmax_definition(fp64):
     """p2/p1 > theta with p = softmax(z) (Eq. 3) evaluated in fp64 on whole rows, away from
     the boundary; and the limits theta <= 0 (always) / theta >= 1 (never for distinct logits)."""
     rng = np.random.default_rng(21)
+
+    def rx(a, b, th, flags):
+        return orc.relax(a, b, th, flags, fp64=fp64)
     n = 0
     for _ in range(3000):
         z = rng.normal(0, 3, 50).astype(np.float32)
@@ -513,16 +588,16 @@ def test_prob_ratio_variant_against_softmax_definition():
         if abs(ratio - float(theta)) < 1e-4:
             continue
         n += 1
-        assert orc.relax(zs[0], zs[1], theta, orc.RULE_PROB_RATIO) == (ratio > float(theta))
+        assert rx(zs[0], zs[1], theta, orc.RULE_PROB_RATIO) == (ratio > float(theta))
     assert n > 2500
-    assert orc.relax(3.0, -40.0, 0.0, orc.RULE_PROB_RATIO) and orc.relax(3.0, -40.0, -1.0, orc.RULE_PROB_RATIO)
-    assert not orc.relax(3.0, 2.999, 1.0, orc.RULE_PROB_RATIO)
-    assert not orc.relax(3.0, 3.0, 1.0, orc.RULE_PROB_RATIO)      # p2/p1 == 1 is not > 1
+    assert rx(3.0, -40.0, 0.0, orc.RULE_PROB_RATIO) and rx(3.0, -40.0, -1.0, orc.RULE_PROB_RATIO)
+    assert not rx(3.0, 2.999, 1.0, orc.RULE_PROB_RATIO)
+    assert not rx(3.0, 3.0, 1.0, orc.RULE_PROB_RATIO)      # p2/p1 == 1 is not > 1
     # equal to the margin variant at c = -ln(theta)
     for theta in (0.3, 0.6, 0.9):
         c = F32(-np.log(np.float64(F32(theta))))
         for z2 in np.linspace(1.0, 3.0, 41):
-            assert orc.relax(3.0, z2, theta, orc.RULE_PROB_RATIO) == orc.relax(3.0, z2, c, orc.RULE_MARGIN)
+            assert rx(3.0, z2, theta, orc.RULE_PROB_RATIO) == rx(3.0, z2, c, orc.RULE_MARGIN)
 
 
 def test_variants_only_change_relaxed_accepts():

@@ -389,3 +389,44 @@ def test_sampled_modes_are_nested():
     r = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, orc.STOCH_RELAX_ONLY)["accept_len"]
     d = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, 1.0, 1.0, 0)["accept_len"]
     assert (a <= r).all() and (r <= d).all() and a.sum() < d.sum()
+
+
+def test_a_negative_draft_ends_the_chain_and_the_token_comes_from_the_target_row():
+    """Reading: a negative draft id is padding -- there is no draft at that position, so nothing
+    was rejected and no residual applies.  The accepted prefix ends there and the emitted token
+    is a plain draw from the target's distribution of that row (numpy CDF inversion of
+    softmax(row / T)), exactly as for the bonus token of a fully accepted chain.  The drafter's
+    row at that position must not enter: the residual max(0, P - Q) would pick another token."""
+    V, K, B, T, Tq = 23, 5, 400, 1.1, 0.7
+    logits, qlogits, draft, qx, u = _sampled_case(16, B, K, V, 1.2, 1.5, T, Tq, same_rows=False)
+    u[:, 1:] = np.float32(1e-7)             # every real draft passes Eq. 1 (P(x) > 1e-7 Q(x))
+    rng = np.random.default_rng(160)
+    cut = rng.integers(0, K - 1, B)         # position of the first padding draft
+    for b in range(B):
+        draft[b, cut[b]] = -1
+    full = orc.verify_chain_sampled(logits, qlogits, draft, qx, u, 0.9, T, Tq, orc.STOCH_PLAIN)
+    assert (full["seq_status"] == 0).all()
+    assert np.array_equal(full["accept_len"], cut.astype(np.int32))
+    assert np.array_equal(full["out_len"], cut.astype(np.int32) + 1)
+    P = softmax(logits.astype(np.float64) / T, axis=1)
+    Q = softmax(qlogits.astype(np.float64) / Tq, axis=1)
+    differs = 0
+    for b in range(B):
+        i = int(cut[b])
+        assert np.array_equal(full["out_tokens"][b, :i], draft[b, :i])
+        assert (full["out_tokens"][b, i + 1:] == -1).all()
+        assert full["node_how"][b, i + 1] == 0          # never judged
+        c = np.cumsum(P[b * K + i])
+        want = int(np.searchsorted(c, float(u[b, 0]) * c[-1], side="right"))
+        assert full["out_tokens"][b, i] == want
+        w = np.maximum(P[b * K + i] - Q[b * (K - 1) + i], 0.0)
+        cr = np.cumsum(w)
+        differs += int(np.searchsorted(cr, float(u[b, 0]) * cr[-1], side="right")) != want
+    assert differs > B // 4                 # the residual would have given another answer
+    # drafts behind the padding are never looked at
+    other = draft.copy()
+    for b in range(B):
+        other[b, cut[b] + 1:] = (other[b, cut[b] + 1:] + 1) % V
+    again = orc.verify_chain_sampled(logits, qlogits, other, qx, u, 0.9, T, Tq, orc.STOCH_PLAIN)
+    for k in ("accept_len", "out_tokens", "out_len"):
+        assert np.array_equal(full[k], again[k]), k
