@@ -176,8 +176,8 @@ size_t mars_lmhead_workspace_bytes(int B, int N, int V, int d);
  *   Remaining arguments, outputs and per-sequence statuses are those of mars_verify_tree.
  *   Accumulation order differs from a sequential sum, so near-ties may resolve differently
  *   from an fp64 evaluation; decisions are still taken in fp32 on the accumulated values.
- *   The first call in a process sets function attributes and queries cluster occupancy
- *   (host-side, once); make that first call outside any stream capture.
+ *   The first call on each device sets function attributes and queries cluster occupancy for
+ *   that device (host-side, once per device); make that first call outside any stream capture.
  *   If a bounded device-side wait gives up (which indicates a fault in the pipeline, not a
  *   property of the data), every sequence gets MARS_SEQ_TIMEOUT, accept_len 0, out_len 0 and
  *   out_tokens / path_nodes filled with -1.
@@ -459,7 +459,9 @@ mars_status_t mars_stochastic_shard_finish(const int32_t *token_all, int shards,
  *     capture.  A failure of the look-up is reported as MARS_ERR_CUDA.
  *   - All calls on one device share the one array.  It keeps whatever the previous call left
  *     in it; the function clears the part that must start at zero (the per-sequence arrival
- *     counters) on the stream before its kernel.  Two calls whose GPU work may overlap --
+ *     counters) on the stream before its kernel, on every call: MARS_COUNTERS_ZERO in `flags`
+ *     is accepted and ignored here, since no caller can vouch for the contents of an array
+ *     that it does not own.  Two calls whose GPU work may overlap --
  *     different streams without an ordering between them, or several host threads -- race on
  *     the array and give undefined results: serialise them, or use mars_verify_tree with
  *     separate workspaces.
@@ -474,6 +476,30 @@ mars_status_t mars_verify_tree_static(const void *logits, int64_t ld, mars_dtype
 
 /* Size in bytes of the built-in scratch array used by mars_verify_tree_static (host, pure). */
 size_t mars_static_scratch_bytes(void);
+
+/*
+ * Host: how the current device compares with the one the launch shapes are tuned for.  (The
+ * paper has no counterpart.)  Grid sizes, row splits and work-item chunking assume a B200 with
+ * 148 SMs; they are pure functions of the call's sizes so that workspace sizes never depend on
+ * the device.  On a part with fewer SMs every result stays correct, but waves no longer fill
+ * evenly.  *sm_count receives the device's SM count, *sm_tuned 148 (either may be NULL).
+ * Returns MARS_OK when they agree and the device is compute capability 10.x,
+ * MARS_ERR_UNSUPPORTED when not, MARS_ERR_CUDA if the device cannot be queried.
+ */
+mars_status_t mars_device_check(int *sm_count, int *sm_tuned);
+
+/*
+ * Test hook (the paper has no counterpart; not for deployment): forces a launch shape that the
+ * library would not choose by itself, so that tests reach those paths with small inputs.
+ * Process-wide, takes effect from the next call, also changes the matching *_workspace_bytes
+ * results.  The library never reads the environment: unless this function is called, behaviour
+ * depends on the arguments of each call alone.
+ *   which 0: slices per logits row (mars_verify_*, mars_top2_shard, mars_topk_rows, stochastic calls)
+ *         1: value 1 selects the single-block MMA kernel of mars_lmhead_verify / _top2_shard
+ *         2: blocks per cluster of the stochastic tail kernel (1, 2, 4 or 8)
+ *   value 0 clears the hook.  Returns the previous value, or -1 for an unknown hook / negative value.
+ */
+int mars_test_hook(int which, int value);
 
 /* Static, human-readable name of a status code (host memory, never NULL). */
 const char *mars_status_string(mars_status_t s);

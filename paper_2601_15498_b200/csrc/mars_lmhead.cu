@@ -25,6 +25,7 @@
 // block-wide abort flag and a status word in the workspace; all roles then fall through to
 // the common exit, which drains outstanding copies (bounded), frees TMEM and returns.
 #include "mars_common.cuh"
+#include "mars_hooks.cuh"
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -673,8 +674,7 @@ struct LmShape { int n_mtiles, n_ntiles, n_chunks, n_items, chunk_tiles; };
 // device so that the workspace size is a pure function of the shapes.
 static bool lm_pair_mode()
 {
-    const char *e = getenv("MARS_LMHEAD_1CTA");    // test hook: force the single-block MMA kernel
-    return !(e && e[0] == '1');
+    return hook(kHookLmheadSingleBlock) != 1;      // test hook: force the single-block MMA kernel
 }
 
 static LmShape lm_shape(long long M, int V)
@@ -705,6 +705,50 @@ static bool lm_supported(int B, int N, int V, int d)
     return true;
 }
 
+// Per-device launch state: the opt-in to more than 48 KB of dynamic shared memory is a function
+// attribute of the device that is current when it is set, and so is the number of 2-block
+// clusters that can be resident at once.
+struct LmDeviceState { int ready; int sms; int max_pairs; };
+constexpr int kLmMaxDevices = 64;
+static std::mutex g_lm_mu;
+static LmDeviceState g_lm_state[kLmMaxDevices] = {};
+
+static bool lm_device_state(LmDeviceState *out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kLmMaxDevices) return false;
+    std::lock_guard<std::mutex> lock(g_lm_mu);
+    LmDeviceState &d = g_lm_state[dev];
+    if (!d.ready) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2)
+            return false;
+        if (cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kLmSmemBytes) != cudaSuccess)
+            return false;
+        if (cudaFuncSetAttribute(lmhead_top2_kernel_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kLm2SmemBytes) != cudaSuccess)
+            return false;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(sms / 2 * 2); cfg.blockDim = dim3(kLmThreads);
+        cfg.dynamicSmemBytes = kLm2SmemBytes;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, lmhead_top2_kernel_pair, &cfg) == cudaSuccess && n > 0)
+            d.max_pairs = n;
+        else
+            d.max_pairs = sms / 2;
+        (void)cudaGetLastError();
+        d.sms = sms;
+        d.ready = 1;
+    }
+    *out = d;
+    return true;
+}
+
 // Shapes, tensor maps and launch of the GEMM + top-2 kernel; fills *pout for the kernels that
 // consume the per-chunk records.
 static mars_status_t lm_launch_gemm(const void *hidden, const void *w_vocab, const float *bias, int d,
@@ -724,40 +768,16 @@ static mars_status_t lm_launch_gemm(const void *hidden, const void *w_vocab, con
     if (!make_map(&map_h, hidden, (uint64_t)M, (uint64_t)d, kBM)) return MARS_ERR_CUDA;
     if (!make_map(&map_w, w_vocab, (uint64_t)V, (uint64_t)d, lm_pair_mode() ? kBN / 2 : kBN)) return MARS_ERR_CUDA;
 
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MARS_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MARS_ERR_CUDA;
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(lmhead_top2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kLmSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(lmhead_top2_kernel_pair, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kLm2SmemBytes);
-    });
-    if (attr_err != cudaSuccess) return MARS_ERR_CUDA;
+    // Function attributes and occupancy belong to a device: set them up once for each device
+    // that this process calls from, with that device current.
+    LmDeviceState dstate;
+    if (!lm_device_state(&dstate)) return MARS_ERR_CUDA;
+    const int sms = dstate.sms;
 
     if (cudaMemsetAsync(p.status, 0, 256, st) != cudaSuccess) return MARS_ERR_CUDA;
     if (lm_pair_mode()) {
         // persistent pairs: never launch more clusters than can be resident together
-        static std::once_flag occ_once;
-        static int max_pairs = 0;
-        std::call_once(occ_once, [&] {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(sms / 2 * 2); cfg.blockDim = dim3(kLmThreads);
-            cfg.dynamicSmemBytes = kLm2SmemBytes;
-            cudaLaunchAttribute at[1];
-            at[0].id = cudaLaunchAttributeClusterDimension;
-            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-            cfg.attrs = at; cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, lmhead_top2_kernel_pair, &cfg) == cudaSuccess && n > 0)
-                max_pairs = n;
-            else
-                max_pairs = sms / 2;
-            (void)cudaGetLastError();
-        });
+        const int max_pairs = dstate.max_pairs;
         int pairs = max_pairs < sms / 2 ? max_pairs : sms / 2;
         if (s.n_items < pairs) pairs = s.n_items;
         lmhead_top2_kernel_pair<<<2 * pairs, kLmThreads, kLm2SmemBytes, st>>>(map_h, map_w, p);

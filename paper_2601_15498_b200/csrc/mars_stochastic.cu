@@ -1186,9 +1186,7 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     int G = 1;
     for (int g = kTailCluster; g > 1; g >>= 1)
         if ((long long)B * g <= (sd ? 1 : 2) * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
-    const char *force = getenv("MARS_STOCH_TAIL_CLUSTER");   // test hook: 1, 2, 4 or 8
-    if (force) {
-        const int g = atoi(force);
+    if (const int g = hook(kHookStochTailCluster)) {         // test hook: 1, 2, 4 or 8
         if ((g == 1 || g == 2 || g == 4 || g == 8) && (g == 1 || (ntiles + g - 1) / g <= kMaxTilesPerBlock)) G = g;
     }
     cudaLaunchConfig_t cfg = {};
@@ -1347,9 +1345,7 @@ mars_status_t mars_stochastic_shard_verify(const void *logits_local, int64_t ld,
     int G = 1;
     for (int g = kTailCluster; g > 1; g >>= 1)
         if ((long long)B * g <= 2 * 148 && (ntiles + g - 1) / g <= kMaxTilesPerBlock) { G = g; break; }
-    const char *force = getenv("MARS_STOCH_TAIL_CLUSTER");   // test hook: 1, 2, 4 or 8
-    if (force) {
-        const int g = atoi(force);
+    if (const int g = hook(kHookStochTailCluster)) {         // test hook: 1, 2, 4 or 8
         if ((g == 1 || g == 2 || g == 4 || g == 8) && (g == 1 || (ntiles + g - 1) / g <= kMaxTilesPerBlock)) G = g;
     }
     cudaLaunchConfig_t cfg = {};

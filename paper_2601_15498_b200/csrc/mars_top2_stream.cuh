@@ -6,6 +6,7 @@
 #include <cstdlib>
 
 #include "mars_common.cuh"
+#include "mars_hooks.cuh"
 #include "mars_stream.cuh"
 
 namespace mars {
@@ -106,9 +107,9 @@ inline Split choose_split(long long R, int V, int dt)
 {
     const int es = dt == MARS_BF16 ? 2 : 4;
     long long S = 1;
-    const char *force = getenv("MARS_FORCE_SPLIT");  // test hook: force slices per row
+    const int force = hook(kHookForceSplit);         // test hook: force slices per row
     int min_elems = kMinSliceBytes / es;
-    if (force && atoi(force) >= 1) { S = atoi(force); min_elems = 64; }
+    if (force >= 1) { S = force; min_elems = 64; }
     else if (R < kTargetBlocks) S = kTargetBlocks / R;   // never more blocks than fit at once
     long long smax = V / min_elems;
     if (smax < 1) smax = 1;

@@ -13,6 +13,7 @@
 // Total order as everywhere in the library: larger value first, lower token id first among
 // equal values, NaN counts as -inf, -0 is reported as +0.
 #include "mars_common.cuh"
+#include "mars_hooks.cuh"
 #include "mars_stream.cuh"
 
 #include <cstdlib>
@@ -422,9 +423,9 @@ static TkSplit topk_split(long long R, int V, int dt)
 {
     const int es = dt == MARS_BF16 ? 2 : 4;
     long long S = 1;
-    const char *force = getenv("MARS_FORCE_SPLIT");   // test hook shared with the top-2 kernel
+    const int force = hook(kHookForceSplit);          // test hook shared with the top-2 kernel
     int min_elems = kTkMinSliceBytes / es;
-    if (force && atoi(force) >= 1) { S = atoi(force); min_elems = 64; }
+    if (force >= 1) { S = force; min_elems = 64; }
     else if (R < kTkTargetBlocks) S = kTkTargetBlocks / R;
     long long smax = V / min_elems;
     if (smax < 1) smax = 1;

@@ -339,7 +339,11 @@ mars_status_t mars_verify_tree_static(const void *logits, int64_t ld, mars_dtype
     if (st != MARS_OK) return st;
     // The arrival counters at the front of the scratch must start at zero; run() clears them
     // on the stream before the kernel.  Everything else in the array is overwritten before
-    // it is read, so the previous call's leftovers are harmless.
+    // it is read, so the previous call's leftovers are harmless.  MARS_COUNTERS_ZERO is a
+    // promise about a workspace that the caller owns; nobody can make it about this array
+    // (its counter region grows with B and may hold an earlier call's records), so the bit is
+    // dropped and the counters are always cleared.
+    flags &= ~MARS_COUNTERS_ZERO;
     return mars::run(logits, ld, dt, tok, parent, 0, B, N, V, theta, flags, accept_len, out_tokens,
                      path_nodes, out_len, Dcap, seq_status, dbg, scratch, MARS_STATIC_SCRATCH_BYTES,
                      cuda_stream);

@@ -100,8 +100,30 @@ def lib() -> ctypes.CDLL:
             L.mars_selftest_stream_read.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
+            L.mars_test_hook.argtypes = [i32, i32]
+            L.mars_test_hook.restype = i32
+            L.mars_device_check.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32)]
+            L.mars_device_check.restype = i32
             _lib = L
     return _lib
+
+
+HOOK_FORCE_SPLIT, HOOK_LMHEAD_SINGLE_BLOCK, HOOK_STOCH_TAIL_CLUSTER = 0, 1, 2
+
+
+def test_hook(which: int, value: int) -> int:
+    """Set a test hook of the library (0 clears it); returns the previous value."""
+    prev = lib().mars_test_hook(int(which), int(value))
+    if prev < 0:
+        raise MarsError(f"unknown test hook {which} or negative value {value}")
+    return prev
+
+
+def device_check() -> dict:
+    """SM count of the current device against the count the launch shapes are tuned for."""
+    sm, tuned = ctypes.c_int(0), ctypes.c_int(0)
+    code = lib().mars_device_check(ctypes.byref(sm), ctypes.byref(tuned))
+    return {"status": int(code), "sm_count": sm.value, "sm_tuned": tuned.value}
 
 
 def _check(code: int, what: str) -> None:

@@ -18,13 +18,23 @@ import torch.distributed as dist
 
 def shard_ranges(V: int, world: int) -> list[tuple[int, int]]:
     """Column range [lo, hi) of each rank: contiguous, sizes differ by at most one multiple of
-    8 columns so that every shard but the last starts 16-byte aligned in bf16."""
+    8 columns so that every shard but the last starts 16-byte aligned in bf16.
+
+    A pure function of (V, world), so every rank reaches the same verdict: if any shard would
+    hold fewer than the two columns the library needs, all ranks raise here, before any of them
+    enters a collective that the others would then wait in."""
+    if world < 1 or V < 2:
+        raise ValueError("need world >= 1 and V >= 2")
     per = -(-V // world)
     per = -(-per // 8) * 8
     out = []
     for r in range(world):
         lo = min(V, r * per)
         out.append((lo, min(V, lo + per)))
+    short = [r for r, (lo, hi) in enumerate(out) if hi - lo < 2]
+    if short:
+        raise ValueError(f"V = {V} over {world} ranks in multiples of 8 columns leaves rank(s) {short} with "
+                         "fewer than 2 columns; use fewer ranks for this vocabulary")
     return out
 
 

@@ -36,3 +36,14 @@ def _built_library():
     except Exception as e:  # pragma: no cover
         print(f"libmars build skipped: {e}")
     yield
+
+
+@pytest.fixture(autouse=True)
+def _hooks_cleared():
+    """No test inherits a forced launch shape from the one before it."""
+    yield
+    try:
+        import hookctl
+        hookctl.clear_all()
+    except Exception:  # pragma: no cover  (library not built: the tests that need it report that)
+        pass

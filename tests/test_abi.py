@@ -10,6 +10,8 @@ import pytest
 
 from paper_2601_15498_b200 import build, mars
 
+import hookctl as hooks
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
@@ -44,7 +46,7 @@ def test_status_strings(lib):
 
 
 def test_workspace_bytes_host_only(lib, monkeypatch):
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
     wb = lib.mars_workspace_bytes
     assert wb(0, 1, 100, 0) == 0 and wb(1, 0, 100, 0) == 0 and wb(1, 1, 1, 0) == 0
     assert wb(1, 1025, 100, 0) == 0 and wb(1, 1, 100, 7) == 0
@@ -54,7 +56,7 @@ def test_workspace_bytes_host_only(lib, monkeypatch):
     small = wb(1, 6, 32000, 1)
     assert small % 16 == 0 and 256 + 6 * 16 < small <= 256 + 6 * 16 * 64
     assert wb(1, 60, 151936, 0) > 256 + 60 * 16
-    monkeypatch.setenv("MARS_FORCE_SPLIT", "3")
+    hooks.set("HOOK_FORCE_SPLIT", 3)
     assert wb(2, 5, 4000, 1) == 256 + 10 * 3 * 16
 
 
@@ -95,3 +97,24 @@ def test_missing_library_is_an_error(monkeypatch, tmp_path):
     monkeypatch.setattr(build, "LIB", str(tmp_path / "nope.so"))
     with pytest.raises(mars.MarsError, match="no fallback"):
         mars.lib()
+
+
+def test_hooks_are_set_only_through_the_abi(lib, monkeypatch):
+    """The library ignores the environment; a hook is a process-wide integer behind
+    mars_test_hook, which returns the previous value and rejects unknown hooks."""
+    wb = lib.mars_workspace_bytes
+    plain = wb(2, 5, 4000, 1)
+    monkeypatch.setenv("MARS_FORCE_SPLIT", "3")
+    assert wb(2, 5, 4000, 1) == plain
+    assert lib.mars_test_hook(0, 3) == 0
+    assert wb(2, 5, 4000, 1) == 256 + 10 * 3 * 16
+    assert lib.mars_test_hook(0, 0) == 3
+    assert wb(2, 5, 4000, 1) == plain
+    assert lib.mars_test_hook(3, 1) == -1 and lib.mars_test_hook(-1, 1) == -1 and lib.mars_test_hook(0, -2) == -1
+
+
+@pytest.mark.skipif(__import__("torch").cuda.is_available(), reason="host without a GPU only")
+def test_device_check_reports_a_missing_device(lib):
+    sm, tuned = ctypes.c_int(-1), ctypes.c_int(-1)
+    assert lib.mars_device_check(ctypes.byref(sm), ctypes.byref(tuned)) == 4      # MARS_ERR_CUDA
+    assert tuned.value == 148

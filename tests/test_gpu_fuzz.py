@@ -9,6 +9,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
+import hookctl as hooks
+
 import stochastic_checks as ts
 
 pytestmark = pytest.mark.gpu
@@ -82,9 +84,9 @@ def random_case(rng, stochastic: bool):
 def test_deterministic_tree_and_chain(seed, monkeypatch):
     rng = np.random.default_rng(1000 + seed)
     if rng.random() < 0.3:
-        monkeypatch.setenv("MARS_FORCE_SPLIT", str(int(rng.integers(2, 6))))
+        hooks.set("HOOK_FORCE_SPLIT", int(rng.integers(2, 6)))
     else:
-        monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+        hooks.clear("HOOK_FORCE_SPLIT")
     for _ in range(4):
         c = random_case(rng, stochastic=False)
         got = mars.to_host(mars.verify_tree(c["view"], c["tok"], c["parent"], c["theta"], c["flags"], c["Dcap"],
@@ -104,13 +106,13 @@ def test_deterministic_tree_and_chain(seed, monkeypatch):
 @pytest.mark.parametrize("seed", range(40))
 def test_stochastic_tree(seed, monkeypatch):
     rng = np.random.default_rng(5000 + seed)
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
     if rng.random() < 0.3:
-        monkeypatch.setenv("MARS_FORCE_SPLIT", str(int(rng.integers(2, 6))))
+        hooks.set("HOOK_FORCE_SPLIT", int(rng.integers(2, 6)))
     if rng.random() < 0.5:
-        monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(int(rng.choice([1, 2, 4, 8]))))
+        hooks.set("HOOK_STOCH_TAIL_CLUSTER", int(rng.choice([1, 2, 4, 8])))
     else:
-        monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+        hooks.clear("HOOK_STOCH_TAIL_CLUSTER")
     for _ in range(3):
         c = random_case(rng, stochastic=True)
         T = float(rng.choice([0.02, 0.3, 0.7, 1.0, 1.7, 50.0]))
@@ -128,11 +130,11 @@ def test_stochastic_tree(seed, monkeypatch):
 @pytest.mark.parametrize("seed", range(20))
 def test_sampled_chains(seed, monkeypatch):
     rng = np.random.default_rng(9000 + seed)
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
     if rng.random() < 0.5:
-        monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(int(rng.choice([1, 2, 4, 8]))))
+        hooks.set("HOOK_STOCH_TAIL_CLUSTER", int(rng.choice([1, 2, 4, 8])))
     else:
-        monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+        hooks.clear("HOOK_STOCH_TAIL_CLUSTER")
     for _ in range(3):
         B, K = int(rng.integers(1, 40)), int(rng.choice([2, 3, 5, 9]))
         V = int(rng.choice([9, 257, 1000, 5001, 40000]))
@@ -153,8 +155,8 @@ def test_sampled_chains(seed, monkeypatch):
 @pytest.mark.parametrize("seed", range(20))
 def test_sharded_stochastic_tree(seed, monkeypatch):
     rng = np.random.default_rng(7000 + seed)
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
-    monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
+    hooks.clear("HOOK_STOCH_TAIL_CLUSTER")
     for _ in range(2):
         c = random_case(rng, stochastic=True)
         if c["V"] < 8:

@@ -14,6 +14,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
+import hookctl as hooks
+
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 RTOL, ATOL = 2e-4, 1e-5
@@ -102,6 +104,25 @@ def test_small_and_medium_shapes(B, N, V, d, bias):
     ties, tol = compare(out, ref, tok, w.parent, w.theta)
     assert ties <= max(2, B * N // 50) and tol <= max(1, B // 3), (ties, tol)
     assert (out["seq_status"] == 0).all()
+
+
+@pytest.mark.parametrize("B,N,V,d,bias", [(2, 5, 300, 128, True), (5, 60, 5000, 256, False)])
+def test_single_block_kernel_variant(B, N, V, d, bias):
+    """The one-SM form of the MMA kernel (128-row tiles, no cluster), selected by a test hook,
+    must meet the same tolerance and agree with the paired form on every id."""
+    w, b, tok, z = make_case(B, N, V, d, seed=B * 100 + N, with_bias=bias)
+    bd = None if b is None else b.to(DEV)
+    pair = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, bd, tok, w.parent, w.theta, debug=True))
+    hooks.set("HOOK_LMHEAD_SINGLE_BLOCK", 1)
+    out = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, bd, tok, w.parent, w.theta, debug=True))
+    hooks.clear("HOOK_LMHEAD_SINGLE_BLOCK")
+    ref = orc.verify_tree(z, tok, w.parent, float(np.float32(w.theta)))
+    ref["logits"] = z
+    ties, tol = compare(out, ref, tok, w.parent, w.theta)
+    assert ties <= max(2, B * N // 50) and tol <= max(1, B // 3), (ties, tol)
+    # the two forms compute the same sums (possibly rounded in another order)
+    assert np.allclose(out["top2_val"], pair["top2_val"], rtol=1e-5, atol=1e-6)
+    assert (out["top2_id"] != pair["top2_id"]).any(axis=1).sum() <= max(2, B * N // 50)
 
 
 def test_cfg4_full_size_sampled():

@@ -12,6 +12,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
+import hookctl as hooks
+
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 KEYS_TREE = ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "top2_id",
@@ -44,7 +46,7 @@ def run_chain(logits, draft, theta, flags=0, V=None):
 
 @pytest.fixture(autouse=True)
 def _no_forced_split(monkeypatch):
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
 
 
 # ------------------------------------------------------------------ the named workloads
@@ -163,7 +165,7 @@ def test_unaligned_rows_with_canaries(dtype, ld_extra, offset):
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 def test_forced_row_split(monkeypatch, S, dtype):
     """The merge is associative and commutative: any number of slices gives the same bits."""
-    monkeypatch.setenv("MARS_FORCE_SPLIT", str(S))
+    hooks.set("HOOK_FORCE_SPLIT", S)
     w = synth.tree_workload("split", 5, 12, 4, 3, 40000 + 7, dtype, DEV, 5, 0.9, 3.0, 15.0, 30.0, 0.5)
     out, ref = run_tree(w.logits, w.tok, w.parent, 0.9)
     assert_same(out, ref, KEYS_TREE, f"S={S}")
@@ -412,3 +414,12 @@ def test_sorted_rows_worst_case_for_the_filter(dtype):
     out = mars.to_host(mars.verify_chain(big, np.zeros((1300, 1), np.int32), 0.9, debug=True))
     assert np.array_equal(out["top2_id"][:2], idx) and np.array_equal(out["top2_id"][-2:], idx)
     assert np.array_equal(out["top2_val"][:2].view(np.uint32), val.view(np.uint32))
+
+
+def test_device_matches_what_the_launch_shapes_are_tuned_for():
+    """Grid sizes assume 148 SMs; the check reports the device's count so that a part with
+    fewer enabled SMs is noticed (results stay correct, waves fill unevenly)."""
+    info = mars.device_check()
+    assert info["sm_tuned"] == 148
+    assert info["sm_count"] == torch.cuda.get_device_properties(0).multi_processor_count
+    assert (info["status"] == 0) == (info["sm_count"] == 148)

@@ -7,6 +7,8 @@ import torch
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
+import hookctl as hooks
+
 from stochastic_checks import (DEV, STATS, check_walk_is_valid, compare, compare_sampled, host_f64,
                                sampled_case)
 
@@ -15,8 +17,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(autouse=True)
 def _no_hooks(monkeypatch):
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
-    monkeypatch.delenv("MARS_STOCH_TAIL_CLUSTER", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
+    hooks.clear("HOOK_STOCH_TAIL_CLUSTER")
 
 
 def run_and_compare(logits, tok, parent, u, theta, T, flags=0, Dcap=None, what="", **kw):
@@ -115,7 +117,7 @@ def test_unaligned_rows_and_odd_sizes(dtype):
 
 @pytest.mark.parametrize("split", [2, 3, 7])
 def test_forced_row_splits(split, monkeypatch):
-    monkeypatch.setenv("MARS_FORCE_SPLIT", str(split))
+    hooks.set("HOOK_FORCE_SPLIT", split)
     w = synth.tree_workload("t", 10, 12, 3, 3, 20011, torch.bfloat16, DEV, 44, 0.9, 1.0, 6.0, 9.0, 0.4)
     u = synth.make_uniforms(w.B, w.N, 44)
     run_and_compare(w.logits, w.tok, w.parent, u, 0.9, 1.3, what=f"split {split}")
@@ -127,7 +129,7 @@ def test_draw_with_one_block_and_with_clusters(cluster, dtype, monkeypatch):
     """The draw's pass over the row runs in one block or is shared by a cluster of 2, 4 or 8 blocks
     (distributed shared memory); every shape must resolve the same element.  Many sequences stop at the
     root (uniforms next to one), so every part of the row gets drawn from."""
-    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    hooks.set("HOOK_STOCH_TAIL_CLUSTER", cluster)
     w = synth.tree_workload("t", 96, 6, 2, 2, 70001, dtype, DEV, 66, 0.9, 1.0, 3.0, 6.0, 0.4)
     u = synth.make_uniforms(w.B, w.N, 66)
     u[::2, 1:] = np.float32(0.99999)
@@ -309,7 +311,7 @@ def test_sampled_chains(dtype, flags):
 
 @pytest.mark.parametrize("cluster", [1, 2, 4, 8])
 def test_sampled_chains_cluster_shapes(cluster, monkeypatch):
-    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    hooks.set("HOOK_STOCH_TAIL_CLUSTER", cluster)
     w, qdev, zq, draft, qx, u = sampled_case(32, 40, 4, 70001, torch.bfloat16, 1.5)
     u[:, 1] = np.float32(0.99999)          # most sequences reject their first draft: residual draws
     got = mars.to_host(mars.verify_chain_sampled(w.logits, qdev, draft, qx, u, 0.9, 1.0, 1.0, mars.STOCH_PLAIN,

@@ -5,6 +5,8 @@ import torch
 
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
+
+import hookctl as hooks
 from tests.test_gpu_parity import special_rows
 
 pytestmark = pytest.mark.gpu
@@ -22,7 +24,7 @@ def check(logits, k, V=None):
 
 @pytest.fixture(autouse=True)
 def _no_forced_split(monkeypatch):
-    monkeypatch.delenv("MARS_FORCE_SPLIT", raising=False)
+    hooks.clear("HOOK_FORCE_SPLIT")
 
 
 @pytest.mark.parametrize("k", [1, 2, 10, 32])
@@ -49,7 +51,7 @@ def test_topk_odd_sizes_and_degenerate_rows(V, dtype):
 
 @pytest.mark.parametrize("S", [2, 5, 64])
 def test_topk_forced_split_and_unaligned(monkeypatch, S):
-    monkeypatch.setenv("MARS_FORCE_SPLIT", str(S))
+    hooks.set("HOOK_FORCE_SPLIT", S)
     g = torch.Generator(device=DEV); g.manual_seed(S)
     big = torch.full((9, 40007 + 11), 3.0e38, dtype=torch.bfloat16, device=DEV)     # canaries around
     view = big[1:-1, 3:3 + 40007]

@@ -7,6 +7,8 @@ import torch
 
 from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth, vocab_parallel
+
+import hookctl as hooks
 from tests.test_gpu_parity import KEYS_TREE, assert_same, special_rows
 
 from stochastic_checks import sharded_stochastic
@@ -132,7 +134,7 @@ def test_stochastic_sharded_degenerate_rows_and_tiny_shards():
 @pytest.mark.parametrize("cluster", [1, 4, 8])
 def test_stochastic_sharded_cluster_shapes(cluster, monkeypatch):
     import stochastic_checks as sc
-    monkeypatch.setenv("MARS_STOCH_TAIL_CLUSTER", str(cluster))
+    hooks.set("HOOK_STOCH_TAIL_CLUSTER", cluster)
     w = synth.tree_workload("vps", 30, 6, 2, 2, 90011, torch.bfloat16, DEV, 140, 0.9, 1.0, 3.0, 6.0, 0.4)
     u = synth.make_uniforms(w.B, w.N, 140)
     u[::2, 1:] = np.float32(0.99999)

@@ -13,12 +13,23 @@ from paper_2601_15498_b200 import vocab_parallel
 
 
 def test_shard_ranges_cover_the_vocabulary():
-    for V, world in ((151936, 8), (32000, 3), (17, 4), (9, 2)):
+    for V, world in ((151936, 8), (32000, 3), (18, 3), (10, 2), (64, 8), (2, 1)):
         r = vocab_parallel.shard_ranges(V, world)
         assert len(r) == world and r[0][0] == 0 and r[-1][1] == V
         for (a, b), (c, d) in zip(r, r[1:]):
             assert b == c and a <= b
-        assert all(lo % 8 == 0 for lo, hi in r if hi > lo)
+        assert all(lo % 8 == 0 for lo, hi in r)
+        assert all(hi - lo >= 2 for lo, hi in r)
+
+
+def test_shard_ranges_refuse_shards_the_library_cannot_take():
+    """A shard of fewer than two columns is rejected by the library on that rank only, which
+    would leave the other ranks waiting in the all-gather.  The split is a pure function of
+    (V, world), so the refusal happens on every rank, before any collective."""
+    import pytest
+    for V, world in ((100, 8), (17, 4), (9, 2), (1, 1), (64, 0)):
+        with pytest.raises(ValueError):
+            vocab_parallel.shard_ranges(V, world)
 
 
 def _free_port():

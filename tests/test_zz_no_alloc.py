@@ -5,8 +5,10 @@ free HBM to its cache pool, a plug-in op, a loop that cannot afford cudaMalloc's
 synchronisation) and therefore cannot hand over a workspace.  The static entry point uses a
 fixed scratch array inside the library instead.  This test calls it through the C ABI twice in
 a row -- the second call with different inputs, so stale scratch contents would show -- and
-requires the same bits as the regular entry point (the library's tolerance for this path is
-bit-exactness).  It also checks the capacity error.  The file name sorts last on purpose: a
+requires the same bits as the regular entry point and as the CPU oracle (the library's
+tolerance for this path is bit-exactness).  It also checks the capacity error, and that a
+caller's MARS_COUNTERS_ZERO promise -- which nobody can keep for an array they do not own --
+is ignored rather than trusted.  The file name sorts last on purpose: a
 run that stops at the first failure has then already run every other test.
 """
 import ctypes
@@ -15,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import mars_oracle as orc
 from paper_2601_15498_b200 import mars, synth
 
 pytestmark = pytest.mark.gpu
@@ -22,19 +25,22 @@ DEV = "cuda:0"
 KEYS = ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "top2_id", "node_flags")
 
 
-def _run_both(w):
+def _run_both(w, flags=0):
     tok = torch.as_tensor(w.tok, device=DEV)
     parent = torch.as_tensor(w.parent, device=DEV)
     ref = mars.to_host(mars.verify_tree(w.logits, tok, parent, w.theta, debug=True))
     out = mars.alloc_outputs(w.B, w.N, w.N - 1, DEV, debug=True)
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
-    mars.verify_tree_static(w.logits, tok, parent, w.theta, out)
+    mars.verify_tree_static(w.logits, tok, parent, w.theta, out, flags=flags)
     assert torch.cuda.memory_allocated() == before        # the wrapper allocated nothing either
     got = mars.to_host(out)
+    want = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, w.theta)
     for k in KEYS:
         assert np.array_equal(got[k], ref[k]), k
+        assert np.array_equal(got[k], want[k]), ("oracle", k)
     assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32))
+    assert np.array_equal(got["top2_val"].view(np.uint32), want["top2_val"].view(np.uint32))
     return got
 
 
@@ -51,6 +57,19 @@ def test_static_scratch_matches_workspace_entry_point_twice():
                                       3.0, 15.0, 30.0, 0.3))
     assert np.array_equal(a["out_tokens"], c["out_tokens"])
     assert a["accept_len"].shape != b["accept_len"].shape
+
+
+def test_counters_zero_flag_is_not_trusted_for_the_shared_array():
+    """A small batch leaves top-2 records right behind its (short) counter region.  A larger
+    batch whose counter region covers those bytes, called with MARS_COUNTERS_ZERO, would start
+    from dirty counters if the flag were honoured: no sequence would ever see its last arrival
+    and the outputs would stay unwritten."""
+    _run_both(synth.tree_workload("na3", 3, 12, 4, 3, 9000, torch.float32, DEV, 503, 0.9,
+                                  2.0, 20.0, 20.0, 0.4))
+    big = synth.tree_workload("na4", 100, 12, 4, 3, 9000, torch.float32, DEV, 504, 0.9,
+                              2.0, 20.0, 20.0, 0.4)
+    _run_both(big, flags=mars.COUNTERS_ZERO)
+    _run_both(big, flags=mars.COUNTERS_ZERO)
 
 
 def test_static_scratch_rejects_batches_beyond_capacity():
