@@ -18,7 +18,14 @@
  *     sequence in `seq_status`.
  *   - Layout: B sequences, N rows ("nodes") per sequence, row r = b*N + node; the
  *     logits matrix is [B*N, ld] with row stride `ld` >= V elements; only the first V
- *     elements of a row are read.  Rows may start at any element-aligned address;
+ *     elements of a row are read.
+ *   - Consecutive calls on one stream may overlap on the GPU (programmatic dependent launch):
+ *     where a row-streaming kernel of this library directly follows another one in the stream,
+ *     the later call may start reading its LOGITS while the earlier one drains, and waits for
+ *     it to finish before it reads anything else or writes workspace and outputs.  Any other
+ *     operation in between (a copy, a memset, another library's kernel, the producer of the
+ *     logits) is ordered as usual.  The one consequence for a caller: the logits of a call
+ *     must not alias an output buffer of the libmars call right before it on the same stream.  Rows may start at any element-aligned address;
  *     16-byte-aligned rows (ld*sizeof(elem) % 16 == 0 and an aligned base) take the
  *     vector path end to end.
  *   - Decisions are taken in fp32: bf16 logits widen exactly, the ratio is one IEEE
@@ -497,6 +504,8 @@ mars_status_t mars_device_check(int *sm_count, int *sm_tuned);
  *   which 0: slices per logits row (mars_verify_*, mars_top2_shard, mars_topk_rows, stochastic calls)
  *         1: value 1 selects the single-block MMA kernel of mars_lmhead_verify / _top2_shard
  *         2: blocks per cluster of the stochastic tail kernel (1, 2, 4 or 8)
+ *         3: value 1 launches every kernel in plain stream order (no programmatic overlap of
+ *            consecutive calls; a measurement aid)
  *   value 0 clears the hook.  Returns the previous value, or -1 for an unknown hook / negative value.
  */
 int mars_test_hook(int which, int value);

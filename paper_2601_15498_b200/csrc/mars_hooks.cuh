@@ -7,7 +7,8 @@
 
 namespace mars {
 
-enum Hook { kHookForceSplit = 0, kHookLmheadSingleBlock = 1, kHookStochTailCluster = 2, kHookCount = 3 };
+enum Hook { kHookForceSplit = 0, kHookLmheadSingleBlock = 1, kHookStochTailCluster = 2, kHookNoOverlap = 3,
+            kHookCount = 4 };
 
 // Current value of a hook; 0 means "not set" (the library chooses).
 int hook(int which);

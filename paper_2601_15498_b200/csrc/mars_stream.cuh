@@ -26,6 +26,31 @@ __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
     return d;
 }
 
+// Programmatic dependent launch (back-to-back calls on one stream).  A kernel that is launched
+// with programmatic stream serialisation may begin while its predecessor still runs, provided
+// the predecessor lets it: pdl_launch_dependents() does that, and is a no-op otherwise.  Such a
+// kernel must call pdl_wait() before its first access to memory that the predecessor may write
+// or still read-modify (here: workspaces and outputs; logits and other inputs are only read);
+// it returns once the predecessor has completed and its writes are visible.  Without the launch
+// attribute, or without a predecessor that triggers early, both calls do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Launch with programmatic stream serialisation allowed (see above); `allow` = false gives the
+// plain stream order (a measurement aid: the cost of a call without any overlap).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(bool allow, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = allow ? 1 : 0;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <int DT> struct Elem;
 
 template <> struct Elem<MARS_BF16> {

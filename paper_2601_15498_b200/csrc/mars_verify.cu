@@ -57,6 +57,9 @@ __global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
     __shared__ Rec s_warp[kThreads / 32];
     __shared__ int s_last;
 
+    // The next call on this stream may start streaming its rows while this one drains: until
+    // its pdl_wait() it only reads its inputs.
+    pdl_launch_dependents();
     const int tid = threadIdx.x;
     const long long blk = blockIdx.x;
     const long long row = blk / p.S;
@@ -125,6 +128,9 @@ __global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
 #pragma unroll
     for (int m = 16; m > 0; m >>= 1) s = merge(s, shfl_xor_rec(s, m));
     if ((tid & 31) == 0) s_warp[tid >> 5] = s;
+    // Everything up to here only read this call's logits.  Workspace and outputs may still be in
+    // use by the previous call on the stream: wait for it to finish before touching them.
+    pdl_wait();
     __syncthreads();
     if (tid == 0) {
         Rec r = s_warp[0];
@@ -249,13 +255,16 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     p.stage_partials = (sp.S > 1 && tail_bytes + stage_bytes <= 48 * 1024) ? 1 : 0;
     p.tail_smem_off = (int)tail_bytes;
     const size_t smem = tail_bytes + (p.stage_partials ? stage_bytes : 0);
+    cudaError_t le;
+    const bool overlap = hook(kHookNoOverlap) == 0;
     if (dt == MARS_BF16 && sp.S == 1 && R >= kDenseMinRows)
-        verify_kernel<MARS_BF16, kUDense, 8><<<grid, kThreads, smem, st>>>(p);
+        le = launch_pdl(overlap, verify_kernel<MARS_BF16, kUDense, 8>, dim3(grid), dim3(kThreads), smem, st, p);
     else if (dt == MARS_BF16)
-        verify_kernel<MARS_BF16, kU, 4><<<grid, kThreads, smem, st>>>(p);
+        le = launch_pdl(overlap, verify_kernel<MARS_BF16, kU, 4>, dim3(grid), dim3(kThreads), smem, st, p);
     else
-        verify_kernel<MARS_FP32, kU, 4><<<grid, kThreads, smem, st>>>(p);
-    return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
+        le = launch_pdl(overlap, verify_kernel<MARS_FP32, kU, 4>, dim3(grid), dim3(kThreads), smem, st, p);
+    if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    return MARS_OK;
 }
 
 }  // namespace mars

@@ -108,7 +108,7 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
-HOOK_FORCE_SPLIT, HOOK_LMHEAD_SINGLE_BLOCK, HOOK_STOCH_TAIL_CLUSTER = 0, 1, 2
+HOOK_FORCE_SPLIT, HOOK_LMHEAD_SINGLE_BLOCK, HOOK_STOCH_TAIL_CLUSTER, HOOK_NO_OVERLAP = 0, 1, 2, 3
 
 
 def test_hook(which: int, value: int) -> int:
@@ -504,12 +504,14 @@ def stochastic_shard_finish(token_all: torch.Tensor, out: dict) -> dict:
     return out
 
 
-def stream_read_probe(buffer: torch.Tensor, chunk_bytes: int) -> torch.Tensor:
+def stream_read_probe(buffer: torch.Tensor, chunk_bytes: int, out: torch.Tensor | None = None) -> torch.Tensor:
     """mars_selftest_stream_read on the current stream over the whole (contiguous) tensor; returns
-    the one-word result tensor (the call is asynchronous)."""
+    the one-word result tensor (the call is asynchronous).  `out` (int32 [1], zeroed by the
+    caller) avoids the allocation and the fill kernel of a fresh result word."""
     if not (buffer.is_cuda and buffer.is_contiguous()):
         raise MarsError("buffer must be a contiguous device tensor")
-    out = torch.zeros((1,), dtype=torch.int32, device=buffer.device)
+    if out is None:
+        out = torch.zeros((1,), dtype=torch.int32, device=buffer.device)
     with torch.cuda.device(buffer.device):
         code = lib().mars_selftest_stream_read(buffer.data_ptr(), buffer.numel() * buffer.element_size(),
                                                int(chunk_bytes), out.data_ptr(), _stream())
@@ -594,15 +596,18 @@ def verify_records(records: torch.Tensor, tok, parent, theta: float, flags: int 
     return out
 
 
-def top2_histograms(top2_val: torch.Tensor, z1_lo: float, z1_hi: float, nbins: int):
+def top2_histograms(top2_val: torch.Tensor, z1_lo: float, z1_hi: float, nbins: int, out=None):
     """mars_top2_histograms on the current stream: returns (hist uint32-as-int32 [3, nbins],
-    outliers [3]) device tensors."""
+    outliers [3]) device tensors; `out` = such a pair to write into."""
     if not (top2_val.is_cuda and top2_val.dtype == torch.float32 and top2_val.is_contiguous()
             and top2_val.dim() == 2 and top2_val.shape[1] == 2):
         raise MarsError("top2_val must be a contiguous float32 [rows, 2] device tensor")
     dev = top2_val.device
-    hist = torch.empty((3, nbins), dtype=torch.int32, device=dev)
-    outl = torch.empty((3,), dtype=torch.int32, device=dev)
+    if out is None:
+        hist = torch.empty((3, nbins), dtype=torch.int32, device=dev)
+        outl = torch.empty((3,), dtype=torch.int32, device=dev)
+    else:
+        hist, outl = out
     with torch.cuda.device(dev):
         code = lib().mars_top2_histograms(top2_val.data_ptr(), top2_val.shape[0], float(z1_lo),
                                           float(z1_hi), int(nbins), hist.data_ptr(), outl.data_ptr(),
@@ -612,8 +617,9 @@ def top2_histograms(top2_val: torch.Tensor, z1_lo: float, z1_hi: float, nbins: i
 
 
 def topk_rows(logits: torch.Tensor, k: int, V: int | None = None,
-              workspace: torch.Tensor | None = None):
-    """mars_topk_rows on the current stream: (values float32 [rows, k], ids int32 [rows, k])."""
+              workspace: torch.Tensor | None = None, out=None):
+    """mars_topk_rows on the current stream: (values float32 [rows, k], ids int32 [rows, k]);
+    `out` = such a pair to write into."""
     dev = logits.device
     dt, ld, V = _logits_args(logits, logits.shape[0], V)
     rows = logits.shape[0]
@@ -622,8 +628,11 @@ def topk_rows(logits: torch.Tensor, k: int, V: int | None = None,
         raise MarsError("unsupported sizes")
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=dev)
-    val = torch.empty((rows, k), dtype=torch.float32, device=dev)
-    idx = torch.empty((rows, k), dtype=torch.int32, device=dev)
+    if out is None:
+        val = torch.empty((rows, k), dtype=torch.float32, device=dev)
+        idx = torch.empty((rows, k), dtype=torch.int32, device=dev)
+    else:
+        val, idx = out
     with torch.cuda.device(dev):
         code = lib().mars_topk_rows(logits.data_ptr(), ld, dt, rows, V, int(k), val.data_ptr(),
                                     idx.data_ptr(), workspace.data_ptr(), workspace.numel(), _stream())

@@ -3,7 +3,7 @@ splits, the single-block MMA kernel, cluster sizes of the stochastic tail.  conf
 all of them after every test."""
 from paper_2601_15498_b200 import mars
 
-NAMES = ("HOOK_FORCE_SPLIT", "HOOK_LMHEAD_SINGLE_BLOCK", "HOOK_STOCH_TAIL_CLUSTER")
+NAMES = ("HOOK_FORCE_SPLIT", "HOOK_LMHEAD_SINGLE_BLOCK", "HOOK_STOCH_TAIL_CLUSTER", "HOOK_NO_OVERLAP")
 
 
 def set(name: str, value: int) -> None:

@@ -67,3 +67,35 @@ def test_reference_arm_prints_contract_line():
                          capture_output=True, text=True, env=dict(env, RANK="1", WORLD_SIZE="2"),
                          timeout=600)
     assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+def test_parity_helpers_count_planted_mismatches():
+    """The in-run parity verdict of bench.py: bit-exact for the deterministic path, and for the
+    stochastic path only decisions / draws that the oracle itself reports as close may differ."""
+    import numpy as np
+    import bench
+    B = 5
+    ref = {"accept_len": np.arange(B, dtype=np.int32), "out_tokens": np.arange(B * 6, dtype=np.int32).reshape(B, 6),
+           "out_len": np.arange(1, B + 1, dtype=np.int32)}
+    got = {k: v.copy() for k, v in ref.items()}
+    keys = ("accept_len", "out_tokens", "out_len")
+    assert bench.parity_deterministic(got, ref, B, keys)["mismatches"] == 0
+    got["out_tokens"][3, 2] += 1
+    got["accept_len"][1] += 1
+    p = bench.parity_deterministic(got, ref, B, keys)
+    assert p["mismatches"] == 2 and p["checked_sequences"] == B
+
+    N = 4
+    ref = {"accept_len": np.array([1, 2, 0], np.int32), "path_nodes": np.zeros((3, N), np.int32),
+           "out_len": np.array([2, 3, 1], np.int32), "seq_status": np.zeros(3, np.int32),
+           "node_how": np.ones((3, N), np.uint8), "out_tokens": np.array([[7, 9, -1, -1], [4, 5, 6, -1], [3, -1, -1, -1]], np.int32),
+           "node_prob": np.full((3, N), 0.25), "margin": np.array([[1e-3, 1e-2], [1e-6, 1e-2], [1e-3, 1e-7]])}
+    got = {k: v.copy() for k, v in ref.items() if k != "margin"}
+    assert bench.parity_stochastic(got, ref, 3)["mismatches"] == 0
+    got["accept_len"][1] = 1                 # a walk that differs, but its closest decision was within tolerance
+    got["out_tokens"][2, 0] = 8              # another drawn token, the oracle's draw sat on a CDF step
+    p = bench.parity_stochastic(got, ref, 3)
+    assert p["mismatches"] == 0 and p["decisions_within_tolerance"] == 1 and p["draws_within_tolerance"] == 1
+    got["out_tokens"][0, 1] = 1              # a clear draw that differs
+    got["node_prob"][0, 0] *= 1.001
+    assert bench.parity_stochastic(got, ref, 3)["mismatches"] == 2
