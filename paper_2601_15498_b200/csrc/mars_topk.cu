@@ -5,16 +5,17 @@
 // Same streaming structure as the top-2 kernel: a block owns a slice of a row and reads it once
 // with 16-byte loads; a batch of 8 vectors per thread is reduced to its maximum with packed max
 // instructions and skipped unless it reaches the floor, a lower bound on the slice's k-th value.
-// Two forms of the slice selection follow: an optimistic one that only collects candidates
-// while streaming (topk_slice_kernel), and an exact one with per-warp ordered lists that the
-// optimistic one falls back to (topk_slice_exact).  A second small kernel merges the slices of
-// a row, completes rows that have fewer than k entries above -inf, and writes best first.
+// Two forms of the slice selection follow: the streaming one with a queue and one ordered list
+// per block that no warp ever waits for (topk_slice_kernel), and one with per-warp ordered lists
+// that a block falls back to when its queue fills up (topk_slice_exact).  A second small kernel
+// merges the slices of a row, completes rows that have fewer than k entries above -inf, and
+// writes best first.
 //
 // Total order as everywhere in the library: larger value first, lower token id first among
 // equal values, NaN counts as -inf, -0 is reported as +0.
 #include "mars_common.cuh"
 #include "mars_hooks.cuh"
-#include "mars_stream.cuh"
+#include "mars_top2_stream.cuh"
 
 #include <cstdlib>
 
@@ -27,7 +28,7 @@ constexpr int kTkU = 8;
 constexpr int kTkMaxK = 32;
 constexpr int kTkTargetBlocks = 148 * 4;
 constexpr int kTkMinSliceBytes = kTkThreads * kTkU * 16;
-constexpr int kTkCap = 2048;       // candidate slots of the optimistic collection
+constexpr int kTkCap = 1024;       // slots of the slice kernel's queue of elements at or above the floor
 
 struct Cand {
     float z;
@@ -39,7 +40,7 @@ struct TopkParams {
     long long ld;
     int V, S, L, k;
     Cand *partial;   // [R*S, k] unused entries {-inf, kNoId}
-    int *redo;       // [R*S] 1: the optimistic pass ran out of candidate slots for this slice
+    int *redo;       // [R*S] 1: the streaming pass ran out of queue slots for this slice, redo it
     long long nslices;
 };
 
@@ -69,8 +70,8 @@ __device__ __forceinline__ void warp_list_insert(float &wz, int &wid, int lane, 
     }
 }
 
-// Exact slice selection with per-warp lists; always correct, used when the optimistic collection
-// below runs out of room.  Called by all threads of the block.
+// Exact slice selection with per-warp lists; always correct, used when the streaming kernel below
+// runs out of room.  Called by all threads of the block.
 template <int DT>
 __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
 {
@@ -211,22 +212,33 @@ __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
     }
 }
 
-// Slice selection, optimistic form: nothing is ordered while the row streams by.  Elements that
-// reach the current floor -- a valid lower bound on the slice's k-th value -- are appended to a
-// block-wide candidate buffer (one shared-memory atomicAdd each); the floor starts as the k-th
-// largest of the threads' first-batch maxima and is raised once per batch by one warp from the
-// candidates collected so far.  The k best of the buffer are rank-counted at the end.  If the
-// buffer ever fills up (adversarially ordered rows), the block redoes its slice with
-// topk_slice_exact.
+// Slice selection.  A block streams its slice once, like the top-2 kernel (batches of 8 vectors
+// per thread reduced with packed max instructions).  A batch is looked at more closely only if
+// its maximum reaches the floor, a lower bound on the slice's k-th value:
+//   - the floor starts as the k-th largest of the threads' first-batch maxima (values of distinct
+//     elements): every warp orders its lanes' maxima, the k best of each warp go to a small
+//     table, and the table's k-th entry is found by rank counting;
+//   - a thread whose batch reaches the floor appends the elements that do to a queue in shared
+//     memory (one atomicAdd each), nothing more;
+//   - the slice's k best so far live in one ordered list in shared memory.  After appending, a
+//     warp TRIES to take the list (one compare-and-swap, no waiting): if it gets it, it holds
+//     the list in its lanes (lane i = entry i), feeds the queued elements into it one by one (a
+//     ballot and a shuffle each), stores it back and publishes the k-th entry's value as the new
+//     floor; if another warp has it, that warp or a later one will pick the elements up.
+// So nobody ever waits, the floor trails the stream by at most a few elements, about
+// k (1 + ln(batches)) elements reach the queue on unordered data, and the list is the result.
+// If the queue fills up (adversarially ordered rows), the slice is flagged and topk_redo_kernel
+// redoes it with topk_slice_exact.
 template <int DT>
 __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkParams p)
 {
     typedef Elem<DT> E;
     constexpr int kWarps = kTkThreads / 32;
     __shared__ __align__(8) Cand s_cand[kTkCap];
-    __shared__ float s_max[kTkThreads];
+    __shared__ __align__(8) Cand s_list[kTkMaxK];
+    __shared__ float s_top[kWarps * kTkMaxK];
     __shared__ unsigned s_floor;
-    __shared__ int s_n, s_overflow, s_seen;
+    __shared__ int s_tail, s_head, s_lock, s_overflow;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, k = p.k;
     const long long blk = blockIdx.x;
@@ -243,16 +255,24 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     const int tlo = vlo + nvec * E::kVec;
     const int ntail = max(hi - tlo, 0);
     const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
+    constexpr int kBatchVecs = kTkThreads * kTkU;
+    const int nfull = nvec / kBatchVecs;
 
+    uint4 v[kTkU];
+    typename E::packed_t q[kTkU];
+    // batch 0: issue its loads first, so that the set-up below overlaps their latency
+    float bm = (nfull > 0) ? load_batch<DT, kTkU, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, kTkU, true>(vbase, tid, nvec, v, q);
     {   // empty slots carry kNoId so that a reader can tell a reserved slot from a written one
         Cand e; e.z = -INFINITY; e.id = kNoId;
         for (int i = tid; i < kTkCap; i += kTkThreads) s_cand[i] = e;
+        if (tid < kTkMaxK) s_list[tid] = e;
     }
-    if (tid == 0) { s_floor = tk_enc(-INFINITY); s_n = 0; s_overflow = 0; s_seen = 0; }
+    if (tid == 0) { s_floor = tk_enc(-INFINITY); s_tail = 0; s_head = 0; s_lock = 0; s_overflow = 0; }
     __syncthreads();
 
     auto append = [&](float x, int idx) {
-        const int pos = atomicAdd(&s_n, 1);
+        const int pos = atomicAdd(&s_tail, 1);
         if (pos < kTkCap) {
             Cand e; e.z = x; e.id = idx;     // one 8-byte store: value and id become visible together
             *reinterpret_cast<volatile unsigned long long *>(&s_cand[pos]) = *reinterpret_cast<unsigned long long *>(&e);
@@ -260,121 +280,126 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
             s_overflow = 1;
         }
     };
-    // One warp: k-th best of (up to 256 of) the candidates so far -> floor.  Slots that are
-    // reserved but not written yet still hold kNoId and are skipped; every written slot is a
-    // distinct element, so the k-th best of any subset is a valid bound.
-    auto raise_floor = [&]() {
-        const int n = min(*(volatile int *)&s_n, min(kTkCap, 8 * 32));
-        Cand mine[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int i = j * 32 + lane;
-            unsigned long long raw = *reinterpret_cast<volatile unsigned long long *>(&s_cand[i < n ? i : 0]);
-            mine[j] = *reinterpret_cast<Cand *>(&raw);
-            if (i >= n) mine[j].id = kNoId;
+    // Feed the queued elements into the list.  Called by whole warps; `force` skips the
+    // compare-and-swap (used once at the end, when no other warp can be in here).
+    auto drain = [&](bool force) {
+        int got = 1;
+        if (!force) {
+            if (lane == 0) got = atomicCAS(&s_lock, 0, 1) == 0 ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
         }
-        Cand win; win.z = -INFINITY; win.id = kNoId;
-        for (int r = 0; r < k; ++r) {
-            Cand b; b.z = -INFINITY; b.id = kNoId;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (mine[j].id != kNoId && beats(mine[j].z, mine[j].id, b.z, b.id)) b = mine[j];
-#pragma unroll
-            for (int msk = 16; msk > 0; msk >>= 1) {
-                float oz = __shfl_xor_sync(0xffffffffu, b.z, msk);
-                int oi = __shfl_xor_sync(0xffffffffu, b.id, msk);
-                if (oi != kNoId && beats(oz, oi, b.z, b.id)) { b.z = oz; b.id = oi; }
+        if (!got) return;
+        __threadfence_block();
+        // one lane reads the queue's bounds for all: the tail moves while other warps append
+        int i = 0, tail = 0;
+        if (lane == 0) { i = *(volatile int *)&s_head; tail = min(*(volatile int *)&s_tail, kTkCap); }
+        i = __shfl_sync(0xffffffffu, i, 0);
+        tail = __shfl_sync(0xffffffffu, tail, 0);
+        unsigned long long raw = *reinterpret_cast<volatile unsigned long long *>(&s_list[lane]);
+        Cand mine = *reinterpret_cast<Cand *>(&raw);
+        // 32 slots at a time, one per lane.  Lanes do not read at the same instant, so what is
+        // "written" is settled by a ballot: every decision below is the same in all lanes.
+        while (i < tail) {
+            Cand c; c.z = -INFINITY; c.id = kNoId;
+            if (i + lane < tail) {
+                raw = *reinterpret_cast<volatile unsigned long long *>(&s_cand[i + lane]);
+                c = *reinterpret_cast<Cand *>(&raw);
             }
-            win = b;
-            if (win.id == kNoId) break;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (mine[j].id == win.id) mine[j].id = kNoId;
+            const unsigned written = __ballot_sync(0xffffffffu, c.id != kNoId);
+            const int n = written == 0xffffffffu ? 32 : __ffs(~written) - 1;    // leading written slots
+            for (int t = 0; t < n; ++t) {
+                const float cz = __shfl_sync(0xffffffffu, c.z, t);
+                const int cid = __shfl_sync(0xffffffffu, c.id, t);
+                warp_list_insert(mine.z, mine.id, lane, k, cz, cid);
+            }
+            i += n;
+            if (n < 32) break;       // a slot that is reserved but not written yet: a later round takes it
         }
-        if (lane == 0 && win.id != kNoId) atomicMax(&s_floor, tk_enc(win.z));
+        *reinterpret_cast<volatile unsigned long long *>(&s_list[lane]) = *reinterpret_cast<unsigned long long *>(&mine);
+        if (lane == k - 1 && mine.id != kNoId) atomicMax(&s_floor, tk_enc(mine.z));
         __syncwarp();
+        if (lane == 0) {
+            *(volatile int *)&s_head = i;
+            __threadfence_block();
+            if (!force) atomicExch(&s_lock, 0);
+        }
     };
 
     if (tid < nhead) { float x = E::scalar(rowp, lo + tid); if (x > -INFINITY) append(x, lo + tid); }
     if (tid < ntail) { float x = E::scalar(rowp, tlo + tid); if (x > -INFINITY) append(x, tlo + tid); }
 
-    constexpr int kBatchVecs = kTkThreads * kTkU;
-    const int nbatches = (nvec + kBatchVecs - 1) / kBatchVecs;
-    for (int bi = 0; bi < nbatches; ++bi) {
-        uint4 v[kTkU];
-        typename E::packed_t q[kTkU];
-        const int v0 = bi * kBatchVecs + tid;
+    // k-th largest of the 256 first-batch maxima.  A lane can only be among the block's k largest
+    // if it is among its warp's k largest: those go to the table, ordered.
+    {
+        const float mine = (bm == bm) ? bm : -INFINITY;
+        int wrank = 0;
 #pragma unroll
-        for (int u = 0; u < kTkU; ++u) {
-            int vi = v0 + u * kTkThreads;
-            v[u] = vi < nvec ? ld_stream(vbase + vi) : E::neg_inf();
+        for (int j = 0; j < 32; ++j) {
+            const float o = __shfl_sync(0xffffffffu, mine, j);
+            wrank += (o > mine || (o == mine && j < lane)) ? 1 : 0;
         }
-        typename E::packed_t m = E::vred(v[0]);
-        q[0] = m;
-#pragma unroll
-        for (int u = 1; u < kTkU; ++u) { q[u] = E::vred(v[u]); m = E::pmax(m, q[u]); }
-        const float bm = E::to_float(m);
-        if (bi == 0) {
-            // floor = k-th largest of the threads' first-batch maxima (values of distinct
-            // elements).  Two levels: a lane can only be among the block's k largest if it is
-            // among its warp's k largest, so only those lanes (at most 8k) are ranked block-wide.
-            const float mine = (bm == bm) ? bm : -INFINITY;
-            int wrank = 0;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float o = __shfl_sync(0xffffffffu, mine, j);
-                wrank += (o > mine || (o == mine && j < lane)) ? 1 : 0;
+        if (wrank < k) s_top[warp * k + wrank] = mine;
+        __syncthreads();
+        const int nt = kWarps * k;
+        if (tid < nt) {
+            const float t = s_top[tid];
+            int rank = 0;
+            for (int j = 0; j < nt; ++j) {
+                const float o = s_top[j];
+                rank += (o > t || (o == t && j < tid)) ? 1 : 0;
             }
-            s_max[tid] = wrank < k ? mine : -INFINITY;     // slot = warp * 32 + lane
-            __syncthreads();
-            if (wrank < k && mine > -INFINITY) {
-                int rank = 0;
-                for (int j = 0; j < kTkThreads; ++j) {
-                    const float o = s_max[j];
-                    rank += (o > mine || (o == mine && j < tid)) ? 1 : 0;
-                }
-                if (rank == k - 1) atomicMax(&s_floor, tk_enc(mine));
-            }
-            __syncthreads();
-        } else if ((bi & (kWarps - 1)) == warp) {
-            // raise the floor when enough new candidates have come in to move the k-th best
-            const int n_now = *(volatile int *)&s_n;
-            if (n_now - *(volatile int *)&s_seen >= max(2, k / 4)) {
-                raise_floor();
-                if (lane == 0) s_seen = n_now;
-            }
+            if (rank == k - 1 && t > -INFINITY) atomicMax(&s_floor, tk_enc(t));
         }
+        __syncthreads();
+    }
+
+    auto scan = [&](int v0) {
         const float floor_v = tk_dec(*(volatile unsigned *)&s_floor);
+        bool appended = false;
         if (bm >= floor_v) {
 #pragma unroll
             for (int u = 0; u < kTkU; ++u) {
                 if (E::to_float(q[u]) >= floor_v) {
-                    const int base = vlo + (v0 + u * kTkThreads) * E::kVec;
+                    unsigned em = 0;
 #pragma unroll
                     for (int e = 0; e < E::kVec; ++e) {
                         const float x = E::elem(v[u], e);
-                        if (x >= floor_v && x > -INFINITY) append(x, base + e);
+                        em |= (x >= floor_v && x > -INFINITY) ? (1u << e) : 0u;
+                    }
+                    const int base = vlo + (v0 + u * kTkThreads) * E::kVec;
+                    while (em) {
+                        const int e = __ffs(em) - 1;
+                        em &= em - 1;
+                        append(E::elem(v[u], e), base + e);
+                        appended = true;
                     }
                 }
             }
         }
+        if (__any_sync(0xffffffffu, appended)) drain(false);
+    };
+
+    scan(tid);
+    for (int bi = 1; bi < nfull; ++bi) {
+        bm = load_batch<DT, kTkU, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
+        scan(bi * kBatchVecs + tid);
+    }
+    if (nfull > 0 && nfull * kBatchVecs < nvec) {
+        bm = load_batch<DT, kTkU, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        scan(nfull * kBatchVecs + tid);
     }
     __syncthreads();
     if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_redo_kernel
     if (s_overflow) return;
-    const int n = s_n;
-    Cand *out = p.partial + (size_t)blk * k;
-    for (int i = tid; i < k; i += kTkThreads) { out[i].z = -INFINITY; out[i].id = kNoId; }
-    __syncthreads();
-    for (int i = tid; i < n; i += kTkThreads) {
-        const Cand c = s_cand[i];
-        int rank = 0;
-        for (int j = 0; j < n && rank < k; ++j) rank += beats(s_cand[j].z, s_cand[j].id, c.z, c.id) ? 1 : 0;
-        if (rank < k) out[rank] = c;
+    if (warp == 0) {
+        drain(true);                             // whatever is still queued
+        __syncwarp();
+        Cand *out = p.partial + (size_t)blk * k;
+        if (lane < k) out[lane] = s_list[lane];  // ordered; unused entries are {-inf, kNoId}
     }
 }
 
-// Slices whose optimistic pass overflowed are redone exactly.  A small persistent grid scans the
+// Slices that the streaming pass flagged are redone exactly.  A small persistent grid scans the
 // flags; without flagged slices this kernel only reads them.
 template <int DT>
 __global__ void __launch_bounds__(kTkThreads) topk_redo_kernel(const TopkParams p)

@@ -70,3 +70,21 @@ def test_topk_host_errors():
     for k in (0, 33, 101):
         with pytest.raises(mars.MarsError):
             mars.topk_rows(z, k)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_topk_whole_rows_that_defeat_the_floor(dtype):
+    """Whole rows (one block per row): ascending values overflow the candidate buffer and take the
+    exact fallback; constant rows tie everywhere (lowest ids win); a row whose large values all sit
+    in the last batch; and a row with fewer than k entries above -inf."""
+    V, k = 151936, 10
+    z = torch.empty((600, V), dtype=dtype, device=DEV)
+    g = torch.Generator(device=DEV); g.manual_seed(77)
+    z.copy_((torch.randn((600, V), generator=g, device=DEV) * 3).to(dtype))
+    z[0] = torch.linspace(-8, 8, V, device=DEV).to(dtype)
+    z[1] = 1.25
+    z[2, -500:] += 40.0
+    z[3] = float("-inf"); z[3, 77] = 1.0; z[3, 140000] = float("nan"); z[3, 9] = -2.0
+    z[4] = torch.linspace(8, -8, V, device=DEV).to(dtype)
+    check(z, k)
+    check(z[:8], 32)
