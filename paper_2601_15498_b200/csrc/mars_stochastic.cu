@@ -635,6 +635,9 @@ __global__ void __launch_bounds__(kTailThreads, MODE == 1 ? 1 : 2) stoch_tail_ke
     const int b = (int)(blockIdx.x / G);
     const int N = p.N, V = p.V, S = p.S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // The next call's streaming kernel may start reading its logits while this kernel runs; it
+    // waits for this kernel before it writes records.
+    pdl_launch_dependents();
 
     int32_t *s_id1 = reinterpret_cast<int32_t *>(smem_dyn);
     int32_t *s_id2 = s_id1 + N;
@@ -1011,6 +1014,9 @@ __global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const Stre
         soft_merge(ref, sum, rb, sb);
     }
     if ((tid & 31) == 0) { s_warp[tid >> 5] = s; s_soft[tid >> 5] = make_float2(ref, sum); }
+    // Up to here only this call's logits were read.  The records below go to the workspace, which
+    // the previous call's tail kernel may still be reading: wait for it (see pdl_wait).
+    pdl_wait();
     __syncthreads();
     if (tid == 0) {
         Rec r = s_warp[0];
@@ -1165,9 +1171,13 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     // 4 vectors per batch in two register buffers, 4 blocks per SM (64 registers): measured
     // best for both dtypes; 5 or 6 blocks per SM spill the second buffer and run at half speed,
     // and 2 vectors per batch at 5 to 8 blocks per SM lose 10 to 50 %.
-    if (dt == MARS_BF16) stoch_stream_kernel<MARS_BF16, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
-    else stoch_stream_kernel<MARS_FP32, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
-    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    {
+        const bool overlap = hook(kHookNoOverlap) == 0;
+        const cudaError_t le = (dt == MARS_BF16)
+            ? launch_pdl(overlap, stoch_stream_kernel<MARS_BF16, 4, 4>, dim3(grid), dim3(kThreads), 0, st, sp1)
+            : launch_pdl(overlap, stoch_stream_kernel<MARS_FP32, 4, 4>, dim3(grid), dim3(kThreads), 0, st, sp1);
+        if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    }
 
     StochTailParams tp;
     tp.logits = logits; tp.ld = ld; tp.V = V; tp.N = N; tp.S = sp.S; tp.c = (float)cd; tp.theta = theta;
@@ -1292,9 +1302,13 @@ mars_status_t mars_stochastic_shard_records(const void *logits_local, int64_t ld
     sp1.logits = logits_local; sp1.ld = ld; sp1.V = V_local; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
     sp1.partial = (SRec *)workspace;
     const unsigned grid = (unsigned)(R * sp.S);
-    if (dt == MARS_BF16) stoch_stream_kernel<MARS_BF16, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
-    else stoch_stream_kernel<MARS_FP32, 4, 4><<<grid, kThreads, 0, st>>>(sp1);
-    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    {
+        const bool overlap = hook(kHookNoOverlap) == 0;
+        const cudaError_t le = (dt == MARS_BF16)
+            ? launch_pdl(overlap, stoch_stream_kernel<MARS_BF16, 4, 4>, dim3(grid), dim3(kThreads), 0, st, sp1)
+            : launch_pdl(overlap, stoch_stream_kernel<MARS_FP32, 4, 4>, dim3(grid), dim3(kThreads), 0, st, sp1);
+        if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    }
     ShardRecordsParams rp;
     rp.logits = logits_local; rp.ld = ld; rp.V = V_local; rp.N = N; rp.S = sp.S; rp.id_offset = id_offset; rp.R = R;
     rp.flags = flags; rp.partial = sp1.partial; rp.tok = tok; rp.parent = parent;

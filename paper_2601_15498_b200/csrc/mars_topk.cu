@@ -388,6 +388,9 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
         bm = load_batch<DT, kTkU, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
         scan(nfull * kBatchVecs + tid);
     }
+    // Up to here only this call's logits were read; the workspace may still be in use by the
+    // previous call's merge kernel (see pdl_wait).
+    pdl_wait();
     __syncthreads();
     if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_redo_kernel
     if (s_overflow) return;
@@ -413,6 +416,7 @@ __global__ void __launch_bounds__(128) topk_merge_kernel(const TopkParams p, flo
 {
     extern __shared__ Cand s_c[];
     __shared__ int s_found;
+    pdl_launch_dependents();     // the next call's slice kernel may start streaming its rows
     const int k = p.k, n = p.S * k;
     const long long row = blockIdx.x;
     const Cand *src = p.partial + (size_t)row * n;
@@ -502,9 +506,13 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
     p.redo = (int *)((char *)workspace + (size_t)p.nslices * k * sizeof(Cand));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const unsigned grid = (unsigned)(rows * sp.S);
-    if (dt == MARS_BF16) topk_slice_kernel<MARS_BF16><<<grid, kTkThreads, 0, st>>>(p);
-    else topk_slice_kernel<MARS_FP32><<<grid, kTkThreads, 0, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
+    {
+        const bool overlap = hook(kHookNoOverlap) == 0;
+        const cudaError_t le = (dt == MARS_BF16)
+            ? launch_pdl(overlap, topk_slice_kernel<MARS_BF16>, dim3(grid), dim3(kTkThreads), 0, st, p)
+            : launch_pdl(overlap, topk_slice_kernel<MARS_FP32>, dim3(grid), dim3(kTkThreads), 0, st, p);
+        if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    }
     const unsigned redo_grid = (unsigned)(p.nslices < 148 * 2 ? p.nslices : 148 * 2);
     if (dt == MARS_BF16) topk_redo_kernel<MARS_BF16><<<redo_grid, kTkThreads, 0, st>>>(p);
     else topk_redo_kernel<MARS_FP32><<<redo_grid, kTkThreads, 0, st>>>(p);

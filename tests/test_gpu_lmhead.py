@@ -125,11 +125,15 @@ def test_single_block_kernel_variant(B, N, V, d, bias):
     assert (out["top2_id"] != pair["top2_id"]).any(axis=1).sum() <= max(2, B * N // 50)
 
 
-def test_cfg4_full_size_sampled():
-    """Full operands (3840 x 4096 hidden, 151 936 x 4096 vocabulary); the fp64 oracle checks a
-    sample of whole sequences, every row's top-2 is checked against a bf16 matmul reference."""
+def test_cfg4_full_size():
+    """Full operands (3840 x 4096 hidden, 151 936 x 4096 vocabulary).  Sixteen whole sequences go
+    through the fp64 oracle (projection in slabs); every other row's top-2 is held against a device
+    fp32 matmul of the same operands under the same near-tie rule: the reported logits must match
+    the reference logits at the reported ids, and another id is accepted only where the reference
+    logits of the two candidates are that close."""
     w = synth.cfg4_operands(DEV)
-    sample = [0, 17, 63]
+    sample = list(range(0, w.B, 4))
+    assert len(sample) == 16
     rows = np.concatenate([np.arange(b * w.N, (b + 1) * w.N) for b in sample])
     hb = bits(w.hidden)[rows]
     z = np.empty((len(rows), w.V))
@@ -144,15 +148,29 @@ def test_cfg4_full_size_sampled():
         lead[r0:r0 + 480] = torch.topk(zz, 2, dim=1).indices.cpu().numpy()
     lead[rows] = lead_s
     tok = synth.make_tokens(w.parent, lead, w.V, 4)
-    out = mars.to_host(mars.lmhead_verify(w.hidden, w.w_vocab, None, tok, w.parent, w.theta, debug=True))
+    dev_out = mars.lmhead_verify(w.hidden, w.w_vocab, None, tok, w.parent, w.theta, debug=True)
+    out = mars.to_host(dev_out)
     assert (out["seq_status"] == 0).all()
     ref = orc.verify_tree(z, tok[sample], w.parent[sample], float(np.float32(w.theta)))
     got = {k: (v[rows] if k in ("top2_val", "top2_id") else v[sample]) for k, v in out.items()}
     ties, tol = compare(got, ref, tok[sample], w.parent[sample], w.theta, z)
-    assert ties <= 4 and tol <= 1, (ties, tol)
-    # every row: ids agree with the device fp32 matmul up to near ties
-    mism = (out["top2_id"] != lead).any(axis=1).mean()
-    assert mism < 0.02, mism
+    assert ties <= 12 and tol <= 3, (ties, tol)
+    # every row against the device fp32 matmul (its own rounding differs from the kernel's by the
+    # order of d additions: both lie within RTOL of the exact logit)
+    near_ties = 0
+    ids = dev_out["top2_id"].long()
+    vals = dev_out["top2_val"]
+    for r0 in range(0, w.B * w.N, 480):
+        zz = w.hidden[r0:r0 + 480].float() @ w.w_vocab.float().T
+        tv, ti = torch.topk(zz, 2, dim=1)
+        gi, gv = ids[r0:r0 + 480], vals[r0:r0 + 480]
+        at_ids = torch.gather(zz, 1, gi)
+        assert torch.allclose(gv, at_ids, rtol=RTOL, atol=ATOL)
+        differ = gi != ti
+        close = (at_ids - tv).abs() <= RTOL * tv.abs() + ATOL
+        assert bool((~differ | close).all()), "another id without a near tie"
+        near_ties += int(differ.any(dim=1).sum())
+    assert near_ties < 0.02 * w.B * w.N, near_ties
     assert ((out["accept_len"] >= 0) & (out["accept_len"] <= w.max_depth)).all()
     assert out["accept_len"].mean() > 0.5
 

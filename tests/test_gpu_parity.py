@@ -96,9 +96,9 @@ def test_cfg3_reduced_batch_full_parity(dtype):
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_cfg3_full_size_sampled(dtype):
-    """The serving-scale workload in the launch configuration the benchmark times; the oracle
-    checks a sample of whole sequences, every sequence is checked for validity."""
+def test_cfg3_full_size_every_sequence(dtype):
+    """The serving-scale workload in the launch configuration the benchmark times: all 256
+    sequences (15 360 rows) bit for bit against the oracle, in host-memory-sized chunks."""
     w = synth.cfg3(DEV, dtype=dtype)
     assert w.R == 15360
     # as the benchmark launches it: workspace zeroed once, counters left to the kernel's own reset
@@ -107,13 +107,13 @@ def test_cfg3_full_size_sampled(dtype):
     mars.verify_tree(w.logits, w.tok, w.parent, w.theta, flags=mars.COUNTERS_ZERO, workspace=work)
     out = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, flags=mars.COUNTERS_ZERO,
                                         debug=True, workspace=work))
-    rng = np.random.default_rng(0)
-    sample = sorted(set(rng.choice(w.B, 10, replace=False).tolist()) | {0, w.B - 1})
-    rows = np.concatenate([np.arange(b * w.N, (b + 1) * w.N) for b in sample])
-    sub = w.logits[torch.as_tensor(rows, device=DEV)]
-    ref = orc.verify_tree(synth.to_numpy_bits(sub), w.tok[sample], w.parent[sample], w.theta)
-    got = {k: (v[rows] if k in ("top2_val", "top2_id") else v[sample]) for k, v in out.items()}
-    assert_same(got, ref, KEYS_TREE, w.name)
+    step = 64
+    for b0 in range(0, w.B, step):
+        b1 = min(w.B, b0 + step)
+        ref = orc.verify_tree(synth.to_numpy_bits(w.logits[b0 * w.N:b1 * w.N]), w.tok[b0:b1], w.parent[b0:b1], w.theta)
+        got = {k: (v[b0 * w.N:b1 * w.N] if k in ("top2_val", "top2_id") else v[b0:b1]) for k, v in out.items()}
+        assert_same(got, ref, KEYS_TREE, f"{w.name} sequences {b0}..{b1}")
+        assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32))
     # properties that hold for every sequence
     assert (out["seq_status"] == 0).all()
     assert ((out["accept_len"] >= 0) & (out["accept_len"] <= w.max_depth)).all()

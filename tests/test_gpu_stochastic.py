@@ -277,20 +277,25 @@ def test_host_errors():
         mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, workspace=small[:16])
 
 
-def test_full_size_batch_sampled_sequences():
+def test_full_size_batch_every_sequence():
     """The serving-scale batch in the launch configuration the benchmark times (256 x 60 rows of
-    151 936 bf16 logits); the oracle checks a sample of whole sequences."""
+    151 936 bf16 logits): every sequence against the oracle under the tolerance policy, in
+    host-memory-sized chunks."""
     w = synth.cfg3(DEV)
     u = synth.make_uniforms(w.B, w.N, 3)
     got = mars.to_host(mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, w.theta, 1.0, debug=True))
     assert (got["seq_status"] == 0).all()
-    pick = np.random.default_rng(0).choice(w.B, 10, replace=False)
-    for b in pick:
-        rows = synth.to_numpy_bits(w.logits[b * w.N:(b + 1) * w.N])
-        ref = orc.verify_tree_stochastic(rows, w.tok[b:b + 1], w.parent[b:b + 1], u[b:b + 1], w.theta, 1.0)
-        one = {k: got[k][b:b + 1] for k in got}
-        compare(one, ref, w.tok[b:b + 1], w.parent[b:b + 1], host_f64(w.logits[b * w.N:(b + 1) * w.N]),
-                u[b:b + 1], 1.0, f"sequence {b}", max_close_frac=1.0)
+    step, close, neigh = 16, 0, 0
+    for b0 in range(0, w.B, step):
+        b1 = b0 + step
+        rows = w.logits[b0 * w.N:b1 * w.N]
+        ref = orc.verify_tree_stochastic(synth.to_numpy_bits(rows), w.tok[b0:b1], w.parent[b0:b1], u[b0:b1], w.theta, 1.0)
+        part = {k: got[k][b0:b1] for k in got}
+        c, n = compare(part, ref, w.tok[b0:b1], w.parent[b0:b1], host_f64(rows), u[b0:b1], 1.0,
+                       f"sequences {b0}..{b1}", max_close_frac=1.0)
+        close += c
+        neigh += n
+    assert close <= 3 and neigh <= 3, (close, neigh)      # 2e-5 / 1e-5 windows over 256 walks and draws
     for b in range(w.B):
         check_walk_is_valid(got, w.tok, w.parent, b)
 
