@@ -671,7 +671,8 @@ def topk_case(name: str, dev, mars, local: int, steps=None, warm=5, parity_rows:
     val_g, id_g = out[0].cpu().numpy()[pick], out[1].cpu().numpy()[pick]
     bad = int(((id_g != id_o).any(axis=1) | (val_g.view(np.uint32) != val_o.view(np.uint32)).any(axis=1)).sum())
     us = r["ms_per_step"] * 1e3
-    roof = hbm_roofline(w.logits_bytes, r["ms_per_step"], "mars::topk_stream_kernel")
+    roof = hbm_roofline(w.logits_bytes, r["ms_per_step"], "mars::topk_slice_kernel",
+                        traffic=ncu_traffic(name) if rows == 7680 else None)
     return {"workload": f"topk_k{k}_rows{rows}_v{w.V}_{dts}", "rows_per_step": rows, "k": k,
             "logits_bytes_per_step": w.logits_bytes, "us_per_step": us, "step_us": r["step_us"], "steps": r["steps"],
             "timed_region_ms": r["region_ms"], "launch": r["launch"], "l2": "inputs larger than L2",

@@ -42,6 +42,8 @@ struct TopkParams {
     Cand *partial;   // [R*S, k] unused entries {-inf, kNoId}
     int *redo;       // [R*S] 1: the streaming pass ran out of queue slots for this slice, redo it
     long long nslices;
+    float *out_val;      // [R, k] final values, best first
+    int32_t *out_id;     // [R, k] final token ids
 };
 
 // Order-preserving float <-> uint encoding for the block-wide bound (atomicMax on shared memory).
@@ -212,6 +214,19 @@ __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
     }
 }
 
+// Fewer than k entries above -inf in a row: the remaining places go to the lowest unused ids at
+// -inf (every -inf / NaN entry ties, lowest id first).  One thread.
+__device__ void complete_row(float *ov, int32_t *oi, int found, int k)
+{
+    int next = 0;
+    while (found < k) {
+        bool used = false;
+        for (int j = 0; j < found; ++j) used |= (oi[j] == next);
+        if (!used) { ov[found] = -INFINITY; oi[found] = next; ++found; }
+        ++next;
+    }
+}
+
 // Slice selection.  A block streams its slice once, like the top-2 kernel (batches of 8 vectors
 // per thread reduced with packed max instructions).  A batch is looked at more closely only if
 // its maximum reaches the floor, a lower bound on the slice's k-th value:
@@ -227,7 +242,7 @@ __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
 //     floor; if another warp has it, that warp or a later one will pick the elements up.
 // So nobody ever waits, the floor trails the stream by at most a few elements, about
 // k (1 + ln(batches)) elements reach the queue on unordered data, and the list is the result.
-// If the queue fills up (adversarially ordered rows), the slice is flagged and topk_redo_kernel
+// If the queue fills up (adversarially ordered rows), the slice is flagged and topk_finish_kernel
 // redoes it with topk_slice_exact.
 template <int DT>
 __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkParams p)
@@ -392,39 +407,54 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     // previous call's merge kernel (see pdl_wait).
     pdl_wait();
     __syncthreads();
-    if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_redo_kernel
+    if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_finish_kernel
     if (s_overflow) return;
     if (warp == 0) {
         drain(true);                             // whatever is still queued
         __syncwarp();
-        Cand *out = p.partial + (size_t)blk * k;
-        if (lane < k) out[lane] = s_list[lane];  // ordered; unused entries are {-inf, kNoId}
+        const Cand c = s_list[lane];             // ordered; unused entries are {-inf, kNoId}
+        if (p.S > 1) {
+            if (lane < k) p.partial[(size_t)blk * k + lane] = c;
+        } else {
+            // a whole row: the list is the row's result, write it out here
+            float *ov = p.out_val + (size_t)row * k;
+            int32_t *oi = p.out_id + (size_t)row * k;
+            const bool real = lane < k && c.id != kNoId;
+            if (real) { ov[lane] = c.z + 0.0f; oi[lane] = c.id; }
+            const int found = __popc(__ballot_sync(0xffffffffu, real));
+            __syncwarp();
+            if (lane == 0 && found < k) complete_row(ov, oi, found, k);
+        }
     }
 }
 
-// Slices that the streaming pass flagged are redone exactly.  A small persistent grid scans the
-// flags; without flagged slices this kernel only reads them.
+// Finish: one block per row.  Slices that the streaming pass flagged are redone exactly; the S
+// ordered slice lists of the row are merged, the row is completed if it has fewer than k entries
+// above -inf, and written best first.  Rows that were not split and not flagged were already
+// written by the slice kernel: their block returns at once.
 template <int DT>
-__global__ void __launch_bounds__(kTkThreads) topk_redo_kernel(const TopkParams p)
-{
-    for (long long blk = blockIdx.x; blk < p.nslices; blk += gridDim.x)
-        if (p.redo[blk]) topk_slice_exact<DT>(p, blk);      // block-uniform condition
-}
-
-// Merge the S sorted slice lists of a row, complete and write it.  One block per row.
-__global__ void __launch_bounds__(128) topk_merge_kernel(const TopkParams p, float *out_val, int32_t *out_id)
+__global__ void __launch_bounds__(kTkThreads) topk_finish_kernel(const TopkParams p)
 {
     extern __shared__ Cand s_c[];
     __shared__ int s_found;
     pdl_launch_dependents();     // the next call's slice kernel may start streaming its rows
-    const int k = p.k, n = p.S * k;
+    const int k = p.k, S = p.S, n = S * k;
     const long long row = blockIdx.x;
+    bool any_redo = false;
+    for (int sl = 0; sl < S; ++sl) any_redo |= p.redo[row * S + sl] != 0;      // block-uniform
+    if (S == 1 && !any_redo) return;
+    if (any_redo) {
+        for (int sl = 0; sl < S; ++sl)
+            if (p.redo[row * S + sl]) topk_slice_exact<DT>(p, row * S + sl);
+        __threadfence_block();
+        __syncthreads();
+    }
     const Cand *src = p.partial + (size_t)row * n;
     if (threadIdx.x == 0) s_found = 0;
     for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
     __syncthreads();
-    float *ov = out_val + (size_t)row * k;
-    int32_t *oi = out_id + (size_t)row * k;
+    float *ov = p.out_val + (size_t)row * k;
+    int32_t *oi = p.out_id + (size_t)row * k;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const Cand c = s_c[i];
         if (c.id == kNoId) continue;
@@ -433,17 +463,7 @@ __global__ void __launch_bounds__(128) topk_merge_kernel(const TopkParams p, flo
         if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
     }
     __syncthreads();
-    // Fewer than k entries above -inf: the remaining places go to the lowest unused ids at -inf
-    // (every -inf / NaN entry ties, lowest id first).
-    if (threadIdx.x == 0 && s_found < k) {
-        int found = s_found, next = 0;
-        while (found < k) {
-            bool used = false;
-            for (int j = 0; j < found; ++j) used |= (oi[j] == next);
-            if (!used) { ov[found] = -INFINITY; oi[found] = next; ++found; }
-            ++next;
-        }
-    }
+    if (threadIdx.x == 0 && s_found < k) complete_row(ov, oi, s_found, k);
 }
 
 struct TkSplit { int S, L; };
@@ -503,6 +523,7 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
     p.logits = logits; p.ld = ld; p.V = V; p.S = sp.S; p.L = sp.L; p.k = k;
     p.partial = (Cand *)workspace;
     p.nslices = rows * sp.S;
+    p.out_val = out_val; p.out_id = out_id;
     p.redo = (int *)((char *)workspace + (size_t)p.nslices * k * sizeof(Cand));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const unsigned grid = (unsigned)(rows * sp.S);
@@ -513,11 +534,9 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
             : launch_pdl(overlap, topk_slice_kernel<MARS_FP32>, dim3(grid), dim3(kTkThreads), 0, st, p);
         if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
     }
-    const unsigned redo_grid = (unsigned)(p.nslices < 148 * 2 ? p.nslices : 148 * 2);
-    if (dt == MARS_BF16) topk_redo_kernel<MARS_BF16><<<redo_grid, kTkThreads, 0, st>>>(p);
-    else topk_redo_kernel<MARS_FP32><<<redo_grid, kTkThreads, 0, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return MARS_ERR_CUDA;
-    topk_merge_kernel<<<(unsigned)rows, 128, (size_t)sp.S * k * sizeof(Cand), st>>>(p, out_val, out_id);
+    const size_t fsmem = (size_t)sp.S * k * sizeof(Cand);
+    if (dt == MARS_BF16) topk_finish_kernel<MARS_BF16><<<(unsigned)rows, kTkThreads, fsmem, st>>>(p);
+    else topk_finish_kernel<MARS_FP32><<<(unsigned)rows, kTkThreads, fsmem, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
