@@ -985,7 +985,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS) + ["cfg4"] + TOPK_WORKLOADS)
+    ap.add_argument("--workload", default="cfg3_bf16", choices=sorted(WORKLOADS) + ["cfg4", "telemetry"] + TOPK_WORKLOADS)
     ap.add_argument("--shard", default="seq", choices=["seq", "vocab"],
                     help="how N > 1 ranks share the work: independent sequences (no collective) or column "
                          "ranges of the vocabulary (one all-gather of 16-byte records per step)")
@@ -1012,7 +1012,7 @@ def main():
         lmhead_arm(args, rank, world, local)
         return
     if args.impl == "reference":
-        if args.workload.startswith("topk"):
+        if args.workload.startswith("topk") or args.workload == "telemetry":
             args.workload = "cfg3_bf16"
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
@@ -1032,6 +1032,17 @@ def main():
             e = topk_case(args.workload, dev, mars, local, steps=args.steps, warm=max(args.warmup or 5, 3),
                           batch=args.batch)
             print(json.dumps(e), flush=True)
+        return
+
+    if args.workload == "telemetry":
+        if rank == 0:
+            build.build()
+            mars.lib()
+            from oracle import mars_oracle as orc
+            w = synth.cfg3(dev, seed=3, B=args.batch or 256)
+            top2_host, _ = orc.top2(synth.to_numpy_bits(w.logits))      # inputs of the call: the oracle's top-2
+            del w
+            print(json.dumps(telemetry_entry(dev, mars, local, top2_host)), flush=True)
         return
 
     default_run = (args.workload == "cfg3_bf16" and world == 1 and not args.batch and not args.stochastic

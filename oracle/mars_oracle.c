@@ -36,7 +36,8 @@
  *     lowest node index among equally deep ones; the emitted next token is the top-1
  *     of that node's row.
  *   Pinned by tests against: a sort-based top-2, the paper's Fig. 2 worked example,
- *   planted ratios one ulp around theta, strict-greedy equivalence for theta >= 1,
+ *   planted ratios one ulp around theta (in fp32 and, for the "_f64" rule, in fp64, directly
+ *   and through a one-hot output projection), strict-greedy equivalence for theta >= 1,
  *   brute-force path enumeration on all small trees, closed-form acceptance rates.
  *   Parity unpinned by the paper (conventions only): the sign guard, NaN handling,
  *   the tie rules (equal logits; equally deep accepted paths).

@@ -428,42 +428,53 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     }
 }
 
-// Finish: one block per row.  Slices that the streaming pass flagged are redone exactly; the S
-// ordered slice lists of the row are merged, the row is completed if it has fewer than k entries
-// above -inf, and written best first.  Rows that were not split and not flagged were already
-// written by the slice kernel: their block returns at once.
+// Finish.  Slices that the streaming pass flagged are redone exactly; the S ordered slice lists of
+// a row are merged, the row is completed if it has fewer than k entries above -inf, and written
+// best first.  Split rows (S > 1) get one block each.  Rows that were not split were already
+// written by the slice kernel unless they were flagged: a small grid looks through the flags, each
+// block at a contiguous range of rows, and usually finds nothing to do.
 template <int DT>
-__global__ void __launch_bounds__(kTkThreads) topk_finish_kernel(const TopkParams p)
+__global__ void __launch_bounds__(kTkThreads) topk_finish_kernel(const TopkParams p, long long rows,
+                                                                 int rows_per_block)
 {
     extern __shared__ Cand s_c[];
     __shared__ int s_found;
     pdl_launch_dependents();     // the next call's slice kernel may start streaming its rows
     const int k = p.k, S = p.S, n = S * k;
-    const long long row = blockIdx.x;
-    bool any_redo = false;
-    for (int sl = 0; sl < S; ++sl) any_redo |= p.redo[row * S + sl] != 0;      // block-uniform
-    if (S == 1 && !any_redo) return;
-    if (any_redo) {
-        for (int sl = 0; sl < S; ++sl)
-            if (p.redo[row * S + sl]) topk_slice_exact<DT>(p, row * S + sl);
-        __threadfence_block();
+    const long long r0 = (long long)blockIdx.x * rows_per_block;
+    const long long r1 = min(rows, r0 + rows_per_block);
+    if (S == 1) {
+        int mine = 0;
+        for (long long r = r0 + threadIdx.x; r < r1; r += blockDim.x) mine |= p.redo[r];
+        if (!__syncthreads_or(mine)) return;
+    }
+    for (long long row = r0; row < r1; ++row) {
+        bool any_redo = false;
+        for (int sl = 0; sl < S; ++sl) any_redo |= p.redo[row * S + sl] != 0;      // block-uniform
+        if (S == 1 && !any_redo) continue;
+        __syncthreads();             // shared arrays may still be in use from the previous row
+        if (any_redo) {
+            for (int sl = 0; sl < S; ++sl)
+                if (p.redo[row * S + sl]) topk_slice_exact<DT>(p, row * S + sl);
+            __threadfence_block();
+            __syncthreads();
+        }
+        const Cand *src = p.partial + (size_t)row * n;
+        if (threadIdx.x == 0) s_found = 0;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
         __syncthreads();
+        float *ov = p.out_val + (size_t)row * k;
+        int32_t *oi = p.out_id + (size_t)row * k;
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const Cand c = s_c[i];
+            if (c.id == kNoId) continue;
+            int rank = 0;
+            for (int j = 0; j < n; ++j) rank += (s_c[j].id != kNoId && beats(s_c[j].z, s_c[j].id, c.z, c.id)) ? 1 : 0;
+            if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && s_found < k) complete_row(ov, oi, s_found, k);
     }
-    const Cand *src = p.partial + (size_t)row * n;
-    if (threadIdx.x == 0) s_found = 0;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
-    __syncthreads();
-    float *ov = p.out_val + (size_t)row * k;
-    int32_t *oi = p.out_id + (size_t)row * k;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const Cand c = s_c[i];
-        if (c.id == kNoId) continue;
-        int rank = 0;
-        for (int j = 0; j < n; ++j) rank += (s_c[j].id != kNoId && beats(s_c[j].z, s_c[j].id, c.z, c.id)) ? 1 : 0;
-        if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
-    }
-    __syncthreads();
-    if (threadIdx.x == 0 && s_found < k) complete_row(ov, oi, s_found, k);
 }
 
 struct TkSplit { int S, L; };
@@ -535,8 +546,12 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
         if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
     }
     const size_t fsmem = (size_t)sp.S * k * sizeof(Cand);
-    if (dt == MARS_BF16) topk_finish_kernel<MARS_BF16><<<(unsigned)rows, kTkThreads, fsmem, st>>>(p);
-    else topk_finish_kernel<MARS_FP32><<<(unsigned)rows, kTkThreads, fsmem, st>>>(p);
+    const long long fgrid = (sp.S > 1 || rows < 148 * 2) ? rows : 148 * 2;
+    const int rows_per_block = (int)((rows + fgrid - 1) / fgrid);
+    if (dt == MARS_BF16)
+        topk_finish_kernel<MARS_BF16><<<(unsigned)fgrid, kTkThreads, fsmem, st>>>(p, (long long)rows, rows_per_block);
+    else
+        topk_finish_kernel<MARS_FP32><<<(unsigned)fgrid, kTkThreads, fsmem, st>>>(p, (long long)rows, rows_per_block);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 

@@ -423,3 +423,43 @@ def test_device_matches_what_the_launch_shapes_are_tuned_for():
     assert info["sm_tuned"] == 148
     assert info["sm_count"] == torch.cuda.get_device_properties(0).multi_processor_count
     assert (info["status"] == 0) == (info["sm_count"] == 148)
+
+
+@pytest.mark.parametrize("use_graph", [False, True])
+def test_back_to_back_calls_overlap_without_mixing_their_data(use_graph):
+    """Consecutive calls on one stream overlap on the GPU (the later one streams its logits while
+    the earlier one drains) and they share one workspace here.  Two different batches alternate,
+    forty calls in a row with nothing in between, directly and from a CUDA graph; every call's
+    outputs must be the oracle's for its own batch."""
+    ws = [synth.tree_workload("bb0", 48, 12, 4, 3, 50000, torch.bfloat16, DEV, 901, 0.9, 3.0, 15.0, 30.0, 0.3),
+          synth.tree_workload("bb1", 48, 12, 4, 3, 50000, torch.bfloat16, DEV, 902, 0.9, 3.0, 15.0, 30.0, 0.3)]
+    refs = [orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, w.theta) for w in ws]
+    toks = [torch.as_tensor(w.tok, device=DEV) for w in ws]
+    pars = [torch.as_tensor(w.parent, device=DEV) for w in ws]
+    n_calls = 40
+    outs = [mars.alloc_outputs(48, 12, 11, DEV, debug=True) for _ in range(n_calls)]
+    work = torch.zeros(mars.workspace_bytes(48, 12, 50000, mars.BF16), dtype=torch.uint8, device=DEV)
+
+    def run_all():
+        for i in range(n_calls):
+            j = i & 1
+            mars.verify_tree(ws[j].logits, toks[j], pars[j], 0.9, flags=mars.COUNTERS_ZERO, workspace=work,
+                             out=outs[i])
+
+    mars.verify_tree(ws[0].logits, toks[0], pars[0], 0.9, workspace=work)      # counters start at zero
+    torch.cuda.synchronize()
+    if use_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            run_all()
+        g.replay()
+        g.replay()
+    else:
+        run_all()
+    torch.cuda.synchronize()
+    for i in range(n_calls):
+        got = mars.to_host(outs[i])
+        assert_same(got, refs[i & 1], KEYS_TREE, f"call {i}")
+        assert np.array_equal(got["top2_val"].view(np.uint32), refs[i & 1]["top2_val"].view(np.uint32))

@@ -244,6 +244,36 @@ def test_repeated_calls_on_one_workspace():
             assert np.array_equal(first[k], again[k]), k
 
 
+def test_back_to_back_calls_overlap_without_mixing_their_data():
+    """A call's streaming kernel may start while the previous call's tail kernel still reads the
+    shared workspace; it must not write its records before that kernel is done.  Two different
+    batches alternate through one workspace, twenty calls with nothing in between; every call must
+    reproduce what the same batch gives when it runs alone."""
+    ws_ = [synth.tree_workload("sb0", 24, 20, 4, 3, 60000, torch.bfloat16, DEV, 911, 0.9, 3.0, 15.0, 30.0, 0.3),
+           synth.tree_workload("sb1", 24, 20, 4, 3, 60000, torch.bfloat16, DEV, 912, 0.9, 3.0, 15.0, 30.0, 0.3)]
+    us = [synth.make_uniforms(24, 20, 911), synth.make_uniforms(24, 20, 912)]
+    alone = [mars.to_host(mars.verify_tree_stochastic(w.logits, w.tok, w.parent, u, 0.9, 1.0, debug=True))
+             for w, u in zip(ws_, us)]
+    for j in (0, 1):        # and what runs alone agrees with the oracle
+        ref = orc.verify_tree_stochastic(synth.to_numpy_bits(ws_[j].logits), ws_[j].tok, ws_[j].parent, us[j], 0.9, 1.0)
+        compare(alone[j], ref, ws_[j].tok, ws_[j].parent, host_f64(ws_[j].logits), us[j], 1.0, f"alone {j}")
+    work = torch.empty(int(mars.lib().mars_stochastic_workspace_bytes(24, 20, 60000, mars.BF16)), dtype=torch.uint8,
+                       device=DEV)
+    toks = [torch.as_tensor(w.tok, device=DEV) for w in ws_]
+    pars = [torch.as_tensor(w.parent, device=DEV) for w in ws_]
+    ud = [torch.as_tensor(u, device=DEV) for u in us]
+    outs = [mars.alloc_stochastic_outputs(24, 20, 19, DEV, debug=True) for _ in range(20)]
+    for i in range(20):
+        j = i & 1
+        mars.verify_tree_stochastic(ws_[j].logits, toks[j], pars[j], ud[j], 0.9, 1.0, workspace=work, out=outs[i])
+    torch.cuda.synchronize()
+    for i in range(20):
+        got = mars.to_host(outs[i])
+        for k in ("accept_len", "out_tokens", "path_nodes", "out_len", "seq_status", "node_how"):
+            assert np.array_equal(got[k], alone[i & 1][k]), (i, k)
+        assert np.array_equal(got["node_prob"].view(np.uint32), alone[i & 1]["node_prob"].view(np.uint32)), i
+
+
 def test_plain_mode_preserves_the_target_distribution_on_the_gpu():
     """A property that needs no oracle: with Eq. 1 alone the first emitted token follows the
     root row's softmax, whatever the candidates are (20 000 sequences over one fixed tree)."""

@@ -88,3 +88,22 @@ def test_topk_whole_rows_that_defeat_the_floor(dtype):
     z[4] = torch.linspace(8, -8, V, device=DEV).to(dtype)
     check(z, k)
     check(z[:8], 32)
+
+
+def test_topk_back_to_back_calls_share_a_workspace():
+    """Consecutive top-k calls overlap on the GPU; alternating inputs through one workspace must
+    still give each call its own rows' answer."""
+    g = torch.Generator(device=DEV); g.manual_seed(5)
+    zs = [(torch.randn((300, 40000), generator=g, device=DEV) * 3).to(torch.bfloat16) for _ in range(2)]
+    want = [orc.topk(synth.to_numpy_bits(z), 10) for z in zs]
+    need = int(mars.lib().mars_topk_workspace_bytes(300, 40000, mars.BF16, 10))
+    work = torch.empty(need, dtype=torch.uint8, device=DEV)
+    outs = [(torch.empty((300, 10), dtype=torch.float32, device=DEV), torch.empty((300, 10), dtype=torch.int32, device=DEV))
+            for _ in range(30)]
+    for i in range(30):
+        mars.topk_rows(zs[i & 1], 10, workspace=work, out=outs[i])
+    torch.cuda.synchronize()
+    for i in range(30):
+        rv, ri = want[i & 1]
+        assert np.array_equal(outs[i][1].cpu().numpy(), ri), i
+        assert np.array_equal(outs[i][0].cpu().numpy().view(np.uint32), rv.view(np.uint32)), i
