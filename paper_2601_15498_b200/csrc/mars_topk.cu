@@ -404,7 +404,7 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
         scan(nfull * kBatchVecs + tid);
     }
     // Up to here only this call's logits were read; the workspace may still be in use by the
-    // previous call's merge kernel (see pdl_wait).
+    // previous call's finish kernel (see pdl_wait).
     pdl_wait();
     __syncthreads();
     if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_finish_kernel

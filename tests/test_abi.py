@@ -118,3 +118,11 @@ def test_device_check_reports_a_missing_device(lib):
     sm, tuned = ctypes.c_int(-1), ctypes.c_int(-1)
     assert lib.mars_device_check(ctypes.byref(sm), ctypes.byref(tuned)) == 4      # MARS_ERR_CUDA
     assert tuned.value == 148
+
+
+def test_binding_declares_every_exported_function(lib):
+    """The Python binding states argument and result types for every function of the header, so
+    that no call goes through ctypes' int-sized defaults (which would truncate 64-bit pointers)."""
+    for n in declared_functions():
+        fn = getattr(lib, n)
+        assert fn.argtypes is not None, n
