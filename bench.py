@@ -396,7 +396,9 @@ class VerifyCase:
         self.parent = torch.as_tensor(w.parent, device=dev)
         self.draft = torch.as_tensor(w.draft, device=dev)
         self.ws = torch.zeros(mars.workspace_bytes(w.B, w.N, w.V, self.dt_code), dtype=torch.uint8, device=dev)
-        self.flags = mars.COUNTERS_ZERO   # zeroed once; every call leaves its counters at zero
+        # workspace zeroed once and every call leaves its counters at zero; the logits are resident
+        # before any step starts, so a step may stream them while the previous one drains
+        self.flags = mars.COUNTERS_ZERO | mars.LOGITS_READY
         if T:
             self.uni_h = synth.make_uniforms(w.B, w.N, seed)
             self.uni = torch.as_tensor(self.uni_h, device=dev)
@@ -418,10 +420,11 @@ class VerifyCase:
         w, m = self.w, self.mars
         lg = self.logits[i % self.copies] if lg is None else lg
         if self.T and w.kind == "chain":
-            m.verify_chain_stochastic(lg, self.draft, self.uni, w.theta, self.T, workspace=self.ws_s, out=self.out)
+            m.verify_chain_stochastic(lg, self.draft, self.uni, w.theta, self.T, flags=m.LOGITS_READY,
+                                      workspace=self.ws_s, out=self.out)
         elif self.T:
-            m.verify_tree_stochastic(lg, self.tok, self.parent, self.uni, w.theta, self.T, workspace=self.ws_s,
-                                     out=self.out)
+            m.verify_tree_stochastic(lg, self.tok, self.parent, self.uni, w.theta, self.T, flags=m.LOGITS_READY,
+                                     workspace=self.ws_s, out=self.out)
         elif w.kind == "chain":
             m.verify_chain(lg, self.draft, w.theta, flags=self.flags, workspace=self.ws, out=self.out)
         else:
@@ -466,9 +469,9 @@ class VerifyCase:
                 "l2": ("inputs larger than L2" if self.copies == 1 else
                        f"rotating over {self.copies} input copies, {self.copies * w.logits_bytes} B > L2"),
                 "launch": launch,
-                "overlap": "consecutive calls on one stream overlap by programmatic dependent launch: a call "
-                           "streams its rows while the previous one drains, and waits for it before touching "
-                           "workspace or outputs",
+                "overlap": "MARS_LOGITS_READY: the logits are resident before the step, so a call streams its rows "
+                           "while the previous call on the stream drains (programmatic dependent launch) and "
+                           "waits for it before touching workspace or outputs",
                 "workspace": ("uninitialised (records only)" if T else
                               "zeroed once; MARS_COUNTERS_ZERO (counters reset by the kernel itself)"),
                 "parallelism": f"dp{world} (independent sequences, no collective)"}
@@ -549,7 +552,7 @@ class VocabShardCase:
 
     def step(self, i=0):
         m, w = self.mars, self.w
-        m.top2_shard(self.local, w.B, w.N, self.lo, V_local=self.hi - self.lo, flags=m.COUNTERS_ZERO,
+        m.top2_shard(self.local, w.B, w.N, self.lo, V_local=self.hi - self.lo, flags=m.COUNTERS_ZERO | m.LOGITS_READY,
                      workspace=self.ws, records=self.rec)
         if self.world > 1:
             import torch.distributed as dist

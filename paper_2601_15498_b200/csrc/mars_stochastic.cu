@@ -635,8 +635,8 @@ __global__ void __launch_bounds__(kTailThreads, MODE == 1 ? 1 : 2) stoch_tail_ke
     const int b = (int)(blockIdx.x / G);
     const int N = p.N, V = p.V, S = p.S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // The next call's streaming kernel may start reading its logits while this kernel runs; it
-    // waits for this kernel before it writes records.
+    // The next call's streaming kernel may be scheduled while this kernel runs (and, if its caller
+    // set MARS_LOGITS_READY, read its logits); it waits for this kernel before it writes records.
     pdl_launch_dependents();
 
     int32_t *s_id1 = reinterpret_cast<int32_t *>(smem_dyn);
@@ -911,6 +911,7 @@ struct StreamParams {
     int L;       // elements per slice (multiple of 16)
     float c;     // log2(e) / T
     SRec *partial;   // [R*S]
+    int early;   // MARS_LOGITS_READY: stream the logits before waiting for the predecessor
 };
 
 template <int DT, int U, int MINB>
@@ -921,6 +922,7 @@ __global__ void __launch_bounds__(kThreads, MINB) stoch_stream_kernel(const Stre
     __shared__ Rec s_warp[kThreads / 32];
     __shared__ float2 s_soft[kThreads / 32];
 
+    if (!p.early) pdl_wait();        // by default nothing is read before the predecessor is done
     const int tid = threadIdx.x;
     const long long blk = blockIdx.x;
     const long long row = blk / p.S;
@@ -1147,7 +1149,7 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     if (!chain && (!tok || !parent)) return MARS_ERR_INVALID_ARG;
     if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
     if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO |
-                  MARS_STOCH_PLAIN | MARS_STOCH_RELAX_ONLY))
+                  MARS_STOCH_PLAIN | MARS_STOCH_RELAX_ONLY | MARS_LOGITS_READY))
         return MARS_ERR_UNSUPPORTED;
     if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
     if ((flags & MARS_STOCH_PLAIN) && (flags & MARS_STOCH_RELAX_ONLY)) return MARS_ERR_INVALID_ARG;
@@ -1167,6 +1169,7 @@ static mars_status_t run_stochastic(const void *logits, int64_t ld, mars_dtype_t
     StreamParams sp1;
     sp1.logits = logits; sp1.ld = ld; sp1.V = V; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
     sp1.partial = (SRec *)workspace;
+    sp1.early = (flags & MARS_LOGITS_READY) ? 1 : 0;
     const unsigned grid = (unsigned)(R * sp.S);
     // 4 vectors per batch in two register buffers, 4 blocks per SM (64 registers): measured
     // best for both dtypes; 5 or 6 blocks per SM spill the second buffer and run at half speed,
@@ -1288,7 +1291,7 @@ mars_status_t mars_stochastic_shard_records(const void *logits_local, int64_t ld
         return MARS_ERR_INVALID_ARG;
     if (ld < V_local || id_offset < 0 || ((uintptr_t)records & 15)) return MARS_ERR_INVALID_ARG;
     if (!(temperature > 0.0f) || !(temperature < INFINITY)) return MARS_ERR_INVALID_ARG;
-    if (flags & ~MARS_SHARED_PARENT) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_SHARED_PARENT | MARS_LOGITS_READY)) return MARS_ERR_UNSUPPORTED;
     if (!stoch_sizes_supported(B, N, V_local, (int)dt)) return MARS_ERR_UNSUPPORTED;
     if ((uintptr_t)logits_local % (dt == MARS_BF16 ? 2 : 4)) return MARS_ERR_INVALID_ARG;
     const double cd = 1.4426950408889634074 / (double)temperature;
@@ -1301,6 +1304,7 @@ mars_status_t mars_stochastic_shard_records(const void *logits_local, int64_t ld
     StreamParams sp1;
     sp1.logits = logits_local; sp1.ld = ld; sp1.V = V_local; sp1.S = sp.S; sp1.L = sp.L; sp1.c = (float)cd;
     sp1.partial = (SRec *)workspace;
+    sp1.early = (flags & MARS_LOGITS_READY) ? 1 : 0;
     const unsigned grid = (unsigned)(R * sp.S);
     {
         const bool overlap = hook(kHookNoOverlap) == 0;

@@ -29,10 +29,12 @@ __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
 // Programmatic dependent launch (back-to-back calls on one stream).  A kernel that is launched
 // with programmatic stream serialisation may begin while its predecessor still runs, provided
 // the predecessor lets it: pdl_launch_dependents() does that, and is a no-op otherwise.  Such a
-// kernel must call pdl_wait() before its first access to memory that the predecessor may write
-// or still read-modify (here: workspaces and outputs; logits and other inputs are only read);
-// it returns once the predecessor has completed and its writes are visible.  Without the launch
-// attribute, or without a predecessor that triggers early, both calls do nothing.
+// kernel must call pdl_wait() before its first access to anything the predecessor may produce or
+// still use; it returns once the predecessor has completed and its writes are visible.  The
+// streaming kernels wait first thing, unless the caller vouched (MARS_LOGITS_READY) that the
+// logits do not come from the predecessor: then only workspaces and outputs are at stake, and the
+// wait moves behind the streaming loop.  Without the launch attribute, or without a predecessor
+// that triggers early, both calls do nothing.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

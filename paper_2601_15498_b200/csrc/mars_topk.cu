@@ -273,6 +273,7 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     constexpr int kBatchVecs = kTkThreads * kTkU;
     const int nfull = nvec / kBatchVecs;
 
+    pdl_wait();     // scheduled early (behind the previous call's finish kernel), reads nothing before it is done
     uint4 v[kTkU];
     typename E::packed_t q[kTkU];
     // batch 0: issue its loads first, so that the set-up below overlaps their latency
@@ -403,9 +404,6 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
         bm = load_batch<DT, kTkU, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
         scan(nfull * kBatchVecs + tid);
     }
-    // Up to here only this call's logits were read; the workspace may still be in use by the
-    // previous call's finish kernel (see pdl_wait).
-    pdl_wait();
     __syncthreads();
     if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_finish_kernel
     if (s_overflow) return;
@@ -439,7 +437,7 @@ __global__ void __launch_bounds__(kTkThreads) topk_finish_kernel(const TopkParam
 {
     extern __shared__ Cand s_c[];
     __shared__ int s_found;
-    pdl_launch_dependents();     // the next call's slice kernel may start streaming its rows
+    pdl_launch_dependents();     // the next call's slice kernel may be scheduled (it waits for this one)
     const int k = p.k, S = p.S, n = S * k;
     const long long r0 = (long long)blockIdx.x * rows_per_block;
     const long long r1 = min(rows, r0 + rows_per_block);

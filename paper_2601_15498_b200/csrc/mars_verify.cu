@@ -43,6 +43,7 @@ struct Params {
     unsigned *counters;  // [B]
     Rec *shard_out;      // non-null: emit merged per-row records [B*N] instead of verifying
     int id_offset;       // ... with this offset added to the token ids (vocabulary shard)
+    int early;           // MARS_LOGITS_READY: stream the logits before waiting for the predecessor
     int stage_partials;  // last block copies the sequence's N*S records to shared memory first
     int tail_smem_off;   // byte offset of that staging area in dynamic shared memory
     TailArgs tail;
@@ -57,9 +58,12 @@ __global__ void __launch_bounds__(kThreads, MINB) verify_kernel(const Params p)
     __shared__ Rec s_warp[kThreads / 32];
     __shared__ int s_last;
 
-    // The next call on this stream may start streaming its rows while this one drains: until
-    // its pdl_wait() it only reads its inputs.
+    // The next call on this stream may be scheduled while this one drains.  This call itself
+    // waits for its predecessor right here unless the caller vouched that the logits do not come
+    // from it (MARS_LOGITS_READY); then the wait moves to the point where the workspace is first
+    // touched.
     pdl_launch_dependents();
+    if (!p.early) pdl_wait();
     const int tid = threadIdx.x;
     const long long blk = blockIdx.x;
     const long long row = blk / p.S;
@@ -216,7 +220,7 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
         if (chain && N > 1 && !tok) return MARS_ERR_INVALID_ARG;
     }
     if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_COUNTERS_ZERO | MARS_RULE_MARGIN |
-                  MARS_RULE_PROB_RATIO))
+                  MARS_RULE_PROB_RATIO | MARS_LOGITS_READY))
         return MARS_ERR_UNSUPPORTED;
     if ((flags & MARS_RULE_MARGIN) && (flags & MARS_RULE_PROB_RATIO)) return MARS_ERR_INVALID_ARG;
     rule_threshold(&theta, &flags);
@@ -234,6 +238,7 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     p.counters = (unsigned *)workspace;
     p.partial = (Rec *)((char *)workspace + counters_bytes(B));
     p.shard_out = shard_out; p.id_offset = id_offset;
+    p.early = (flags & MARS_LOGITS_READY) ? 1 : 0;
     p.tail.tok = tok; p.tail.parent = parent;
     p.tail.accept_len = accept_len; p.tail.out_tokens = out_tokens; p.tail.path_nodes = path_nodes;
     p.tail.out_len = out_len; p.tail.seq_status = seq_status;
@@ -363,7 +368,7 @@ mars_status_t mars_top2_shard(const void *logits, int64_t ld, mars_dtype_t dt, i
                               size_t workspace_bytes, void *cuda_stream)
 {
     if (!records || ((uintptr_t)records & 15) || id_offset < 0) return MARS_ERR_INVALID_ARG;
-    if (flags & ~MARS_COUNTERS_ZERO) return MARS_ERR_UNSUPPORTED;
+    if (flags & ~(MARS_COUNTERS_ZERO | MARS_LOGITS_READY)) return MARS_ERR_UNSUPPORTED;
     return mars::run(logits, ld, dt, nullptr, nullptr, 0, B, N, V_local, 0.0f, flags, nullptr, nullptr,
                      nullptr, nullptr, 0, nullptr, nullptr, workspace, workspace_bytes, cuda_stream,
                      (mars::Rec *)records, id_offset);

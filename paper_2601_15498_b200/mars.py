@@ -17,6 +17,7 @@ from . import build as _build
 BF16, FP32 = 0, 1
 SIGN_LITERAL, SHARED_PARENT, COUNTERS_ZERO, RULE_MARGIN, RULE_PROB_RATIO = 1, 2, 4, 8, 16
 STOCH_PLAIN, STOCH_RELAX_ONLY = 32, 64
+LOGITS_READY = 128
 MAX_NODES = 1024
 
 _lock = threading.Lock()

@@ -74,7 +74,7 @@ def test_argument_checks_return_before_any_cuda_call(lib):
     assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, float("nan"), 0, dummy, dummy, dummy,
                                  n, None, dummy, 1 << 20, n) == 1
     # unknown flag / too many nodes / unknown dtype
-    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 128, dummy, dummy, dummy, n, None,
+    assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2, 10, 0.9, 1024, dummy, dummy, dummy, n, None,
                                  dummy, 1 << 20, n) == 3
     assert lib.mars_verify_chain(dummy, 10, 0, dummy, 1, 2000, 10, 0.9, 0, dummy, dummy, dummy, n, None,
                                  dummy, 1 << 20, n) == 3

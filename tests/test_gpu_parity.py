@@ -425,10 +425,12 @@ def test_device_matches_what_the_launch_shapes_are_tuned_for():
     assert (info["status"] == 0) == (info["sm_count"] == 148)
 
 
+@pytest.mark.parametrize("early", [False, True])
 @pytest.mark.parametrize("use_graph", [False, True])
-def test_back_to_back_calls_overlap_without_mixing_their_data(use_graph):
-    """Consecutive calls on one stream overlap on the GPU (the later one streams its logits while
-    the earlier one drains) and they share one workspace here.  Two different batches alternate,
+def test_back_to_back_calls_overlap_without_mixing_their_data(use_graph, early):
+    """With MARS_LOGITS_READY consecutive calls on one stream overlap on the GPU (the later one
+    streams its logits while the earlier one drains), without it only their launches do; they
+    share one workspace here.  Two different batches alternate,
     forty calls in a row with nothing in between, directly and from a CUDA graph; every call's
     outputs must be the oracle's for its own batch."""
     ws = [synth.tree_workload("bb0", 48, 12, 4, 3, 50000, torch.bfloat16, DEV, 901, 0.9, 3.0, 15.0, 30.0, 0.3),
@@ -443,8 +445,8 @@ def test_back_to_back_calls_overlap_without_mixing_their_data(use_graph):
     def run_all():
         for i in range(n_calls):
             j = i & 1
-            mars.verify_tree(ws[j].logits, toks[j], pars[j], 0.9, flags=mars.COUNTERS_ZERO, workspace=work,
-                             out=outs[i])
+            mars.verify_tree(ws[j].logits, toks[j], pars[j], 0.9,
+                             flags=mars.COUNTERS_ZERO | (mars.LOGITS_READY if early else 0), workspace=work, out=outs[i])
 
     mars.verify_tree(ws[0].logits, toks[0], pars[0], 0.9, workspace=work)      # counters start at zero
     torch.cuda.synchronize()

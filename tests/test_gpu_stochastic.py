@@ -265,7 +265,8 @@ def test_back_to_back_calls_overlap_without_mixing_their_data():
     outs = [mars.alloc_stochastic_outputs(24, 20, 19, DEV, debug=True) for _ in range(20)]
     for i in range(20):
         j = i & 1
-        mars.verify_tree_stochastic(ws_[j].logits, toks[j], pars[j], ud[j], 0.9, 1.0, workspace=work, out=outs[i])
+        mars.verify_tree_stochastic(ws_[j].logits, toks[j], pars[j], ud[j], 0.9, 1.0,
+                                    flags=(mars.LOGITS_READY if i % 4 < 2 else 0), workspace=work, out=outs[i])
     torch.cuda.synchronize()
     for i in range(20):
         got = mars.to_host(outs[i])
