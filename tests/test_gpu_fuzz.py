@@ -176,3 +176,53 @@ def test_sharded_stochastic_tree(seed, monkeypatch):
         for o in outs:
             ts.compare(o, ref, c["tok"], c["parent"], c["z"].double().numpy(), u, T, f"fuzz sharded {seed}",
                        max_close_frac=0.25)
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_topk_rows(seed):
+    """Exact top-k against the oracle over random shapes, k, dtypes, value patterns that stress
+    the floor and the queue (ties, sorted rows, constant rows, NaN / +-inf / +-0, a heavy second
+    half), unaligned padded views and forced row splits; a second call must repeat the first."""
+    rng = np.random.default_rng(7000 + seed)
+    for _ in range(4):
+        V = int(rng.choice([int(rng.integers(1, 300)), int(rng.integers(300, 20000)), int(rng.integers(20000, 160000))]))
+        k = int(min(V, rng.choice([1, 2, 3, 7, 10, 16, 31, 32])))
+        rows = int(max(1, min(rng.choice([1, 3, 17, 200, 700]), 12_000_000 // V)))
+        dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+        kind = str(rng.choice(["normal", "ties", "asc", "desc", "const", "special", "blocks"]))
+        g = torch.Generator(device=DEV)
+        g.manual_seed(int(rng.integers(1 << 30)))
+        z = torch.randn((rows, V), generator=g, device=DEV) * 3
+        if kind == "ties":
+            z = torch.round(z)
+        elif kind == "asc":
+            z = torch.sort(z, dim=1).values
+        elif kind == "desc":
+            z = torch.sort(z, dim=1, descending=True).values
+        elif kind == "const":
+            z[:] = 1.5
+        elif kind == "special":
+            m = torch.rand((rows, V), generator=g, device=DEV)
+            z[m < 0.01] = float("nan")
+            z[(m > 0.01) & (m < 0.02)] = float("-inf")
+            z[(m > 0.02) & (m < 0.021)] = float("inf")
+            z[m > 0.9] = 0.0
+            z[(m > 0.8) & (m < 0.9)] = -0.0
+        elif kind == "blocks":
+            z[:, V // 2:] += 10
+        if rng.random() < 0.3 and V > 16:
+            big = torch.full((rows, V + 13), 3e38, dtype=dtype, device=DEV)
+            zz = big[:, 5:5 + V]
+            zz.copy_(z.to(dtype))
+        else:
+            zz = z.to(dtype)
+        hooks.set("HOOK_FORCE_SPLIT", int(rng.choice([0, 0, 0, 2, 5])))
+        val, idx = mars.topk_rows(zz, k)
+        val2, idx2 = mars.topk_rows(zz, k)
+        torch.cuda.synchronize()
+        hooks.clear("HOOK_FORCE_SPLIT")
+        rv, ri = orc.topk(synth.to_numpy_bits(zz.contiguous()), k)
+        what = (V, k, rows, str(dtype), kind)
+        assert np.array_equal(idx.cpu().numpy(), ri), what
+        assert np.array_equal(val.cpu().numpy().view(np.uint32), rv.view(np.uint32)), what
+        assert torch.equal(idx, idx2) and torch.equal(val.view(torch.int32), val2.view(torch.int32)), what
