@@ -1082,7 +1082,10 @@ def main():
     # ---- this GPU's read-only ceiling on the same bytes: the library's streaming probe ----
     probe = c.probe() if w.logits.is_contiguous() else None
 
-    # ---- end to end: host buffers in, results out, copies inside the timed region ----
+    # ---- end to end: host buffers in, results out, copies inside the timed region.  The
+    # deterministic path goes through the library's host-buffer entry point (one C-ABI call does the
+    # copies in, the kernel and the copies out); the stochastic path copies with torch around the
+    # device-buffer call ----
     e2e = None
     h_logits = None
     if args.e2e_steps > 0:
@@ -1091,24 +1094,36 @@ def main():
         h_tok = torch.as_tensor(w.tok).pin_memory()
         h_par = torch.as_tensor(w.parent).pin_memory()
         h_uni = torch.as_tensor(c.uni_h).pin_memory() if T else None
-        h_out = {k: torch.empty(c.out[k].shape, dtype=c.out[k].dtype, pin_memory=True)
-                 for k in ("accept_len", "out_tokens", "out_len")}
-        d_logits = torch.empty_like(w.logits)
+        if T:
+            h_out = {k: torch.empty(c.out[k].shape, dtype=c.out[k].dtype, pin_memory=True)
+                     for k in ("accept_len", "out_tokens", "out_len")}
+            d_logits = torch.empty_like(w.logits)
 
-        def e2e_step():
-            d_logits.copy_(h_logits, non_blocking=True)
-            c.tok.copy_(h_tok, non_blocking=True)
-            c.parent.copy_(h_par, non_blocking=True)
-            if T:
+            def e2e_step():
+                d_logits.copy_(h_logits, non_blocking=True)
+                c.tok.copy_(h_tok, non_blocking=True)
+                c.parent.copy_(h_par, non_blocking=True)
                 c.uni.copy_(h_uni, non_blocking=True)
-            if w.kind == "chain":
-                c.draft.copy_(c.tok[:, 1:])
-            c.step(0, d_logits)
-            for k, h in h_out.items():
-                h.copy_(c.out[k], non_blocking=True)
+                if w.kind == "chain":
+                    c.draft.copy_(c.tok[:, 1:])
+                c.step(0, d_logits)
+                for k, h in h_out.items():
+                    h.copy_(c.out[k], non_blocking=True)
+            api = "torch copies around mars_verify_*_stochastic"
+        else:
+            h_out = mars.alloc_host_outputs(w.B, w.N - 1)
+            staging = torch.empty(int(mars.lib().mars_verify_tree_host_staging_bytes(
+                w.B, w.N, w.V, c.dt_code, w.logits.shape[1], w.N - 1)), dtype=torch.uint8, device=dev)
+
+            def e2e_step():
+                mars.verify_tree_host(h_logits, h_tok, h_par, w.theta, staging, h_out, V=w.V)
+            api = "mars_verify_tree_host (copies in, kernel, copies out in one C-ABI call; chains as linear trees)"
 
         e2e_step()
         torch.cuda.synchronize()
+        if not T:        # the host-buffer call must give what the device-buffer call gave
+            for k in ("accept_len", "out_len"):
+                assert np.array_equal(h_out[k].numpy(), timed_out[k]), k
         barrier(world)
         f0, f1 = ev(), ev()
         f0.record()
@@ -1120,8 +1135,11 @@ def main():
         h2d = w.logits_bytes + h_tok.numel() * 4 + h_par.numel() * 4 + (h_uni.numel() * 4 if T else 0)
         d2h = sum(h.numel() * h.element_size() for h in h_out.values())
         e2e = {"value": e2e_units / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps}
-        del d_logits
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps, "api": api}
+        if T:
+            del d_logits
+        else:
+            del staging
 
     if rank != 0:
         if world > 1:

@@ -173,6 +173,35 @@ mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * mars_verify_tree for inputs and outputs that live in HOST memory (the form a caller uses when
+ * the logits were not produced on this GPU).  Same rule, outputs and statuses as
+ * mars_verify_tree (Sec. 3.4 of the paper; chains are trees with parent[i] = i - 1).  The call
+ * enqueues, on `cuda_stream` and in this order: the copies of logits, tokens and parents into the
+ * caller's device staging buffer, the verification kernel, and the copies of the results back to
+ * the host pointers.  It allocates nothing and does not synchronise: the host buffers must stay
+ * valid, and the results are there, once the stream has passed that point.  Pinned host memory
+ * makes the copies asynchronous; pageable memory works and is slower.  The step is bound by the
+ * host link: B*N*ld*sizeof(elem) bytes cross it per call.
+ *
+ *   logits_host [B*N, ld]; tok_host [B, N]; parent_host [B, N] ([N] with MARS_SHARED_PARENT)
+ *   accept_len_host [B], out_tokens_host [B, Dcap+1], out_len_host [B]        required
+ *   path_nodes_host [B, Dcap+1], seq_status_host [B]                          may be NULL
+ *   staging      device memory, 256-byte aligned, at least
+ *                mars_verify_tree_host_staging_bytes(B, N, V, dt, ld, Dcap) bytes (holds the
+ *                device copies of all of the above plus the workspace); contents need not be
+ *                initialised; two calls that may overlap need separate staging buffers.
+ *   flags        MARS_SIGN_LITERAL, MARS_SHARED_PARENT, MARS_RULE_*.
+ * The size query returns 0 for unsupported sizes (host function, no CUDA call).
+ */
+size_t mars_verify_tree_host_staging_bytes(int B, int N, int V, mars_dtype_t dt, int64_t ld, int Dcap);
+mars_status_t mars_verify_tree_host(const void *logits_host, int64_t ld, mars_dtype_t dt,
+                                    const int32_t *tok_host, const int32_t *parent_host, int B, int N,
+                                    int V, float theta, uint32_t flags, int32_t *accept_len_host,
+                                    int32_t *out_tokens_host, int32_t *path_nodes_host,
+                                    int32_t *out_len_host, int Dcap, int32_t *seq_status_host,
+                                    void *staging, size_t staging_bytes, void *cuda_stream);
+
+/*
  * Bytes of workspace (device memory, 256-byte aligned) for mars_lmhead_verify with these
  * sizes.  Host function, no CUDA call.  Returns 0 for unsupported sizes (d must be a
  * multiple of 64).  Contents need not be initialised or preserved.

@@ -306,6 +306,88 @@ mars_status_t mars_verify_tree(const void *logits, int64_t ld, mars_dtype_t dt, 
                      path_nodes, out_len, Dcap, seq_status, dbg, workspace, workspace_bytes, cuda_stream);
 }
 
+// ---- host-buffer form: copies in, verification, copies out, all on the caller's stream --------
+
+namespace mars {
+struct HostStaging {       // byte offsets into the device staging buffer, each 256-byte aligned
+    size_t logits, tok, parent, accept_len, out_tokens, path_nodes, out_len, seq_status, workspace, total;
+    size_t logits_bytes, tok_bytes, parent_bytes, per_seq_bytes, path_bytes, workspace_bytes;
+};
+
+static bool host_staging_layout(int B, int N, int V, int dt, long long ld, int Dcap, bool shared_parent,
+                                HostStaging *h)
+{
+    if (!sizes_supported(B, N, V, dt) || ld < V || Dcap < 0 || Dcap > MARS_MAX_NODES) return false;
+    const size_t es = dt == MARS_BF16 ? 2 : 4;
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    h->logits_bytes = (size_t)B * N * (size_t)ld * es;
+    h->tok_bytes = (size_t)B * N * sizeof(int32_t);
+    h->parent_bytes = shared_parent ? (size_t)N * sizeof(int32_t) : h->tok_bytes;
+    h->per_seq_bytes = (size_t)B * sizeof(int32_t);
+    h->path_bytes = (size_t)B * (Dcap + 1) * sizeof(int32_t);
+    const Split sp = choose_split((long long)B * N, V, dt);
+    h->workspace_bytes = counters_bytes(B) + (size_t)B * N * sp.S * sizeof(Rec);
+    size_t o = 0;
+    h->logits = o; o += up(h->logits_bytes);
+    h->tok = o; o += up(h->tok_bytes);
+    h->parent = o; o += up(h->tok_bytes);            // room for per-sequence parents either way
+    h->accept_len = o; o += up(h->per_seq_bytes);
+    h->out_tokens = o; o += up(h->path_bytes);
+    h->path_nodes = o; o += up(h->path_bytes);
+    h->out_len = o; o += up(h->per_seq_bytes);
+    h->seq_status = o; o += up(h->per_seq_bytes);
+    h->workspace = o; o += up(h->workspace_bytes);
+    h->total = o;
+    return true;
+}
+}  // namespace mars
+
+size_t mars_verify_tree_host_staging_bytes(int B, int N, int V, mars_dtype_t dt, int64_t ld, int Dcap)
+{
+    mars::HostStaging h;
+    return mars::host_staging_layout(B, N, V, (int)dt, ld, Dcap, false, &h) ? h.total : 0;
+}
+
+mars_status_t mars_verify_tree_host(const void *logits_host, int64_t ld, mars_dtype_t dt, const int32_t *tok_host,
+                                    const int32_t *parent_host, int B, int N, int V, float theta, uint32_t flags,
+                                    int32_t *accept_len_host, int32_t *out_tokens_host, int32_t *path_nodes_host,
+                                    int32_t *out_len_host, int Dcap, int32_t *seq_status_host, void *staging,
+                                    size_t staging_bytes, void *cuda_stream)
+{
+    if (!logits_host || !tok_host || !parent_host || !accept_len_host || !out_tokens_host || !out_len_host)
+        return MARS_ERR_INVALID_ARG;
+    if (B < 1 || N < 1 || V < 2 || ld < V || Dcap < 0 || theta != theta) return MARS_ERR_INVALID_ARG;
+    if (flags & ~(MARS_SIGN_LITERAL | MARS_SHARED_PARENT | MARS_RULE_MARGIN | MARS_RULE_PROB_RATIO))
+        return MARS_ERR_UNSUPPORTED;
+    mars::HostStaging h;
+    if (!mars::host_staging_layout(B, N, V, (int)dt, ld, Dcap, (flags & MARS_SHARED_PARENT) != 0, &h))
+        return MARS_ERR_UNSUPPORTED;
+    if (!staging || ((uintptr_t)staging & 255) || staging_bytes < h.total) return MARS_ERR_WORKSPACE;
+    char *d = (char *)staging;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(d + h.logits, logits_host, h.logits_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d + h.tok, tok_host, h.tok_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d + h.parent, parent_host, h.parent_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return MARS_ERR_CUDA;
+    }
+    // the staging buffer's workspace is not known to be clean: the counters are cleared on the stream
+    const mars_status_t rs = mars::run(d + h.logits, ld, dt, (const int32_t *)(d + h.tok), (const int32_t *)(d + h.parent), 0,
+                                       B, N, V, theta, flags, (int32_t *)(d + h.accept_len), (int32_t *)(d + h.out_tokens),
+                                       (int32_t *)(d + h.path_nodes), (int32_t *)(d + h.out_len), Dcap,
+                                       (int32_t *)(d + h.seq_status), nullptr, d + h.workspace, h.workspace_bytes, st);
+    if (rs != MARS_OK) return rs;
+    bool ok = cudaMemcpyAsync(accept_len_host, d + h.accept_len, h.per_seq_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out_tokens_host, d + h.out_tokens, h.path_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(out_len_host, d + h.out_len, h.per_seq_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (path_nodes_host)
+        ok = ok && cudaMemcpyAsync(path_nodes_host, d + h.path_nodes, h.path_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (seq_status_host)
+        ok = ok && cudaMemcpyAsync(seq_status_host, d + h.seq_status, h.per_seq_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    return MARS_OK;
+}
+
 // ---- verification without any caller-provided or allocated scratch -------------------------
 //
 // Scratch for mars_verify_tree_static lives in this fixed device array.  Every GPU that loads

@@ -101,6 +101,11 @@ def lib() -> ctypes.CDLL:
             L.mars_selftest_stream_read.restype = i32
             L.mars_status_string.argtypes = [i32]
             L.mars_status_string.restype = ctypes.c_char_p
+            L.mars_verify_tree_host_staging_bytes.argtypes = [i32, i32, i32, i32, i64, i32]
+            L.mars_verify_tree_host_staging_bytes.restype = sz
+            L.mars_verify_tree_host.argtypes = [vp, i64, i32, vp, vp, i32, i32, i32, f32, u32, vp, vp, vp, vp, i32,
+                                                vp, vp, sz, vp]
+            L.mars_verify_tree_host.restype = i32
             L.mars_test_hook.argtypes = [i32, i32]
             L.mars_test_hook.restype = i32
             L.mars_device_check.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32)]
@@ -235,6 +240,46 @@ def verify_tree_static(logits: torch.Tensor, tok: torch.Tensor, parent: torch.Te
             out["seq_status"].data_ptr(), ctypes.byref(dbg) if dbg is not None else None, _stream())
     _check(code, "mars_verify_tree_static")
     return out
+
+
+def alloc_host_outputs(B: int, Dcap: int) -> dict:
+    """Pinned host buffers for the results of ``verify_tree_host``."""
+    def full(shape):
+        return torch.full(shape, -777, dtype=torch.int32).pin_memory()
+    return {"accept_len": full((B,)), "out_tokens": full((B, Dcap + 1)), "path_nodes": full((B, Dcap + 1)),
+            "out_len": full((B,)), "seq_status": full((B,))}
+
+
+def verify_tree_host(logits_host: torch.Tensor, tok_host: torch.Tensor, parent_host: torch.Tensor, theta: float,
+                     staging: torch.Tensor, out_host: dict, flags: int = 0, Dcap: int | None = None,
+                     V: int | None = None) -> dict:
+    """mars_verify_tree_host on the current stream of `staging`'s device: every input and output is a
+    HOST tensor (pinned for asynchronous copies), `staging` a uint8 device tensor of at least
+    ``mars_verify_tree_host_staging_bytes`` bytes.  Results are valid once the stream has passed."""
+    for t in (logits_host, tok_host, parent_host, *out_host.values()):
+        if t.is_cuda or not t.is_contiguous():
+            raise MarsError("inputs and outputs of verify_tree_host are contiguous host tensors")
+    if tok_host.dtype != torch.int32 or parent_host.dtype != torch.int32:
+        raise MarsError("tok and parent must be int32")
+    B, N = tok_host.shape
+    if parent_host.dim() == 1:
+        flags |= SHARED_PARENT
+    dt = _dtype_code(logits_host)
+    if logits_host.dim() != 2 or logits_host.shape[0] != B * N:
+        raise MarsError("logits must be [B*N, ld]")
+    ld = logits_host.shape[1]
+    V = ld if V is None else int(V)
+    Dcap = N - 1 if Dcap is None else int(Dcap)
+    with torch.cuda.device(staging.device):
+        code = lib().mars_verify_tree_host(
+            logits_host.data_ptr(), ld, dt, tok_host.data_ptr(), parent_host.data_ptr(), B, N, V, float(theta), flags,
+            out_host["accept_len"].data_ptr(), out_host["out_tokens"].data_ptr(),
+            out_host["path_nodes"].data_ptr() if "path_nodes" in out_host else None,
+            out_host["out_len"].data_ptr(),
+            Dcap, out_host["seq_status"].data_ptr() if "seq_status" in out_host else None,
+            staging.data_ptr(), staging.numel(), _stream())
+    _check(code, "mars_verify_tree_host")
+    return out_host
 
 
 def verify_chain(logits: torch.Tensor, draft, theta: float, flags: int = 0, V: int | None = None,

@@ -126,3 +126,19 @@ def test_binding_declares_every_exported_function(lib):
     for n in declared_functions():
         fn = getattr(lib, n)
         assert fn.argtypes is not None, n
+
+
+def test_host_buffer_entry_point_checks_its_arguments_on_the_host(lib):
+    n = None
+    p = ctypes.c_void_p(4096)
+    size = lib.mars_verify_tree_host_staging_bytes
+    assert size(0, 3, 100, 0, 100, 2) == 0 and size(2, 3, 100, 0, 50, 2) == 0 and size(2, 3, 100, 7, 100, 2) == 0
+    need = size(2, 3, 100, 1, 104, 2)
+    # logits 2*3*104*4 B, tokens and parents, five result arrays, workspace: each rounded up to 256 B
+    assert need % 256 == 0 and need >= 2 * 3 * 104 * 4 + lib.mars_workspace_bytes(2, 3, 100, 1)
+    call = lib.mars_verify_tree_host
+    assert call(n, 104, 1, p, p, 2, 3, 100, 0.9, 0, p, p, n, p, 2, n, p, need, n) == 1          # NULL logits
+    assert call(p, 104, 1, p, p, 2, 3, 100, float("nan"), 0, p, p, n, p, 2, n, p, need, n) == 1  # NaN theta
+    assert call(p, 104, 1, p, p, 2, 3, 100, 0.9, 4, p, p, n, p, 2, n, p, need, n) == 3            # flag not taken here
+    assert call(p, 104, 1, p, p, 2, 3, 100, 0.9, 0, p, p, n, p, 2, n, p, need - 1, n) == 2        # staging too small
+    assert call(p, 104, 1, p, p, 2, 3, 100, 0.9, 0, p, p, n, p, 2, n, ctypes.c_void_p(4100), need, n) == 2

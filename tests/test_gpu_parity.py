@@ -465,3 +465,29 @@ def test_back_to_back_calls_overlap_without_mixing_their_data(use_graph, early):
         got = mars.to_host(outs[i])
         assert_same(got, refs[i & 1], KEYS_TREE, f"call {i}")
         assert np.array_equal(got["top2_val"].view(np.uint32), refs[i & 1]["top2_val"].view(np.uint32))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_host_buffer_entry_point(dtype):
+    """mars_verify_tree_host: inputs and outputs in (pinned) host memory, one call does the copies
+    in, the verification and the copies out; results are the oracle's, twice in a row on one
+    staging buffer, with and without the optional outputs, and for a padded row stride."""
+    w = synth.tree_workload("hb", 9, 21, 4, 3, 30011, dtype, "cpu", 931, 0.9, 3.0, 15.0, 30.0, 0.3, ld=30016)
+    ref = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, w.theta, V=w.V)
+    lg = w.logits.pin_memory()
+    tok, par = torch.as_tensor(w.tok).pin_memory(), torch.as_tensor(w.parent).pin_memory()
+    code = mars.BF16 if dtype == torch.bfloat16 else mars.FP32
+    need = int(mars.lib().mars_verify_tree_host_staging_bytes(w.B, w.N, w.V, code, 30016, w.N - 1))
+    assert need > w.logits.numel() * w.logits.element_size()
+    staging = torch.full((need,), 0xCD, dtype=torch.uint8, device=DEV)
+    for rep in range(2):
+        out = mars.alloc_host_outputs(w.B, w.N - 1)
+        if rep == 1:
+            del out["path_nodes"], out["seq_status"]
+        mars.verify_tree_host(lg, tok, par, w.theta, staging, out, V=w.V)
+        torch.cuda.synchronize()
+        for k, v in out.items():
+            assert np.array_equal(v.numpy(), ref[k]), (rep, k)
+    small = torch.empty(need - 256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(mars.MarsError, match="workspace"):
+        mars.verify_tree_host(lg, tok, par, w.theta, small, mars.alloc_host_outputs(w.B, w.N - 1), V=w.V)
