@@ -389,8 +389,8 @@ class VerifyCase:
             self.w = w = WORKLOADS[key](dev, seed, batch) if batch else WORKLOADS[key](dev, seed)
         self.dt_code = mars.BF16 if w.logits.dtype == torch.bfloat16 else mars.FP32
         self.copies = 1
-        if w.logits_bytes < 3 * L2_BYTES:
-            self.copies = -(-3 * L2_BYTES // w.logits_bytes)
+        if w.logits_bytes < 3 * L2_BYTES:       # at least 8 copies, and more than 3 x L2 in total
+            self.copies = max(8, -(-3 * L2_BYTES // w.logits_bytes))
         self.logits = [w.logits] + [w.logits.clone() for _ in range(self.copies - 1)]
         self.tok = torch.as_tensor(w.tok, device=dev)
         self.parent = torch.as_tensor(w.parent, device=dev)
