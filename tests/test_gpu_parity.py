@@ -491,3 +491,30 @@ def test_host_buffer_entry_point(dtype):
     small = torch.empty(need - 256, dtype=torch.uint8, device=DEV)
     with pytest.raises(mars.MarsError, match="workspace"):
         mars.verify_tree_host(lg, tok, par, w.theta, small, mars.alloc_host_outputs(w.B, w.N - 1), V=w.V)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_very_long_rows(dtype):
+    """Rows of two million logits (fourteen times the largest vocabulary of the paper's models):
+    many batches per block when rows are whole, and every slice far beyond one batch when the few
+    rows are split; the winners sit in the last elements of the row, and ids need 21 bits."""
+    V = (1 << 21) + 37
+    g = torch.Generator(device=DEV); g.manual_seed(21)
+    z = (torch.randn((5, V), generator=g, device=DEV) * 3).to(dtype)
+    z[0, V - 1] = 40.0
+    z[0, V - 2] = 39.0
+    z[1, V - 3] = 25.0
+    z[2, 0] = 33.0
+    z[2, V - 1] = 33.0                                  # a tie across the whole row: the lower id leads
+    tok = np.array([[-1, V - 1, V - 3, 0, V - 1]], np.int32)
+    parent = np.array([[-1, 0, 1, 2, 2]], np.int32)
+    ref = orc.verify_tree(synth.to_numpy_bits(z), tok, parent, 0.9)
+    got = mars.to_host(mars.verify_tree(z, tok, parent, 0.9, debug=True))
+    assert_same(got, ref, KEYS_TREE, "long rows")
+    assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32))
+    assert ref["top2_id"][0].tolist() == [V - 1, V - 2] and ref["top2_id"][2].tolist() == [0, V - 1]
+    assert ref["accept_len"][0] >= 2
+    val, idx = mars.topk_rows(z, 10)
+    torch.cuda.synchronize()
+    rv, ri = orc.topk(synth.to_numpy_bits(z), 10)
+    assert np.array_equal(idx.cpu().numpy(), ri) and np.array_equal(val.cpu().numpy().view(np.uint32), rv.view(np.uint32))
