@@ -606,29 +606,52 @@ __global__ void __launch_bounds__(128) lmhead_tail_kernel(const LmParams p, cons
         }
         return;
     }
+    // Merge every row's per-chunk records first: a warp per row, lanes across the chunks, so that
+    // the loads are coalesced and independent (one thread per row walking its chunks one load
+    // after the other took 250 us at 66 chunks); the rows' records go to shared memory.
     const int nch = p.n_chunks;
     const Rec *base = p.partial + (size_t)b * t.N * nch;
-    verify_tail(t, b, smem_dyn, [&](int i) {
+    Rec *s_rec = reinterpret_cast<Rec *>(smem_dyn + (tail_smem_bytes(t.N) + 15) / 16 * 16);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int row = warp; row < t.N; row += nwarps) {
         Rec acc = empty_rec();
-        for (int k = 0; k < nch; ++k) acc = merge(acc, base[(size_t)i * nch + k]);
-        return finish_record(acc);
-    });
+        for (int k = lane; k < nch; k += 32) {
+            const int4 w = __ldcg(reinterpret_cast<const int4 *>(base + (size_t)row * nch + k));
+            Rec r;
+            r.z1 = __int_as_float(w.x); r.id1 = w.y; r.z2 = __int_as_float(w.z); r.id2 = w.w;
+            acc = merge(acc, r);
+        }
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) acc = merge(acc, shfl_xor_rec(acc, m));
+        if (lane == 0) s_rec[row] = acc;
+    }
+    __syncthreads();
+    verify_tail(t, b, smem_dyn, [&](int i) { return finish_record(s_rec[i]); });
 }
 
 // Vocabulary shard: merge a row's per-chunk records into one record with global token ids
-// (local id + id_offset), left unfinished for mars_verify_records.  One thread per row.
+// (local id + id_offset), left unfinished for mars_verify_records.  One warp per row, lanes
+// across the chunks.
 __global__ void __launch_bounds__(128) lmhead_records_kernel(const LmParams p, int id_offset, Rec *records)
 {
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= p.M) return;
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= p.M) return;          // warp-uniform
     Rec acc = empty_rec();
     if (*(volatile unsigned *)p.status == 0) {
         const Rec *base = p.partial + (size_t)row * p.n_chunks;
-        for (int k = 0; k < p.n_chunks; ++k) acc = merge(acc, base[k]);
+        for (int k = lane; k < p.n_chunks; k += 32) {
+            const int4 w = __ldcg(reinterpret_cast<const int4 *>(base + k));
+            Rec r;
+            r.z1 = __int_as_float(w.x); r.id1 = w.y; r.z2 = __int_as_float(w.z); r.id2 = w.w;
+            acc = merge(acc, r);
+        }
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) acc = merge(acc, shfl_xor_rec(acc, m));
         if (acc.id1 != kNoId) acc.id1 += id_offset;
         if (acc.id2 != kNoId) acc.id2 += id_offset;
     }
-    records[row] = acc;     // after a device-side timeout every record stays empty
+    if (lane == 0) records[row] = acc;     // after a device-side timeout every record stays empty
 }
 
 // ----------------------------------------------------------------------------- host side
@@ -670,7 +693,8 @@ struct LmShape { int n_mtiles, n_ntiles, n_chunks, n_items, chunk_tiles; };
 
 // Work items are (vocabulary chunk, M-tile) pairs dealt round-robin to `blocks` persistent
 // blocks.  The chunk length is the one that wastes the least of the last round: cost =
-// rounds x tiles per item; ties go to the longer chunk (fewer records per row to merge).  Host-only and independent of the
+// rounds x (tiles per item + half a tile of per-item overhead); ties go to the longer chunk
+// (fewer records per row to merge).  Host-only and independent of the
 // device so that the workspace size is a pure function of the shapes.
 static bool lm_pair_mode()
 {
@@ -689,7 +713,10 @@ static LmShape lm_shape(long long M, int V)
     s.chunk_tiles = 1;
     for (int c = 1; c <= kMaxChunkTiles && c <= s.n_ntiles; ++c) {
         const long long items = (long long)m_units * ((s.n_ntiles + c - 1) / c);
-        const long long cost = ((items + blocks - 1) / blocks) * c;
+        // in half tiles: every item also costs about half a tile (accumulator hand-over, records),
+        // and every chunk is one more record per row for the tail to merge -- without this term a
+        // tie in rounds x tiles could pick one-tile chunks (594 records per row)
+        const long long cost = ((items + blocks - 1) / blocks) * (2 * c + 1);
         if (best_cost < 0 || cost <= best_cost) { best_cost = cost; s.chunk_tiles = c; }
     }
     s.n_chunks = (s.n_ntiles + s.chunk_tiles - 1) / s.chunk_tiles;
@@ -816,7 +843,7 @@ mars_status_t mars_lmhead_top2_shard(const void *hidden, const void *w_shard, co
     LmParams p;
     const mars_status_t gs = lm_launch_gemm(hidden, w_shard, bias_shard, d, B, N, V_local, workspace, st, &p);
     if (gs != MARS_OK) return gs;
-    lmhead_records_kernel<<<(p.M + 127) / 128, 128, 0, st>>>(p, id_offset, (Rec *)records);
+    lmhead_records_kernel<<<(p.M + 3) / 4, 128, 0, st>>>(p, id_offset, (Rec *)records);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
@@ -862,7 +889,7 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
     t.dbg_flags = dbg ? dbg->node_flags : nullptr;
     t.N = N; t.Dcap = Dcap; t.theta = theta; t.flags = flags; t.chain = 0;
 
-    lmhead_tail_kernel<<<B, 128, tail_smem_bytes(N), st>>>(p, t);
+    lmhead_tail_kernel<<<B, 128, (tail_smem_bytes(N) + 15) / 16 * 16 + (size_t)N * sizeof(Rec), st>>>(p, t);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
