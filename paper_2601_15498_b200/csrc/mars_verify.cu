@@ -262,7 +262,14 @@ static mars_status_t run(const void *logits, int64_t ld, mars_dtype_t dt, const 
     const size_t smem = tail_bytes + (p.stage_partials ? stage_bytes : 0);
     cudaError_t le;
     const bool overlap = hook(kHookNoOverlap) == 0;
-    if (dt == MARS_BF16 && sp.S == 1 && R >= kDenseMinRows)
+    // The variant with 4 vectors per batch and 8 blocks per SM: large batches; also whenever a
+    // batch just overflows one wave of the 4-blocks-per-SM variant (592 rows) but fits one of
+    // this one, and for short rows (up to 128 KB: a block lives for a few batches only, and twice
+    // the resident blocks hide twice the start-up and merge phases).
+    const bool dense = dt == MARS_BF16 && sp.S == 1 &&
+                       (R >= kDenseMinRows ||
+                        (R > kTargetBlocks && ((long long)V * 2 <= 128 * 1024 || R <= kTargetBlocks * 3 / 2)));
+    if (dense)
         le = launch_pdl(overlap, verify_kernel<MARS_BF16, kUDense, 8>, dim3(grid), dim3(kThreads), smem, st, p);
     else if (dt == MARS_BF16)
         le = launch_pdl(overlap, verify_kernel<MARS_BF16, kU, 4>, dim3(grid), dim3(kThreads), smem, st, p);
