@@ -518,3 +518,15 @@ def test_very_long_rows(dtype):
     torch.cuda.synchronize()
     rv, ri = orc.topk(synth.to_numpy_bits(z), 10)
     assert np.array_equal(idx.cpu().numpy(), ri) and np.array_equal(val.cpu().numpy().view(np.uint32), rv.view(np.uint32))
+
+
+@pytest.mark.parametrize("B,N,V", [(75, 8, 32000), (100, 7, 151936), (40, 40, 50000)])
+def test_batches_just_above_one_wave_and_short_rows(B, N, V):
+    """Row counts between 593 and about 900, and short rows in larger batches, run the bf16 variant
+    with 8 resident blocks per SM: same bits as the oracle."""
+    w = synth.tree_workload("w8", B, N, 3, 3, V, torch.bfloat16, DEV, 940 + N, 0.9, 3.0, 15.0, 30.0, 0.3)
+    assert w.R > 592
+    ref = orc.verify_tree(synth.to_numpy_bits(w.logits), w.tok, w.parent, w.theta)
+    got = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, debug=True))
+    assert_same(got, ref, KEYS_TREE, w.name)
+    assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32))
