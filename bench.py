@@ -679,7 +679,7 @@ def topk_case(name: str, dev, mars, local: int, steps=None, warm=5, parity_rows:
     return {"workload": f"topk_k{k}_rows{rows}_v{w.V}_{dts}", "rows_per_step": rows, "k": k,
             "logits_bytes_per_step": w.logits_bytes, "us_per_step": us, "step_us": r["step_us"], "steps": r["steps"],
             "timed_region_ms": r["region_ms"], "launch": r["launch"], "l2": "inputs larger than L2",
-            "rows_per_s": rows / (us * 1e-6), "gpu_launches_per_step": 3,
+            "rows_per_s": rows / (us * 1e-6), "gpu_launches_per_step": 1 if rows > 296 else 2,
             "roofline": roof, "read_only_probe": pr, "frac_of_read_only_probe": roof["achieved"] / pr["mean_gbs"],
             "clocks": r["clocks"], "cycles_per_step": r["cycles_per_step"],
             "parity": {"checked_rows": int(len(pick)), "mismatches": bad,

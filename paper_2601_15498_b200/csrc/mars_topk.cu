@@ -28,7 +28,8 @@ constexpr int kTkU = 8;
 constexpr int kTkMaxK = 32;
 constexpr int kTkTargetBlocks = 148 * 4;
 constexpr int kTkMinSliceBytes = kTkThreads * kTkU * 16;
-constexpr int kTkCap = 1024;       // slots of the slice kernel's queue of elements at or above the floor
+constexpr int kTkCap = kTkThreads * 8;   // slots of the slice kernel's queue of elements at or above the floor
+                                         // (the exact fallback reuses them: one vector step per thread)
 
 struct Cand {
     float z;
@@ -40,7 +41,6 @@ struct TopkParams {
     long long ld;
     int V, S, L, k;
     Cand *partial;   // [R*S, k] unused entries {-inf, kNoId}
-    int *redo;       // [R*S] 1: the streaming pass ran out of queue slots for this slice, redo it
     long long nslices;
     float *out_val;      // [R, k] final values, best first
     int32_t *out_id;     // [R, k] final token ids
@@ -73,23 +73,20 @@ __device__ __forceinline__ void warp_list_insert(float &wz, int &wid, int lane, 
 }
 
 // Exact slice selection with per-warp lists; always correct, used when the streaming kernel below
-// runs out of room.  Called by all threads of the block.
+// runs out of room.  Called by all threads of the block.  The caller lends its shared memory:
+//   queue_mem  kTkThreads * 8 candidates (per warp: the candidates of one vector step)
+//   s_list     (kTkThreads / 32) * kTkMaxK candidates (the warps' lists for the final ranking)
+//   s_qn       kTkThreads / 32 counters;  s_bound  block-wide lower bound on the slice's k-th value
 template <int DT>
-__device__ void topk_slice_exact(const TopkParams &p, const long long blk)
+__device__ __noinline__ void topk_slice_exact(const char *rowp, const int lo, const int hi, const int k,
+                                              Cand *out, Cand *queue_mem, Cand *s_list, int *s_qn,
+                                              unsigned *s_bound_p)
 {
     typedef Elem<DT> E;
     constexpr int kWarps = kTkThreads / 32;
-    __shared__ Cand s_queue[kWarps][32 * 8];     // per warp: candidates of one vector step
-    __shared__ int s_qn[kWarps];
-    __shared__ unsigned s_bound;                 // block-wide lower bound on the slice's k-th value
-    __shared__ Cand s_list[kWarps * kTkMaxK];
+    unsigned &s_bound = *s_bound_p;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, k = p.k;
-    const long long row = blk / p.S;
-    const int slice = (int)(blk - row * p.S);
-    const int lo = slice * p.L;
-    const int hi = min(p.V, lo + p.L);
-    const char *rowp = (const char *)p.logits + (size_t)row * (size_t)p.ld * E::kBytes;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     const uintptr_t a0 = (uintptr_t)(rowp + (size_t)lo * E::kBytes);
     int nhead = (int)(((16 - (a0 & 15)) & 15) / E::kBytes);
@@ -110,7 +107,7 @@ __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
     float kth = -INFINITY;      // value / id of the warp's k-th best (entry of lane k-1)
     int kth_id = kNoId;
     float warp_floor = -INFINITY;   // value-only bound from the warp's first batch
-    Cand *queue = s_queue[warp];
+    Cand *queue = queue_mem + warp * (32 * 8);
 
     // Drain the warp's queue into its list (all lanes), then publish the warp's k-th value.
     auto drain = [&]() {
@@ -200,7 +197,6 @@ __device__ void topk_slice_exact(const TopkParams &p, const long long blk)
     // ---- block: the k best of the warps' lists by rank counting ----
     if (lane < kTkMaxK) { s_list[warp * kTkMaxK + lane].z = lane < k ? wz : -INFINITY;
                           s_list[warp * kTkMaxK + lane].id = lane < k ? wid : kNoId; }
-    Cand *out = p.partial + (size_t)blk * k;
     for (int i = tid; i < k; i += kTkThreads) { out[i].z = -INFINITY; out[i].id = kNoId; }
     __syncthreads();
     constexpr int kAll = kWarps * kTkMaxK;
@@ -242,8 +238,8 @@ __device__ void complete_row(float *ov, int32_t *oi, int found, int k)
 //     floor; if another warp has it, that warp or a later one will pick the elements up.
 // So nobody ever waits, the floor trails the stream by at most a few elements, about
 // k (1 + ln(batches)) elements reach the queue on unordered data, and the list is the result.
-// If the queue fills up (adversarially ordered rows), the slice is flagged and topk_finish_kernel
-// redoes it with topk_slice_exact.
+// If the queue fills up (adversarially ordered rows), the block redoes its slice with
+// topk_slice_exact.
 template <int DT>
 __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkParams p)
 {
@@ -251,9 +247,11 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     constexpr int kWarps = kTkThreads / 32;
     __shared__ __align__(8) Cand s_cand[kTkCap];
     __shared__ __align__(8) Cand s_list[kTkMaxK];
+    __shared__ __align__(8) Cand s_xlist[kWarps * kTkMaxK];    // exact fallback only
     __shared__ float s_top[kWarps * kTkMaxK];
     __shared__ unsigned s_floor;
     __shared__ int s_tail, s_head, s_lock, s_overflow;
+    __shared__ int s_xqn[kWarps];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, k = p.k;
     const long long blk = blockIdx.x;
@@ -273,7 +271,8 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     constexpr int kBatchVecs = kTkThreads * kTkU;
     const int nfull = nvec / kBatchVecs;
 
-    pdl_wait();     // scheduled early (behind the previous call's finish kernel), reads nothing before it is done
+    pdl_launch_dependents();    // the next call's kernel may be scheduled; it waits for this one first thing
+    pdl_wait();     // scheduled early itself (behind the previous call's last kernel), reads nothing before that is done
     uint4 v[kTkU];
     typename E::packed_t q[kTkU];
     // batch 0: issue its loads first, so that the set-up below overlaps their latency
@@ -405,14 +404,28 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
         scan(nfull * kBatchVecs + tid);
     }
     __syncthreads();
-    if (tid == 0) p.redo[blk] = s_overflow;      // flagged slices are redone by topk_finish_kernel
-    if (s_overflow) return;
+    if (s_overflow) {
+        // The queue ran out of room (adversarially ordered data): redo the slice with the exact
+        // per-warp lists, which leave the slice's ordered list in the workspace.
+        const long long xrow = (long long)blockIdx.x / p.S;
+        const int xlo = (int)((long long)blockIdx.x - xrow * p.S) * p.L;
+        topk_slice_exact<DT>((const char *)p.logits + (size_t)xrow * (size_t)p.ld * E::kBytes, xlo,
+                             min(p.V, xlo + p.L), p.k, p.partial + (size_t)blockIdx.x * p.k, s_cand,
+                             s_xlist, s_xqn, &s_floor);
+        __threadfence_block();
+        __syncthreads();
+    }
     if (warp == 0) {
-        drain(true);                             // whatever is still queued
-        __syncwarp();
-        const Cand c = s_list[lane];             // ordered; unused entries are {-inf, kNoId}
+        Cand c; c.z = -INFINITY; c.id = kNoId;   // ordered; unused entries are {-inf, kNoId}
+        if (s_overflow) {
+            if (lane < k) c = p.partial[(size_t)blk * k + lane];
+        } else {
+            drain(true);                         // whatever is still queued
+            __syncwarp();
+            c = s_list[lane];
+        }
         if (p.S > 1) {
-            if (lane < k) p.partial[(size_t)blk * k + lane] = c;
+            if (!s_overflow && lane < k) p.partial[(size_t)blk * k + lane] = c;
         } else {
             // a whole row: the list is the row's result, write it out here
             float *ov = p.out_val + (size_t)row * k;
@@ -426,53 +439,31 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     }
 }
 
-// Finish.  Slices that the streaming pass flagged are redone exactly; the S ordered slice lists of
-// a row are merged, the row is completed if it has fewer than k entries above -inf, and written
-// best first.  Split rows (S > 1) get one block each.  Rows that were not split were already
-// written by the slice kernel unless they were flagged: a small grid looks through the flags, each
-// block at a contiguous range of rows, and usually finds nothing to do.
-template <int DT>
-__global__ void __launch_bounds__(kTkThreads) topk_finish_kernel(const TopkParams p, long long rows,
-                                                                 int rows_per_block)
+// Rows that were split over several blocks: merge the S ordered slice lists of a row, complete the
+// row if it has fewer than k entries above -inf, and write it best first.  One block per row.
+// (Rows that one block streamed whole are written by that block; this kernel is not launched.)
+__global__ void __launch_bounds__(128) topk_merge_kernel(const TopkParams p)
 {
     extern __shared__ Cand s_c[];
     __shared__ int s_found;
     pdl_launch_dependents();     // the next call's slice kernel may be scheduled (it waits for this one)
-    const int k = p.k, S = p.S, n = S * k;
-    const long long r0 = (long long)blockIdx.x * rows_per_block;
-    const long long r1 = min(rows, r0 + rows_per_block);
-    if (S == 1) {
-        int mine = 0;
-        for (long long r = r0 + threadIdx.x; r < r1; r += blockDim.x) mine |= p.redo[r];
-        if (!__syncthreads_or(mine)) return;
+    const int k = p.k, n = p.S * k;
+    const long long row = blockIdx.x;
+    const Cand *src = p.partial + (size_t)row * n;
+    if (threadIdx.x == 0) s_found = 0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
+    __syncthreads();
+    float *ov = p.out_val + (size_t)row * k;
+    int32_t *oi = p.out_id + (size_t)row * k;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const Cand c = s_c[i];
+        if (c.id == kNoId) continue;
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (s_c[j].id != kNoId && beats(s_c[j].z, s_c[j].id, c.z, c.id)) ? 1 : 0;
+        if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
     }
-    for (long long row = r0; row < r1; ++row) {
-        bool any_redo = false;
-        for (int sl = 0; sl < S; ++sl) any_redo |= p.redo[row * S + sl] != 0;      // block-uniform
-        if (S == 1 && !any_redo) continue;
-        __syncthreads();             // shared arrays may still be in use from the previous row
-        if (any_redo) {
-            for (int sl = 0; sl < S; ++sl)
-                if (p.redo[row * S + sl]) topk_slice_exact<DT>(p, row * S + sl);
-            __threadfence_block();
-            __syncthreads();
-        }
-        const Cand *src = p.partial + (size_t)row * n;
-        if (threadIdx.x == 0) s_found = 0;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
-        __syncthreads();
-        float *ov = p.out_val + (size_t)row * k;
-        int32_t *oi = p.out_id + (size_t)row * k;
-        for (int i = threadIdx.x; i < n; i += blockDim.x) {
-            const Cand c = s_c[i];
-            if (c.id == kNoId) continue;
-            int rank = 0;
-            for (int j = 0; j < n; ++j) rank += (s_c[j].id != kNoId && beats(s_c[j].z, s_c[j].id, c.z, c.id)) ? 1 : 0;
-            if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
-        }
-        __syncthreads();
-        if (threadIdx.x == 0 && s_found < k) complete_row(ov, oi, s_found, k);
-    }
+    __syncthreads();
+    if (threadIdx.x == 0 && s_found < k) complete_row(ov, oi, s_found, k);
 }
 
 struct TkSplit { int S, L; };
@@ -512,7 +503,7 @@ size_t mars_topk_workspace_bytes(int64_t rows, int V, mars_dtype_t dt, int k)
 {
     if (!mars::topk_supported(rows, V, (int)dt, k)) return 0;
     const mars::TkSplit sp = mars::topk_split(rows, V, (int)dt);
-    return (size_t)rows * sp.S * (k * sizeof(mars::Cand) + sizeof(int));
+    return (size_t)rows * sp.S * (k * sizeof(mars::Cand));
 }
 
 mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, int64_t rows, int V, int k,
@@ -526,14 +517,13 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
     if ((uintptr_t)logits % es) return MARS_ERR_INVALID_ARG;
     const TkSplit sp = topk_split(rows, V, (int)dt);
     if (rows * sp.S > 0x7fffffffll) return MARS_ERR_UNSUPPORTED;
-    const size_t need = (size_t)rows * sp.S * (k * sizeof(Cand) + sizeof(int));
+    const size_t need = (size_t)rows * sp.S * (k * sizeof(Cand));
     if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < need) return MARS_ERR_WORKSPACE;
     TopkParams p;
     p.logits = logits; p.ld = ld; p.V = V; p.S = sp.S; p.L = sp.L; p.k = k;
     p.partial = (Cand *)workspace;
     p.nslices = rows * sp.S;
     p.out_val = out_val; p.out_id = out_id;
-    p.redo = (int *)((char *)workspace + (size_t)p.nslices * k * sizeof(Cand));
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const unsigned grid = (unsigned)(rows * sp.S);
     {
@@ -543,13 +533,8 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
             : launch_pdl(overlap, topk_slice_kernel<MARS_FP32>, dim3(grid), dim3(kTkThreads), 0, st, p);
         if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
     }
-    const size_t fsmem = (size_t)sp.S * k * sizeof(Cand);
-    const long long fgrid = (sp.S > 1 || rows < 148 * 2) ? rows : 148 * 2;
-    const int rows_per_block = (int)((rows + fgrid - 1) / fgrid);
-    if (dt == MARS_BF16)
-        topk_finish_kernel<MARS_BF16><<<(unsigned)fgrid, kTkThreads, fsmem, st>>>(p, (long long)rows, rows_per_block);
-    else
-        topk_finish_kernel<MARS_FP32><<<(unsigned)fgrid, kTkThreads, fsmem, st>>>(p, (long long)rows, rows_per_block);
+    if (sp.S > 1)
+        topk_merge_kernel<<<(unsigned)rows, 128, (size_t)sp.S * k * sizeof(Cand), st>>>(p);
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
