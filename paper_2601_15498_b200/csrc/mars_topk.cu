@@ -7,9 +7,10 @@
 // instructions and skipped unless it reaches the floor, a lower bound on the slice's k-th value.
 // Two forms of the slice selection follow: the streaming one with a queue and one ordered list
 // per block that no warp ever waits for (topk_slice_kernel), and one with per-warp ordered lists
-// that a block falls back to when its queue fills up (topk_slice_exact).  A second small kernel
-// merges the slices of a row, completes rows that have fewer than k entries above -inf, and
-// writes best first.
+// that a block falls back to when its queue fills up (topk_slice_exact).  A block that streamed
+// a whole row writes the row's result itself (one launch per call); only rows split over several
+// blocks take a second small kernel that merges the slices' lists.  Either one completes rows
+// that have fewer than k entries above -inf and writes best first.
 //
 // Total order as everywhere in the library: larger value first, lower token id first among
 // equal values, NaN counts as -inf, -0 is reported as +0.
