@@ -344,9 +344,13 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     if (tid < nhead) { float x = E::scalar(rowp, lo + tid); if (x > -INFINITY) append(x, lo + tid); }
     if (tid < ntail) { float x = E::scalar(rowp, tlo + tid); if (x > -INFINITY) append(x, tlo + tid); }
 
-    // k-th largest of the 256 first-batch maxima.  A lane can only be among the block's k largest
-    // if it is among its warp's k largest: those go to the table, ordered.
+    // First floor: the k-th largest of the threads' first-batch maxima, or a value just below it.
+    // Each warp enters its m = min(k, 4 + k/4) largest maxima, ordered, into a table and the
+    // k-th largest table entry is taken: the table is a subset of the maxima (8 m >= k entries),
+    // so its k-th largest never exceeds theirs, and it falls short of it only when one warp
+    // holds more than m of the block's k largest (k = 32: 12 of 32 in one of 8 warps).
     {
+        const int m = min(k, 4 + (k >> 2));
         const float mine = (bm == bm) ? bm : -INFINITY;
         int wrank = 0;
 #pragma unroll
@@ -354,9 +358,9 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
             const float o = __shfl_sync(0xffffffffu, mine, j);
             wrank += (o > mine || (o == mine && j < lane)) ? 1 : 0;
         }
-        if (wrank < k) s_top[warp * k + wrank] = mine;
+        if (wrank < m) s_top[warp * m + wrank] = mine;
         __syncthreads();
-        const int nt = kWarps * k;
+        const int nt = kWarps * m;
         if (tid < nt) {
             const float t = s_top[tid];
             int rank = 0;
