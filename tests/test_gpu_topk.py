@@ -107,3 +107,18 @@ def test_topk_back_to_back_calls_share_a_workspace():
         rv, ri = want[i & 1]
         assert np.array_equal(outs[i][1].cpu().numpy(), ri), i
         assert np.array_equal(outs[i][0].cpu().numpy().view(np.uint32), rv.view(np.uint32)), i
+
+
+@pytest.mark.parametrize("k,dtype", [(10, torch.bfloat16), (32, torch.bfloat16), (10, torch.float32)])
+def test_topk_full_bench_batch_every_row(k, dtype):
+    """The batch the bench times (7 680 rows of 151 936 logits, one launch, one block per row):
+    every row against the oracle, values and ids."""
+    w = synth.cfg3(DEV, seed=5, B=128, dtype=dtype)
+    assert w.R == 7680
+    val, idx = mars.topk_rows(w.logits, k)
+    torch.cuda.synchronize()
+    val, idx = val.cpu().numpy(), idx.cpu().numpy()
+    for lo in range(0, w.R, 1920):                        # the oracle takes the rows in four parts
+        rv, ri = orc.topk(synth.to_numpy_bits(w.logits[lo:lo + 1920]), k)
+        assert np.array_equal(idx[lo:lo + 1920], ri), (k, lo)
+        assert np.array_equal(val[lo:lo + 1920].view(np.uint32), rv.view(np.uint32)), (k, lo)
