@@ -27,6 +27,7 @@ namespace mars {
 constexpr int kTkThreads = 256;
 constexpr int kTkU = 8;
 constexpr int kTkMaxK = 32;
+constexpr int kTkMergeThreads = 512;   // merge kernel: one entry per thread for most rows
 constexpr int kTkTargetBlocks = 148 * 4;
 constexpr int kTkMinSliceBytes = kTkThreads * kTkU * 16;
 constexpr int kTkCap = kTkThreads * 8;   // slots of the slice kernel's queue of elements at or above the floor
@@ -447,24 +448,58 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
 // Rows that were split over several blocks: merge the S ordered slice lists of a row, complete the
 // row if it has fewer than k entries above -inf, and write it best first.  One block per row.
 // (Rows that one block streamed whole are written by that block; this kernel is not launched.)
-__global__ void __launch_bounds__(128) topk_merge_kernel(const TopkParams p)
+// The lists prove lower bounds on the row's k-th value (see below); only entries at or above
+// the largest bound can be in the result or ahead of one that is, so only they are kept and
+// ranked against each other (of up to S k entries, k plus a few dozen).
+__global__ void __launch_bounds__(kTkMergeThreads) topk_merge_kernel(const TopkParams p)
 {
-    extern __shared__ Cand s_c[];
-    __shared__ int s_found;
+    extern __shared__ Cand s_c[];            // [n] the slices' lists, then [n] the entries kept
+    __shared__ int s_found, s_nkeep;
+    __shared__ unsigned s_thr;
     pdl_launch_dependents();     // the next call's slice kernel may be scheduled (it waits for this one)
     const int k = p.k, n = p.S * k;
+    Cand *s_keep = s_c + n;
     const long long row = blockIdx.x;
     const Cand *src = p.partial + (size_t)row * n;
-    if (threadIdx.x == 0) s_found = 0;
+    if (threadIdx.x == 0) { s_found = 0; s_nkeep = 0; s_thr = tk_enc(-INFINITY); }
+    pdl_wait();                  // scheduled while the slice kernel runs: its lists are complete after this
     for (int i = threadIdx.x; i < n; i += blockDim.x) s_c[i] = src[i];
     __syncthreads();
-    float *ov = p.out_val + (size_t)row * k;
-    int32_t *oi = p.out_id + (size_t)row * k;
+    // Two lower bounds on the row's k-th value: the last entry of any full list, and, with
+    // pp + 1 = ceil(k / S) and m = ceil(k / (pp + 1)), the m-th largest of the lists' entries at
+    // position pp (m lists hold pp + 1 entries each at or above it: k or more in all).
+    const int pp = (k + p.S - 1) / p.S - 1, m = (k + pp) / (pp + 1);
+    for (int sl = threadIdx.x; sl < p.S; sl += blockDim.x) {
+        const Cand last = s_c[sl * k + k - 1];
+        if (last.id != kNoId) atomicMax(&s_thr, tk_enc(last.z));
+        const Cand a = s_c[sl * k + pp];
+        if (a.id != kNoId) {
+            int ahead = 0;
+            for (int s2 = 0; s2 < p.S; ++s2) {
+                const Cand b = s_c[s2 * k + pp];
+                ahead += (b.id != kNoId && (b.z > a.z || (b.z == a.z && s2 < sl))) ? 1 : 0;
+            }
+            if (ahead == m - 1) atomicMax(&s_thr, tk_enc(a.z));
+        }
+    }
+    __syncthreads();
+    const float thr = tk_dec(s_thr);
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const Cand c = s_c[i];
-        if (c.id == kNoId) continue;
+        if (c.id != kNoId && c.z >= thr) s_keep[atomicAdd(&s_nkeep, 1)] = c;
+    }
+    __syncthreads();
+    const int nk = s_nkeep;
+    float *ov = p.out_val + (size_t)row * k;
+    int32_t *oi = p.out_id + (size_t)row * k;
+    for (int i = threadIdx.x; i < nk; i += blockDim.x) {
+        const Cand c = s_keep[i];
         int rank = 0;
-        for (int j = 0; j < n; ++j) rank += (s_c[j].id != kNoId && beats(s_c[j].z, s_c[j].id, c.z, c.id)) ? 1 : 0;
+#pragma unroll 8
+        for (int j = 0; j < nk; ++j) {
+            const Cand o = s_keep[j];
+            rank += beats(o.z, o.id, c.z, c.id) ? 1 : 0;
+        }
         if (rank < k) { ov[rank] = c.z + 0.0f; oi[rank] = c.id; atomicAdd(&s_found, 1); }
     }
     __syncthreads();
@@ -538,8 +573,12 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
             : launch_pdl(overlap, topk_slice_kernel<MARS_FP32>, dim3(grid), dim3(kTkThreads), 0, st, p);
         if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
     }
-    if (sp.S > 1)
-        topk_merge_kernel<<<(unsigned)rows, 128, (size_t)sp.S * k * sizeof(Cand), st>>>(p);
+    if (sp.S > 1) {
+        const bool overlap = hook(kHookNoOverlap) == 0;
+        const cudaError_t le = launch_pdl(overlap, topk_merge_kernel, dim3((unsigned)rows), dim3(kTkMergeThreads),
+                                          2 * (size_t)sp.S * k * sizeof(Cand), st, p);
+        if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
+    }
     return cudaGetLastError() == cudaSuccess ? MARS_OK : MARS_ERR_CUDA;
 }
 
