@@ -530,3 +530,46 @@ def test_batches_just_above_one_wave_and_short_rows(B, N, V):
     got = mars.to_host(mars.verify_tree(w.logits, w.tok, w.parent, w.theta, debug=True))
     assert_same(got, ref, KEYS_TREE, w.name)
     assert np.array_equal(got["top2_val"].view(np.uint32), ref["top2_val"].view(np.uint32))
+
+
+def test_default_calls_are_ordered_behind_a_producer_that_rewrites_the_logits():
+    """Without MARS_LOGITS_READY a call may be scheduled early but reads nothing before its
+    predecessor on the stream is done.  One logits buffer is rewritten in place by a copy kernel
+    between calls of three different entry points (deterministic tree, top-k, stochastic tree),
+    thirty rounds with nothing in between; every call must see exactly the contents that stream
+    order gives it."""
+    B, N, V = 24, 10, 40000
+    ws = [synth.tree_workload(f"mix{j}", B, N, 4, 3, V, torch.bfloat16, DEV, 940 + j, 0.9, 3.0, 15.0, 30.0, 0.3)
+          for j in range(2)]
+    hosts = [synth.to_numpy_bits(w.logits) for w in ws]
+    tok = torch.as_tensor(ws[0].tok, device=DEV)
+    par = torch.as_tensor(ws[0].parent, device=DEV)
+    u = synth.make_uniforms(B, N, 7)
+    u_dev = torch.as_tensor(u, device=DEV)
+    ref_tree = [orc.verify_tree(h, ws[0].tok, ws[0].parent, 0.9) for h in hosts]
+    ref_topk = [orc.topk(h, 10) for h in hosts]
+    ref_st = [orc.verify_tree_stochastic(h, ws[0].tok, ws[0].parent, u, 0.9, 1.0) for h in hosts]
+    live = torch.empty_like(ws[0].logits)
+    rounds = 30
+    o_tree = [mars.alloc_outputs(B, N, N - 1, DEV, debug=True) for _ in range(rounds)]
+    o_topk = [(torch.empty((B * N, 10), dtype=torch.float32, device=DEV),
+               torch.empty((B * N, 10), dtype=torch.int32, device=DEV)) for _ in range(rounds)]
+    o_st = [mars.alloc_stochastic_outputs(B, N, N - 1, DEV, debug=True) for _ in range(rounds)]
+    work = torch.zeros(mars.workspace_bytes(B, N, V, mars.BF16), dtype=torch.uint8, device=DEV)
+    work_k = torch.empty(int(mars.lib().mars_topk_workspace_bytes(B * N, V, mars.BF16, 10)), dtype=torch.uint8, device=DEV)
+    work_s = torch.empty(int(mars.lib().mars_stochastic_workspace_bytes(B, N, V, mars.BF16)), dtype=torch.uint8, device=DEV)
+    torch.cuda.synchronize()
+    for i in range(rounds):
+        live.copy_(ws[i & 1].logits)                       # the producer: rewrites the rows in place
+        mars.verify_tree(live, tok, par, 0.9, workspace=work, out=o_tree[i])
+        mars.topk_rows(live, 10, workspace=work_k, out=o_topk[i])
+        mars.verify_tree_stochastic(live, tok, par, u_dev, 0.9, 1.0, workspace=work_s, out=o_st[i])
+    torch.cuda.synchronize()
+    import stochastic_checks as ts
+    for i in range(rounds):
+        j = i & 1
+        assert_same(mars.to_host(o_tree[i]), ref_tree[j], KEYS_TREE, f"round {i} tree")
+        assert np.array_equal(o_topk[i][1].cpu().numpy(), ref_topk[j][1]), f"round {i} top-k ids"
+        assert np.array_equal(o_topk[i][0].cpu().numpy().view(np.uint32), ref_topk[j][0].view(np.uint32)), i
+        ts.compare(mars.to_host(o_st[i]), ref_st[j], ws[0].tok, ws[0].parent,
+                   ws[j].logits.float().cpu().numpy().astype(np.float64), u, 1.0, f"round {i} stochastic")
