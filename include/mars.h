@@ -546,6 +546,8 @@ mars_status_t mars_device_check(int *sm_count, int *sm_tuned);
  *         2: blocks per cluster of the stochastic tail kernel (1, 2, 4 or 8)
  *         3: value 1 launches every kernel in plain stream order (no programmatic overlap of
  *            consecutive calls; a measurement aid)
+ *         4: mars_topk_rows: 1 = 8 vectors per batch and 4 blocks per SM, 2 = 4 vectors per
+ *            batch and 6 blocks per SM, whatever the size
  *   value 0 clears the hook.  Returns the previous value, or -1 for an unknown hook / negative value.
  */
 int mars_test_hook(int which, int value);

@@ -27,6 +27,7 @@ namespace mars {
 constexpr int kTkThreads = 256;
 constexpr int kTkU = 8;
 constexpr int kTkMaxK = 32;
+constexpr int kTkDenseMinRows = 148 * 24;   // rows from which the 6-blocks-per-SM shape is considered
 constexpr int kTkMergeThreads = 512;   // merge kernel: one entry per thread for most rows
 constexpr int kTkTargetBlocks = 148 * 4;
 constexpr int kTkMinSliceBytes = kTkThreads * kTkU * 16;
@@ -242,8 +243,8 @@ __device__ void complete_row(float *ov, int32_t *oi, int found, int k)
 // k (1 + ln(batches)) elements reach the queue on unordered data, and the list is the result.
 // If the queue fills up (adversarially ordered rows), the block redoes its slice with
 // topk_slice_exact.
-template <int DT>
-__global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkParams p)
+template <int DT, int U, int MINB>
+__global__ void __launch_bounds__(kTkThreads, MINB) topk_slice_kernel(const TopkParams p)
 {
     typedef Elem<DT> E;
     constexpr int kWarps = kTkThreads / 32;
@@ -270,16 +271,16 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
     const int tlo = vlo + nvec * E::kVec;
     const int ntail = max(hi - tlo, 0);
     const uint4 *vbase = (const uint4 *)(rowp + (size_t)vlo * E::kBytes);
-    constexpr int kBatchVecs = kTkThreads * kTkU;
+    constexpr int kBatchVecs = kTkThreads * U;
     const int nfull = nvec / kBatchVecs;
 
     pdl_launch_dependents();    // the next call's kernel may be scheduled; it waits for this one first thing
     pdl_wait();     // scheduled early itself (behind the previous call's last kernel), reads nothing before that is done
-    uint4 v[kTkU];
-    typename E::packed_t q[kTkU];
+    uint4 v[U];
+    typename E::packed_t q[U];
     // batch 0: issue its loads first, so that the set-up below overlaps their latency
-    float bm = (nfull > 0) ? load_batch<DT, kTkU, false>(vbase, tid, nvec, v, q)
-                           : load_batch<DT, kTkU, true>(vbase, tid, nvec, v, q);
+    float bm = (nfull > 0) ? load_batch<DT, U, false>(vbase, tid, nvec, v, q)
+                           : load_batch<DT, U, true>(vbase, tid, nvec, v, q);
     {   // empty slots carry kNoId so that a reader can tell a reserved slot from a written one
         Cand e; e.z = -INFINITY; e.id = kNoId;
         for (int i = tid; i < kTkCap; i += kTkThreads) s_cand[i] = e;
@@ -379,7 +380,7 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
         bool appended = false;
         if (bm >= floor_v) {
 #pragma unroll
-            for (int u = 0; u < kTkU; ++u) {
+            for (int u = 0; u < U; ++u) {
                 if (E::to_float(q[u]) >= floor_v) {
                     unsigned em = 0;
 #pragma unroll
@@ -402,11 +403,11 @@ __global__ void __launch_bounds__(kTkThreads, 4) topk_slice_kernel(const TopkPar
 
     scan(tid);
     for (int bi = 1; bi < nfull; ++bi) {
-        bm = load_batch<DT, kTkU, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
+        bm = load_batch<DT, U, false>(vbase, bi * kBatchVecs + tid, nvec, v, q);
         scan(bi * kBatchVecs + tid);
     }
     if (nfull > 0 && nfull * kBatchVecs < nvec) {
-        bm = load_batch<DT, kTkU, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
+        bm = load_batch<DT, U, true>(vbase, nfull * kBatchVecs + tid, nvec, v, q);
         scan(nfull * kBatchVecs + tid);
     }
     __syncthreads();
@@ -568,9 +569,22 @@ mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, in
     const unsigned grid = (unsigned)(rows * sp.S);
     {
         const bool overlap = hook(kHookNoOverlap) == 0;
-        const cudaError_t le = (dt == MARS_BF16)
-            ? launch_pdl(overlap, topk_slice_kernel<MARS_BF16>, dim3(grid), dim3(kTkThreads), 0, st, p)
-            : launch_pdl(overlap, topk_slice_kernel<MARS_FP32>, dim3(grid), dim3(kTkThreads), 0, st, p);
+        // Two shapes of the same kernel.  8 vectors per batch and 4 blocks per SM is the faster
+        // one nearly everywhere; with k above 16 on many long bf16 rows the kernel is bound by
+        // instruction issue in its list and queue code, and 4 vectors per batch with 6 blocks per
+        // SM (40 registers) gives the schedulers more warps to choose from (k = 32: 6-12 % faster
+        // from 3 552 rows of 151 936 on; 15-20 % slower on rows of 32 000, slower at k = 10).
+        const int variant = hook(kHookTopkVariant);
+        const bool dense = variant ? variant == 2
+                                   : (dt == MARS_BF16 && sp.S == 1 && k > 16 && V >= 65536 &&
+                                      rows >= kTkDenseMinRows);
+        const cudaError_t le =
+            dense ? ((dt == MARS_BF16)
+                         ? launch_pdl(overlap, topk_slice_kernel<MARS_BF16, 4, 6>, dim3(grid), dim3(kTkThreads), 0, st, p)
+                         : launch_pdl(overlap, topk_slice_kernel<MARS_FP32, 4, 6>, dim3(grid), dim3(kTkThreads), 0, st, p))
+                  : ((dt == MARS_BF16)
+                         ? launch_pdl(overlap, topk_slice_kernel<MARS_BF16, kTkU, 4>, dim3(grid), dim3(kTkThreads), 0, st, p)
+                         : launch_pdl(overlap, topk_slice_kernel<MARS_FP32, kTkU, 4>, dim3(grid), dim3(kTkThreads), 0, st, p));
         if (le != cudaSuccess) { (void)cudaGetLastError(); return MARS_ERR_CUDA; }
     }
     if (sp.S > 1) {

@@ -114,7 +114,7 @@ def lib() -> ctypes.CDLL:
     return _lib
 
 
-HOOK_FORCE_SPLIT, HOOK_LMHEAD_SINGLE_BLOCK, HOOK_STOCH_TAIL_CLUSTER, HOOK_NO_OVERLAP = 0, 1, 2, 3
+HOOK_FORCE_SPLIT, HOOK_LMHEAD_SINGLE_BLOCK, HOOK_STOCH_TAIL_CLUSTER, HOOK_NO_OVERLAP, HOOK_TOPK_VARIANT = 0, 1, 2, 3, 4
 
 
 def test_hook(which: int, value: int) -> int:

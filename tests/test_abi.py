@@ -110,7 +110,7 @@ def test_hooks_are_set_only_through_the_abi(lib, monkeypatch):
     assert wb(2, 5, 4000, 1) == 256 + 10 * 3 * 16
     assert lib.mars_test_hook(0, 0) == 3
     assert wb(2, 5, 4000, 1) == plain
-    assert lib.mars_test_hook(4, 1) == -1 and lib.mars_test_hook(-1, 1) == -1 and lib.mars_test_hook(0, -2) == -1
+    assert lib.mars_test_hook(5, 1) == -1 and lib.mars_test_hook(-1, 1) == -1 and lib.mars_test_hook(0, -2) == -1
 
 
 @pytest.mark.skipif(__import__("torch").cuda.is_available(), reason="host without a GPU only")

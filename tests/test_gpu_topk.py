@@ -25,6 +25,7 @@ def check(logits, k, V=None):
 @pytest.fixture(autouse=True)
 def _no_forced_split(monkeypatch):
     hooks.clear("HOOK_FORCE_SPLIT")
+    hooks.clear("HOOK_TOPK_VARIANT")
 
 
 @pytest.mark.parametrize("k", [1, 2, 10, 32])
@@ -70,6 +71,23 @@ def test_topk_host_errors():
     for k in (0, 33, 101):
         with pytest.raises(mars.MarsError):
             mars.topk_rows(z, k)
+
+
+@pytest.mark.parametrize("variant", [1, 2])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_topk_both_batch_shapes_of_the_kernel(dtype, variant):
+    """The kernel has two launch shapes (8 vectors per batch at 4 blocks per SM, 4 at 6) and picks
+    by size; both are forced here on whole rows, split rows, ragged and degenerate rows."""
+    hooks.set("HOOK_TOPK_VARIANT", variant)
+    g = torch.Generator(device=DEV); g.manual_seed(variant)
+    for R, V in ((700, 40007), (9, 151936), (650, 2049)):
+        z = (torch.randn((R, V), generator=g, device=DEV) * 3).to(dtype)
+        z[0] = torch.linspace(-8, 8, V, device=DEV).to(dtype)         # overflows the queue
+        z[1] = 0.5
+        z[2] = float("-inf"); z[2, V // 2] = 3.0
+        for k in (1, 10, 32):
+            check(z, k)
+    check(special_rows(4099, dtype), 9)
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
