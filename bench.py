@@ -813,7 +813,8 @@ def lmhead_entry(dev, mars, local: int) -> dict:
             "l2": "L2 flushed (252 MB written, then 252 MB read through it) before every timed step", "positions_per_s": M / (us * 1e-6),
             "gpu_launches_per_step": 2, "tflops": tfs,
             "roofline": {"bound": "tensor", "achieved": tfs, "peak": peak, "unit": "TFLOP/s", "frac": tfs / peak,
-                         "traffic": None, "peak_source": src, "kernel": "mars::lmhead_top2_kernel_pair",
+                         "traffic": ncu_traffic("cfg4") if w.B == 64 else None, "peak_source": src,
+                         "kernel": "mars::lmhead_top2_kernel_pair",
                          "algorithmic_flops_per_launch": flops, "frac_of_2250_nominal": tfs / 2250.0},
             "clocks": r["clocks"], "cycles_per_step": r["cycles_per_step"],
             "parity": c.parity([0, 63])}
@@ -924,7 +925,8 @@ def lmhead_arm(args, rank: int, world: int, local: int):
         "us_per_step": 1e3 * total_ms / steps, "tflops": tfs, "timed_region_ms": total_ms,
         "clocks": r["clocks"], "cycles_per_step": r["cycles_per_step"], "e2e": e2e, "gpu_launches": 2 * steps,
         "roofline": {"bound": "tensor", "achieved": tfs, "peak": peak, "unit": "TFLOP/s",
-                     "frac": tfs / peak, "traffic": None, "peak_source": src,
+                     "frac": tfs / peak, "traffic": ncu_traffic("cfg4") if (w.B == 64 and world == 1) else None,
+                     "peak_source": src,
                      "kernel": "mars::lmhead_top2_kernel_pair", "algorithmic_flops_per_launch": flops},
         "parity": parity, "cpu_baseline": cpu}), flush=True)
     if world > 1:
