@@ -245,7 +245,10 @@ mars_status_t mars_lmhead_verify(const void *hidden, const void *w_vocab, const 
  * above -inf are completed with the lowest unused ids at value -inf.
  *   logits    [rows, ld] of `dt`, first V columns of each row are read.
  *   out_val   float [rows, k], out_id int32 [rows, k]: best first.
- *   workspace mars_topk_workspace_bytes(rows, V, dt, k) bytes, 256-byte aligned.
+ *   workspace mars_topk_workspace_bytes(rows, V, dt, k) bytes, 256-byte aligned; contents need
+ *             not be initialised.  One kernel is enqueued when every row is streamed by one
+ *             block (from 297 rows on), two when rows are split over several blocks (the
+ *             second merges the blocks' lists); nothing is allocated.
  */
 size_t mars_topk_workspace_bytes(int64_t rows, int V, mars_dtype_t dt, int k);
 mars_status_t mars_topk_rows(const void *logits, int64_t ld, mars_dtype_t dt, int64_t rows, int V,
